@@ -1,0 +1,16 @@
+"""CPU oracle for PCG verification -- test infrastructure, not product code.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It shares nothing with the CUDA library and never imports it.
+"""
+from .pcg_oracle import (  # noqa: F401
+    F32,
+    BF16,
+    FLAG_ZERO_RESIDUAL,
+    build,
+    max_threads,
+    softmax,
+    group_probs,
+    verify,
+    OracleResult,
+)
