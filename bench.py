@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the PCG verification hot path (pcg_verify) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C5]
+
+One step = one pcg_verify call over one whole batch of the workload: every drafted position's target and draft
+row is streamed (softmax statistics, group label, label-group masses, accept test), then per sequence the first
+rejection is found and the residual / bonus group and token are drawn.  The default workload is C5 (B=256, K=16,
+V=65536, bf16 logits, 16384 groups of top-6 membership), the configuration the headline metric is quoted on.
+Inputs are seeded synthetic stand-ins for the paper's TTS logits (see paper_2511_13732_b200/workloads.py).
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank verifies its own batch of the same shape (weak
+scaling; sequences are independent, so there is no data-path collective) and the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2511_13732_b200 import workloads as W  # noqa: E402
+
+METRIC = "verified draft positions/sec"
+UNIT = "positions/s"
+FALLBACK_HBM_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
+# dram__bytes_read.sum + dram__bytes_write.sum of one position_kernel launch, from the ncu capture summarised in
+# profiles/ (null until a capture of that workload exists)
+NCU_TRAFFIC_BYTES = {}
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except (OSError, KeyError, ValueError):
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+
+    def start(self):
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+            return self
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        return self
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    bits = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in names.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            pass
+    return local_rank
+
+
+def oracle_leg(cfg, groups, batch, max_seconds=30.0):
+    """Time the CPU oracle, as it stands, on (a bounded sample of) the batch with all host cores."""
+    import oracle
+
+    oracle.build()
+    cores = oracle.max_threads()
+    B = batch.draft_tokens.shape[0]
+    # a quick probe on 8 sequences sizes the sample so that the leg stays bounded
+    t0 = time.perf_counter()
+    oracle.verify(batch.target_logits[:8], batch.draft_logits[:8], batch.draft_tokens[:8], groups.group_ptr,
+                  groups.group_tok, groups.tok_degree, batch.uniforms[:8], batch.temperature, threads=cores)
+    probe = max(time.perf_counter() - t0, 1e-4)
+    nseq = int(min(B, max(8, (max_seconds / 2) / (probe / 8))))
+    t0 = time.perf_counter()
+    oracle.verify(batch.target_logits[:nseq], batch.draft_logits[:nseq], batch.draft_tokens[:nseq], groups.group_ptr,
+                  groups.group_tok, groups.tok_degree, batch.uniforms[:nseq], batch.temperature, threads=cores)
+    dt = time.perf_counter() - t0
+    return {"value": nseq * cfg.K / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {nseq} of {B} sequences of {cfg.name} ({nseq * cfg.K} drafted positions), one pass, "
+                      f"{dt:.3f} s wall, OpenMP over sequences"}, dt, nseq
+
+
+def run_reference(args, cfg, rank):
+    """Reference arm: the CPU oracle on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    groups = W.make_groups(cfg)
+    nseq = min(cfg.B, 64)
+    batch = W.make_batch(cfg, B=nseq)
+    import oracle
+
+    oracle.build()
+    cores = oracle.max_threads()
+
+    def step():
+        oracle.verify(batch.target_logits, batch.draft_logits, batch.draft_tokens, groups.group_ptr, groups.group_tok,
+                      groups.tok_degree, batch.uniforms, batch.temperature, threads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = nseq * cfg.K * args.steps / dt
+    sample = f"each step = first {nseq} of {cfg.B} sequences of {cfg.name} ({nseq * cfg.K} drafted positions)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(cfg),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg):
+    return {"workload": cfg.name, "B": cfg.B, "K": cfg.K, "V": cfg.V, "M": cfg.M, "logits_dtype": cfg.dtype,
+            "temperature": cfg.temperature, "membership": f"{cfg.groups} (mean degree {cfg.degree})",
+            "l2": "not flushed: each step streams the whole batch, larger than the 126 MB L2"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C5", choices=sorted(W.CONFIGS))
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = W.CONFIGS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if args.steps == 2000:
+            args.steps = 5
+        args.warmup = min(args.warmup, 2)
+        run_reference(args, cfg, rank)
+        return
+
+    import torch
+
+    from paper_2511_13732_b200 import binding
+    from paper_2511_13732_b200.sharding import max_over_ranks, rank_sequences
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    binding.load()
+
+    # ---- inputs: this rank's own batch (sequences rank*B .. rank*B+B-1 of the workload's stream) ----
+    groups = W.make_groups(cfg)
+    seqs = rank_sequences(cfg.B, rank, world, weak=True)
+    batch = W.make_batch(cfg, seqs=seqs)
+    handle = binding.Groups(groups.V, groups.group_ptr, groups.group_tok, groups.tok_degree)
+    bf16 = cfg.dtype == "bf16"
+
+    def host(a):
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).pin_memory()
+        return torch.from_numpy(a).pin_memory()
+
+    h_tl, h_dl, h_x, h_u = host(batch.target_logits), host(batch.draft_logits), host(batch.draft_tokens), host(batch.uniforms)
+    tl, dl = h_tl.cuda(non_blocking=True), h_dl.cuda(non_blocking=True)
+    if bf16:
+        tl, dl = tl.view(torch.bfloat16), dl.view(torch.bfloat16)
+    x, u = h_x.cuda(), h_u.cuda()
+    B, K, V, M = cfg.B, cfg.K, cfg.V, groups.M
+    dt_code = binding.PCG_BF16 if bf16 else binding.PCG_F32
+    ws = torch.empty(binding.pcg_verify_workspace_bytes(B, K, V, M, dt_code), dtype=torch.uint8, device="cuda")
+    out = (torch.empty(B, dtype=torch.int32, device="cuda"), torch.empty((B, K + 1), dtype=torch.int32, device="cuda"),
+           torch.empty((B, K + 1), dtype=torch.int32, device="cuda"), torch.empty(B, dtype=torch.int32, device="cuda"))
+    esz = 2 if bf16 else 4
+
+    def step(events=None):
+        binding.pcg_verify(tl, dl, x, handle, u, cfg.temperature, workspace=ws, out=out, stage_events=events)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    # stage events of every timed step (recorded once here so that their handles exist)
+    stage = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for evs in stage:
+        for e in evs:
+            e.record()
+    barrier()
+    sampler = ClockSampler(physical_gpu_index(local_rank)).start()
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(args.steps):
+        step(stage[i])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(t_begin.elapsed_time(t_end), dist)
+    ms_step = ms_total / args.steps
+    pos_ms = statistics.fmean(e[0].elapsed_time(e[1]) for e in stage)
+    term_ms = statistics.fmean(e[1].elapsed_time(e[2]) for e in stage)
+    accept_len = out[0].cpu().numpy()
+
+    # ---- end to end through the host entry point: pinned host inputs in, host outputs back, every step ----
+    arena = torch.empty(binding.pcg_verify_host_arena_bytes(B, K, V, M, dt_code), dtype=torch.uint8, device="cuda")
+    h_out = (torch.empty(B, dtype=torch.int32).pin_memory(), torch.empty((B, K + 1), dtype=torch.int32).pin_memory(),
+             torch.empty((B, K + 1), dtype=torch.int32).pin_memory(), torch.empty(B, dtype=torch.int32).pin_memory())
+
+    def e2e_step():
+        binding.pcg_verify_host(h_tl, h_dl, h_x, handle, h_u, cfg.temperature, arena, h_out)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist) / args.e2e_steps
+    assert np.array_equal(h_out[0].numpy(), accept_len), "host and device entry points disagree"
+    h2d = (B * (2 * K + 1) * V * esz) + B * K * 4 + B * (K + 1) * 8
+    d2h = B * 4 * 2 + B * (K + 1) * 4 * 2
+
+    if rank == 0:
+        peak, peak_src = hbm_peak()
+        alg_bytes = B * K * 2 * V * esz  # per drafted position: one target and one draft row, read once
+        achieved = alg_bytes / (pos_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": world * B * K / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(cfg),
+            "hbm": {"counted_bytes_per_step": B * (2 * K + 1) * V * esz,
+                    "whole_step_gbs": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9,
+                    "whole_step_frac_of_measured_peak": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9 / peak,
+                    "whole_step_frac_of_8tbs": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9 / 8000.0},
+            "roofline": {"bound": "hbm", "kernel": "position_kernel", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": alg_bytes,
+                         "avg_launch_ms": pos_ms},
+            "stages_ms": {"position_kernel": pos_ms, "terminal_kernel": term_ms},
+            "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
+                    "api": "pcg_verify_host (pinned host tensors)"},
+            "gpu_launches": 2 * args.steps,
+            "clocks": clocks,
+            "mean_accept_len": float(accept_len.mean()),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"], _, _ = oracle_leg(cfg, groups, batch)
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

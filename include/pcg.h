@@ -1,0 +1,201 @@
+/*
+ * pcg.h -- C interface of libpcg: batched group-level verification for
+ * speculative decoding with Principled Coarse-Graining (PCG) on NVIDIA B200.
+ *
+ * Letters used throughout (NOTE: the paper's body uses the opposite letters):
+ *   p = TARGET token distribution, q = DRAFT token distribution,
+ *   P[g] / Q[g] = target / draft coarse-grained mass of group g.
+ *
+ * Unless a parameter says HOST, every pointer is DEVICE memory of the device
+ * that was current when the group handle was created; that device must also be
+ * current when a call is made.  All tensors are dense, row-major, contiguous.
+ * Inputs are never written.  No call allocates or frees device memory except
+ * pcg_groups_create / pcg_groups_destroy.  Calls that take a stream only
+ * enqueue work on it and return without synchronising, except where stated.
+ *
+ * Every function returns a pcg_status; errors the host can see (null pointers,
+ * bad sizes, a handle of another device, too small a workspace) are returned
+ * before anything is launched.  Nothing prints, aborts or throws.
+ */
+#ifndef PCG_H
+#define PCG_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PCG_OK = 0,
+    PCG_ERR_INVALID_ARG = 1,    /* null pointer, non-positive size, misaligned base, wrong device */
+    PCG_ERR_INVALID_GROUPS = 2, /* the membership CSR breaks one of its rules (see pcg_csr) */
+    PCG_ERR_UNSUPPORTED = 3,    /* sizes beyond what the kernels are built for (see pcg_groups_create) */
+    PCG_ERR_WORKSPACE = 4,      /* workspace missing, misaligned or smaller than the query says */
+    PCG_ERR_CUDA = 5            /* a CUDA runtime call failed; pcg_last_error() has the text */
+} pcg_status;
+
+typedef enum {
+    PCG_F32 = 0, /* IEEE float32 logits */
+    PCG_BF16 = 1 /* bfloat16 logits (upper 16 bits of a float32) */
+} pcg_dtype;
+
+/* CUDA stream handle (a cudaStream_t / CUstream); NULL is the default stream. */
+typedef struct CUstream_st *pcg_stream;
+/* CUDA event handle (a cudaEvent_t / CUevent). */
+typedef struct CUevent_st *pcg_event;
+
+/* Bits of out_flags[b] written by pcg_verify. */
+#define PCG_FLAG_BAD_DRAFT_TOKEN 1 /* a draft token id outside [0,V) was seen and treated as token 0 */
+#define PCG_FLAG_ZERO_RESIDUAL 2   /* a rejection whose residual mass summed to <= 0; drew from P instead */
+#define PCG_FLAG_NONFINITE 4       /* a row's maximum or normaliser was not finite (NaN/+inf logits, or all -inf) */
+
+/* Bits of the `mode` argument of pcg_verify. */
+#define PCG_VERIFY_DEFAULT 0u
+#define PCG_VERIFY_DENSE 1u /* form P and Q of ALL groups at EVERY position (through the workspace) */
+
+/*
+ * Group membership: the Acoustic Similarity Groups as a group->token CSR plus
+ * every token's degree N(t) = number of groups containing it (Sec. 2.2, "let
+ * S(t) := {k : t in G_k} and N(t) := |S(t)|").
+ *
+ * Rules (checked by pcg_groups_create, PCG_ERR_INVALID_GROUPS otherwise):
+ *   group_ptr[0] == 0, non-decreasing, group_ptr[M] == nnz;
+ *   token ids in [0,V), strictly ascending inside a group (no duplicates);
+ *   tok_degree[t] equals the number of groups listing t, and is >= 1 for every
+ *   token (a token in no group would leak probability mass);
+ *   weights, if not NULL: finite, >= 0, and summing to 1 (+-1e-4) over the
+ *   groups of each token (the weight equation of Sec. 2.2).
+ * Empty groups and duplicate groups are allowed.
+ * The three/four arrays may live in HOST or DEVICE memory (they are copied with
+ * cudaMemcpyDefault) and may be freed as soon as pcg_groups_create returns.
+ */
+typedef struct {
+    int32_t V;                 /* vocabulary size */
+    int32_t M;                 /* number of groups */
+    int64_t nnz;               /* number of stored (group, token) pairs */
+    const int32_t *group_ptr;  /* [M+1] */
+    const int32_t *group_tok;  /* [nnz] */
+    const int32_t *tok_degree; /* [V] */
+    const float *weights;      /* [nnz] split weights w_{k,t}, or NULL for the paper's default equal split 1/N(t) */
+} pcg_csr;
+
+/* Opaque handle: device-resident membership in the layouts the kernels want. */
+typedef struct pcg_groups pcg_groups;
+
+typedef struct {
+    int32_t V, M;
+    int64_t nnz;
+    int32_t slices;          /* token slices per row = thread-block cluster size of the aggregation kernels */
+    int32_t slice_len;       /* tokens per slice */
+    int32_t max_group_size;  /* largest |G_g| */
+    int32_t max_degree;      /* largest N(t) */
+    int32_t device;          /* CUDA device ordinal the handle lives on */
+    int32_t has_weights;     /* 1 if general weights were given */
+    int64_t device_bytes;    /* device memory held by the handle */
+} pcg_groups_info_t;
+
+const char *pcg_status_string(pcg_status s);
+
+/* Text of the last error raised on the calling thread ("" if none). The pointer stays valid until the next call. */
+const char *pcg_last_error(void);
+
+/*
+ * Build the handle (the groups are "precomputed once and cached", Sec. 2.2
+ * "Complexity and memory").  One-time set-up, not part of the hot path:
+ * validates the CSR on the host, builds the reverse membership S(t) (ascending
+ * group id -- the "optional reverse indices" of the same paragraph), the 1/N(t)
+ * table and a token-sliced copy of the CSR with 16-bit in-slice token offsets,
+ * uploads them and synchronises the device.
+ *
+ *   slices_hint: 0 = choose automatically; 1, 2, 4 or 8 = force that many token
+ *                slices (= cluster size).  Rounded up if a slice would not fit
+ *                in shared memory.
+ * Limits (PCG_ERR_UNSUPPORTED beyond them): per thread block, slice_len*4 +
+ * M*4 + (M/slices)*4 bytes plus 2 KB must fit in 227 KB of shared memory with
+ * slices <= 8 and slice_len <= 65536; e.g. V <= 262144 with M <= 32768.
+ * Errors: INVALID_ARG (null, V/M < 1), INVALID_GROUPS, UNSUPPORTED, CUDA.
+ */
+pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg_groups **out);
+
+/* Free the handle and its device memory. NULL is allowed. The caller must have synchronised all work using it. */
+void pcg_groups_destroy(pcg_groups *groups);
+
+pcg_status pcg_groups_info(const pcg_groups *groups, pcg_groups_info_t *out);
+
+/*
+ * Coarse-grained group distribution of every row (the coarse-grained
+ * distribution equations of Sec. 2.2):
+ *     out[r, g] = sum_{t in G_g} softmax(logits[r, :] / temperature)[t] * w_{g,t},
+ * w_{g,t} = 1/N(t) unless the handle carries weights.  Each row of out sums to
+ * 1 up to rounding; no renormalisation is applied.
+ *
+ *   logits  [rows, V] of `dtype`; base 16-byte aligned for the vector path
+ *           (other alignments, or V*elemsize not a multiple of 16, use a slower scalar path)
+ *   out     [rows, M] float32, fully overwritten
+ * rows == 0 is a no-op.  Errors: INVALID_ARG (null, rows < 0, temperature <= 0 or not finite, bad dtype,
+ * wrong device), CUDA (launch failure).
+ */
+pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64_t rows, float temperature,
+                           const pcg_groups *groups, float *out, pcg_stream stream);
+
+/* Bytes of workspace pcg_verify needs for these sizes and mode (256-byte aligned base required). Never 0. */
+size_t pcg_verify_workspace_bytes(int32_t B, int32_t K, int32_t V, int32_t M, pcg_dtype dtype, uint32_t mode);
+
+/*
+ * Batched PCG verification: Algorithm 1 from the label draw to the returned
+ * token list, for B sequences of K drafted positions, with all randomness
+ * supplied by the caller.
+ *
+ * For sequence b and drafted position i < K (x = draft_tokens[b,i]):
+ *   label   g = the j-th smallest group id containing x, j = min(floor(u[b,i,0] * N(x)), N(x)-1)
+ *           (with weights: inverse CDF of w_{.,x} over S(x) in ascending group id)   -- group-label coupling
+ *   accept  iff P[g] >= Q[g] or u[b,i,1] * Q[g] < P[g]                               -- min(1, P/Q) acceptance
+ * n_b = first rejected position (K if none).  Terminal draw at position n_b:
+ *   R[g] = max(0, P[g] - Q[g]) if n_b < K (residual), R[g] = P[g] of target row K otherwise (bonus token);
+ *   g* = first g whose inclusive prefix of R exceeds u[b,K,0] * sum(R) (last g with R > 0 if rounding leaves none);
+ *   z  = first token t of G_g* (CSR order) whose inclusive prefix of p(t) w_{g*,t} exceeds u[b,K,1] * its sum.
+ * Emitted: out_tokens[b, i<n_b] = draft token (kept on acceptance), out_tokens[b, n_b] = z, later slots -1;
+ *          out_accept_len[b] = n_b; out_groups likewise (labels, then g*, then -1).
+ *
+ *   target_logits [B, K+1, V], draft_logits [B, K, V] of `dtype`, same alignment rule as pcg_group_probs
+ *   draft_tokens  [B, K] int32          uniforms [B, K+1, 2] float32 in [0,1)
+ *   out_accept_len [B] int32            out_tokens [B, K+1] int32
+ *   out_groups [B, K+1] int32 or NULL   out_flags [B] int32 or NULL (PCG_FLAG_* bits)
+ *   workspace: >= pcg_verify_workspace_bytes(...) bytes, 256-byte aligned, contents irrelevant on entry;
+ *              calls that share a workspace must not overlap on the device
+ *   stage_events: NULL, or 3 events recorded on `stream` before the position kernel, between it and the
+ *              terminal kernel, and after the terminal kernel (for timing the stages)
+ * Results are bit-identical from run to run.  1 <= K <= 32, B >= 0 (B == 0 is a no-op).
+ * Masses below the float32 normal range flush to zero.
+ * Errors: INVALID_ARG, UNSUPPORTED (K > 32), WORKSPACE, CUDA.
+ */
+pcg_status pcg_verify(const void *target_logits, const void *draft_logits, pcg_dtype dtype, int32_t B, int32_t K,
+                      const int32_t *draft_tokens, const pcg_groups *groups, const float *uniforms, float temperature,
+                      int32_t *out_accept_len, int32_t *out_tokens, int32_t *out_groups, int32_t *out_flags,
+                      void *workspace, size_t workspace_bytes, uint32_t mode, pcg_stream stream,
+                      const pcg_event *stage_events);
+
+/* Bytes of device staging memory pcg_verify_host needs (inputs, outputs and the verify workspace). */
+size_t pcg_verify_host_arena_bytes(int32_t B, int32_t K, int32_t V, int32_t M, pcg_dtype dtype, uint32_t mode);
+
+/*
+ * pcg_verify for callers whose tensors live in HOST memory (pinned memory makes
+ * the copies asynchronous and fast; pageable memory works but is slower).
+ * Copies the inputs into `device_arena`, runs pcg_verify there, copies the
+ * outputs back and SYNCHRONISES `stream` before returning.
+ *   target_logits, draft_logits, draft_tokens, uniforms, out_*: HOST pointers, shapes as in pcg_verify
+ *   device_arena: DEVICE memory, >= pcg_verify_host_arena_bytes(...), 256-byte aligned, caller-owned
+ * Errors: as pcg_verify.
+ */
+pcg_status pcg_verify_host(const void *target_logits, const void *draft_logits, pcg_dtype dtype, int32_t B, int32_t K,
+                           const int32_t *draft_tokens, const pcg_groups *groups, const float *uniforms,
+                           float temperature, int32_t *out_accept_len, int32_t *out_tokens, int32_t *out_groups,
+                           int32_t *out_flags, void *device_arena, size_t device_arena_bytes, uint32_t mode,
+                           pcg_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PCG_H */

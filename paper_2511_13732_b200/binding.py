@@ -1,0 +1,226 @@
+"""Thin ctypes binding of libpcg.so: argument marshalling only.
+
+Every function mirrors the C entry point of the same name in ``include/pcg.h``.
+Tensors are torch CUDA tensors (torch is used for device memory and streams
+only); their ``data_ptr()`` is handed to the library unchanged.  There is no
+fallback of any kind: if the shared library is missing or a call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+from . import build as _build
+
+PCG_F32, PCG_BF16 = 0, 1
+FLAG_BAD_DRAFT_TOKEN, FLAG_ZERO_RESIDUAL, FLAG_NONFINITE = 1, 2, 4
+VERIFY_DEFAULT, VERIFY_DENSE = 0, 1
+STATUS_NAMES = {0: "PCG_OK", 1: "PCG_ERR_INVALID_ARG", 2: "PCG_ERR_INVALID_GROUPS", 3: "PCG_ERR_UNSUPPORTED",
+                4: "PCG_ERR_WORKSPACE", 5: "PCG_ERR_CUDA"}
+
+EXPORTS = [
+    "pcg_status_string", "pcg_last_error", "pcg_groups_create", "pcg_groups_destroy", "pcg_groups_info",
+    "pcg_group_probs", "pcg_verify_workspace_bytes", "pcg_verify", "pcg_verify_host_arena_bytes", "pcg_verify_host",
+]
+
+
+class PcgError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+class _Csr(ctypes.Structure):
+    _fields_ = [("V", ctypes.c_int32), ("M", ctypes.c_int32), ("nnz", ctypes.c_int64),
+                ("group_ptr", ctypes.c_void_p), ("group_tok", ctypes.c_void_p), ("tok_degree", ctypes.c_void_p),
+                ("weights", ctypes.c_void_p)]
+
+
+class GroupsInfo(ctypes.Structure):
+    _fields_ = [("V", ctypes.c_int32), ("M", ctypes.c_int32), ("nnz", ctypes.c_int64), ("slices", ctypes.c_int32),
+                ("slice_len", ctypes.c_int32), ("max_group_size", ctypes.c_int32), ("max_degree", ctypes.c_int32),
+                ("device", ctypes.c_int32), ("has_weights", ctypes.c_int32), ("device_bytes", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True):
+    """Load libpcg.so (building it first if it is missing or stale and nvcc is present)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if build_if_missing:
+        try:
+            path = _build.build()
+        except (RuntimeError, FileNotFoundError):
+            if not os.path.exists(path):
+                raise
+    lib = ctypes.CDLL(path)
+    vp, i32, i64, f32, u32, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_uint32,
+                                  ctypes.c_size_t)
+    lib.pcg_status_string.argtypes, lib.pcg_status_string.restype = [ctypes.c_int], ctypes.c_char_p
+    lib.pcg_last_error.argtypes, lib.pcg_last_error.restype = [], ctypes.c_char_p
+    lib.pcg_groups_create.argtypes = [ctypes.POINTER(_Csr), ctypes.c_int, ctypes.POINTER(vp)]
+    lib.pcg_groups_create.restype = ctypes.c_int
+    lib.pcg_groups_destroy.argtypes, lib.pcg_groups_destroy.restype = [vp], None
+    lib.pcg_groups_info.argtypes, lib.pcg_groups_info.restype = [vp, ctypes.POINTER(GroupsInfo)], ctypes.c_int
+    lib.pcg_group_probs.argtypes = [vp, ctypes.c_int, i64, f32, vp, vp, vp]
+    lib.pcg_group_probs.restype = ctypes.c_int
+    lib.pcg_verify_workspace_bytes.argtypes = [i32, i32, i32, i32, ctypes.c_int, u32]
+    lib.pcg_verify_workspace_bytes.restype = sz
+    lib.pcg_verify.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, f32, vp, vp, vp, vp, vp, sz, u32, vp, vp]
+    lib.pcg_verify.restype = ctypes.c_int
+    lib.pcg_verify_host_arena_bytes.argtypes = [i32, i32, i32, i32, ctypes.c_int, u32]
+    lib.pcg_verify_host_arena_bytes.restype = sz
+    lib.pcg_verify_host.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, f32, vp, vp, vp, vp, vp, sz, u32, vp]
+    lib.pcg_verify_host.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _check(status: int):
+    if status != 0:
+        raise PcgError(status, load().pcg_last_error().decode())
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _dev_ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def dtype_code(t) -> int:
+    import torch
+
+    if t.dtype == torch.float32:
+        return PCG_F32
+    if t.dtype == torch.bfloat16 or t.dtype == torch.uint16 or t.dtype == torch.int16:
+        return PCG_BF16
+    raise TypeError(f"logits must be float32 or bfloat16 (or 16-bit integer bit patterns), got {t.dtype}")
+
+
+class Groups:
+    """Owner of a ``pcg_groups`` handle built from host numpy arrays (``pcg_groups_create``)."""
+
+    def __init__(self, V: int, group_ptr, group_tok, tok_degree, weights=None, slices_hint: int = 0):
+        lib = load()
+        self._keep = (np.ascontiguousarray(group_ptr, np.int32), np.ascontiguousarray(group_tok, np.int32),
+                      np.ascontiguousarray(tok_degree, np.int32),
+                      None if weights is None else np.ascontiguousarray(weights, np.float32))
+        gp, gt, dg, w = self._keep
+        csr = _Csr(int(V), int(gp.shape[0] - 1), int(gt.shape[0]), _np_ptr(gp), _np_ptr(gt), _np_ptr(dg), _np_ptr(w))
+        self.handle = ctypes.c_void_p()
+        _check(lib.pcg_groups_create(ctypes.byref(csr), int(slices_hint), ctypes.byref(self.handle)))
+        info = GroupsInfo()
+        _check(lib.pcg_groups_info(self.handle, ctypes.byref(info)))
+        self.info = info
+        self.V, self.M = info.V, info.M
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load().pcg_groups_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def pcg_group_probs(logits, groups: Groups, temperature: float = 1.0, out=None, stream=None):
+    """``pcg_group_probs``: logits [rows, V] (CUDA, float32 or bfloat16) -> float32 [rows, M]."""
+    import torch
+
+    if logits.dim() != 2 or logits.shape[1] != groups.V or not logits.is_contiguous() or not logits.is_cuda:
+        raise ValueError("logits must be a contiguous CUDA tensor [rows, V]")
+    rows = logits.shape[0]
+    if out is None:
+        out = torch.empty((rows, groups.M), dtype=torch.float32, device=logits.device)
+    _check(load().pcg_group_probs(_dev_ptr(logits), dtype_code(logits), rows, float(temperature), groups.handle,
+                                  _dev_ptr(out), _stream_ptr(stream)))
+    return out
+
+
+def pcg_verify_workspace_bytes(B: int, K: int, V: int, M: int, dtype: int, mode: int = 0) -> int:
+    return int(load().pcg_verify_workspace_bytes(B, K, V, M, dtype, mode))
+
+
+def pcg_verify(target_logits, draft_logits, draft_tokens, groups: Groups, uniforms, temperature: float = 1.0,
+               workspace=None, mode: int = 0, stream=None, want_groups: bool = True, want_flags: bool = True,
+               out=None, stage_events=None):
+    """``pcg_verify`` on CUDA tensors.  Returns (accept_len [B], tokens [B,K+1], groups or None, flags or None).
+
+    ``workspace`` is a uint8 CUDA tensor of at least ``pcg_verify_workspace_bytes`` bytes (allocated here if
+    omitted); ``out`` optionally supplies the four output tensors; ``stage_events`` is a list of three
+    ``torch.cuda.Event(enable_timing=True)`` that were recorded at least once (their handles are passed down).
+    """
+    import torch
+
+    B, K1, V = target_logits.shape
+    K = K1 - 1
+    dev = target_logits.device
+    for t, shape in ((draft_logits, (B, K, V)), (draft_tokens, (B, K)), (uniforms, (B, K + 1, 2))):
+        if tuple(t.shape) != shape or not t.is_contiguous() or t.device != dev:
+            raise ValueError(f"expected a contiguous tensor of shape {shape} on {dev}")
+    if not target_logits.is_contiguous() or draft_logits.dtype != target_logits.dtype:
+        raise ValueError("target and draft logits must be contiguous and share a dtype")
+    if draft_tokens.dtype != torch.int32 or uniforms.dtype != torch.float32:
+        raise TypeError("draft_tokens must be int32 and uniforms float32")
+    dt = dtype_code(target_logits)
+    need = pcg_verify_workspace_bytes(B, K, V, groups.M, dt, mode)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    if out is None:
+        accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+        tokens = torch.empty((B, K + 1), dtype=torch.int32, device=dev)
+        grp = torch.empty((B, K + 1), dtype=torch.int32, device=dev) if want_groups else None
+        flags = torch.empty(B, dtype=torch.int32, device=dev) if want_flags else None
+    else:
+        accept_len, tokens, grp, flags = out
+    ev = None
+    if stage_events is not None:
+        ev = (ctypes.c_void_p * 3)(*[ctypes.c_void_p(e.cuda_event) for e in stage_events])
+    _check(load().pcg_verify(_dev_ptr(target_logits), _dev_ptr(draft_logits), dt, B, K, _dev_ptr(draft_tokens),
+                             groups.handle, _dev_ptr(uniforms), float(temperature), _dev_ptr(accept_len),
+                             _dev_ptr(tokens), _dev_ptr(grp), _dev_ptr(flags), _dev_ptr(workspace),
+                             workspace.numel() * workspace.element_size(), mode, _stream_ptr(stream), ev))
+    return accept_len, tokens, grp, flags
+
+
+def pcg_verify_host_arena_bytes(B: int, K: int, V: int, M: int, dtype: int, mode: int = 0) -> int:
+    return int(load().pcg_verify_host_arena_bytes(B, K, V, M, dtype, mode))
+
+
+def pcg_verify_host(target_logits, draft_logits, draft_tokens, groups: Groups, uniforms, temperature: float,
+                    arena, out, mode: int = 0, stream=None):
+    """``pcg_verify_host``: inputs and the four ``out`` tensors are HOST torch tensors (pinned for speed);
+    ``arena`` is a uint8 CUDA tensor of at least ``pcg_verify_host_arena_bytes`` bytes.  Synchronises."""
+    B, K1, V = target_logits.shape
+    K = K1 - 1
+    accept_len, tokens, grp, flags = out
+    _check(load().pcg_verify_host(_dev_ptr(target_logits), _dev_ptr(draft_logits), dtype_code(target_logits), B, K,
+                                  _dev_ptr(draft_tokens), groups.handle, _dev_ptr(uniforms), float(temperature),
+                                  _dev_ptr(accept_len), _dev_ptr(tokens), _dev_ptr(grp), _dev_ptr(flags),
+                                  _dev_ptr(arena), arena.numel() * arena.element_size(), mode, _stream_ptr(stream)))
+    return out

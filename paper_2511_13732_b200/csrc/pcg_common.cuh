@@ -1,0 +1,203 @@
+// Shared device helpers and the group handle of libpcg (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pcg.h"
+
+#ifndef __CUDA_ARCH__
+#define PCG_HOST_ONLY 1
+#endif
+
+namespace pcg {
+
+constexpr float kNegInf = -__builtin_huge_valf();
+
+// Device-resident membership, built once by pcg_groups_create.
+struct GroupsDev {
+    int32_t V, M;
+    int32_t slices;     // C: token slices per row = cluster size of the aggregation kernels
+    int32_t slice_len;  // tokens per slice (multiple of 64)
+    int32_t groups_per_slice;  // ceil(M / C): groups whose totals a CTA of the cluster owns
+    const int32_t *group_ptr;  // [M+1]   original CSR
+    const int32_t *group_tok;  // [nnz]
+    const float *inv_deg;      // [V]     1/N(t)
+    const int32_t *rev_ptr;    // [V+1]   reverse membership S(t), ascending group id
+    const int32_t *rev_grp;    // [nnz]
+    const int32_t *slice_ptr;  // [C][M+1] start of (slice, group) sub-list in slice_tok
+    const uint16_t *slice_tok; // [nnz]   in-slice token offsets, ordered by (slice, group, token)
+    const float *pair_w;       // [nnz] CSR-order weights w_{g,t} or nullptr (equal split)
+    const float *slice_w;      // [nnz] the same in slice order, or nullptr
+    const float *rev_w;        // [nnz] the same in reverse-membership order, or nullptr
+};
+
+}  // namespace pcg
+
+struct pcg_groups {
+    pcg::GroupsDev dev;
+    int64_t nnz;
+    int device;
+    int max_group_size;
+    int max_degree;
+    int64_t device_bytes;
+    void *allocation;  // single device allocation holding every array
+    size_t agg_smem_bytes;  // dynamic shared memory of the aggregation kernels
+};
+
+namespace pcg {
+
+void set_error(const char *fmt, ...);
+pcg_status cuda_fail(cudaError_t e, const char *what);
+
+#ifdef __CUDACC__
+
+// ---- loading 16 bytes of logits and widening them to float -------------------------------------------------
+template <typename T>
+struct Elem;
+template <>
+struct Elem<float> {
+    static constexpr int kPerVec = 4;
+    static __device__ __forceinline__ float widen(float x) { return x; }
+    static __device__ __forceinline__ void unpack(const uint4 &r, float (&v)[4]) {
+        v[0] = __uint_as_float(r.x);
+        v[1] = __uint_as_float(r.y);
+        v[2] = __uint_as_float(r.z);
+        v[3] = __uint_as_float(r.w);
+    }
+};
+template <>
+struct Elem<uint16_t> {  // bfloat16 bit patterns: the upper half of a float
+    static constexpr int kPerVec = 8;
+    static __device__ __forceinline__ float widen(uint16_t x) { return __uint_as_float(((uint32_t)x) << 16); }
+    static __device__ __forceinline__ void unpack(const uint4 &r, float (&v)[8]) {
+        v[0] = __uint_as_float(r.x << 16);
+        v[1] = __uint_as_float(r.x & 0xffff0000u);
+        v[2] = __uint_as_float(r.y << 16);
+        v[3] = __uint_as_float(r.y & 0xffff0000u);
+        v[4] = __uint_as_float(r.z << 16);
+        v[5] = __uint_as_float(r.z & 0xffff0000u);
+        v[6] = __uint_as_float(r.w << 16);
+        v[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+};
+
+// Streaming 128-bit load that does not allocate in L1 (each logit is read once per kernel).
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ float ex2(float x) {  // 2^x, MUFU, flushes subnormal results to zero
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// e = 2^(l*s - ms): the unnormalised softmax term of logit l with s = log2(e)/T and ms = max*s.
+__device__ __forceinline__ float softmax_term(float l, float s, float ms) { return ex2(__fmaf_rn(l, s, -ms)); }
+
+// ---- running (max, sum of 2^((l - max) s)) pairs ------------------------------------------------------------
+struct MaxSum {
+    float m;    // running maximum of the raw logits
+    float acc;  // sum of 2^((l - m) * s) over the logits seen so far
+};
+
+__device__ __forceinline__ MaxSum combine(const MaxSum &a, const MaxSum &b, float s) {
+    MaxSum r;
+    r.m = fmaxf(a.m, b.m);
+    if (r.m == kNegInf) {
+        r.acc = 0.f;
+    } else {
+        r.acc = a.acc * ex2((a.m - r.m) * s) + b.acc * ex2((b.m - r.m) * s);
+    }
+    return r;
+}
+
+// Deterministic block-wide combine: xor butterfly inside a warp, then a fixed-order pass over the warps.
+// `scratch` holds 2*NWARPS floats.  Every thread returns the same pair.
+template <int NT>
+__device__ __forceinline__ MaxSum block_combine(MaxSum v, float s, float *scratch) {
+    constexpr int NW = NT / 32;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        MaxSum w;
+        w.m = __shfl_xor_sync(0xffffffffu, v.m, o);
+        w.acc = __shfl_xor_sync(0xffffffffu, v.acc, o);
+        v = combine(v, w, s);
+    }
+    __syncthreads();  // scratch may still be read by a previous use
+    if ((threadIdx.x & 31) == 0) {
+        scratch[2 * (threadIdx.x >> 5)] = v.m;
+        scratch[2 * (threadIdx.x >> 5) + 1] = v.acc;
+    }
+    __syncthreads();
+    MaxSum r{scratch[0], scratch[1]};
+#pragma unroll
+    for (int w = 1; w < NW; ++w) r = combine(r, MaxSum{scratch[2 * w], scratch[2 * w + 1]}, s);
+    return r;
+}
+
+template <int NT>
+__device__ __forceinline__ float block_sum(float v, float *scratch) {
+    constexpr int NW = NT / 32;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = scratch[0];
+#pragma unroll
+    for (int w = 1; w < NW; ++w) r += scratch[w];
+    return r;
+}
+
+template <int NT>
+__device__ __forceinline__ float block_max(float v, float *scratch) {
+    constexpr int NW = NT / 32;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = scratch[0];
+#pragma unroll
+    for (int w = 1; w < NW; ++w) r = fmaxf(r, scratch[w]);
+    return r;
+}
+
+// Prefix sums (in double) of one value per thread, in thread order.  *incl is this thread's inclusive
+// prefix and *excl is exactly the previous thread's inclusive prefix (0 for thread 0), so the intervals
+// [excl, incl) of consecutive threads tile [0, total) without cracks.  `scratch` holds NWARPS doubles.
+template <int NT>
+__device__ __forceinline__ void block_scan(double v, double *scratch, double *excl, double *incl, double *total) {
+    constexpr int NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        double up = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += up;
+    }
+    double prev = __shfl_up_sync(0xffffffffu, inc, 1);
+    if (lane == 0) prev = 0.0;
+    __syncthreads();
+    if (lane == 31) scratch[warp] = inc;
+    __syncthreads();
+    double base = 0.0, tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+        if (w == warp) base = tot;
+        tot += scratch[w];
+    }
+    *total = tot;
+    *excl = base + prev;
+    *incl = base + inc;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace pcg

@@ -1,0 +1,302 @@
+// Group handle: host-side validation of the membership CSR and construction of the device layouts.
+// One-time set-up (the groups are precomputed once and cached); not part of the verification hot path.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "pcg_common.cuh"
+
+namespace pcg {
+
+static thread_local char g_error[512] = "";
+
+void set_error(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof g_error, fmt, ap);
+    va_end(ap);
+}
+
+pcg_status cuda_fail(cudaError_t e, const char *what) {
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    return PCG_ERR_CUDA;
+}
+
+constexpr size_t kMaxSmem = 227 * 1024;
+constexpr size_t kAggScratch = 2048;
+
+size_t agg_smem_bytes(int slice_len, int M, int slices) {
+    size_t mc = (size_t)(M + slices - 1) / slices;
+    return (size_t)slice_len * 4 + (size_t)M * 4 + mc * 4 + kAggScratch;
+}
+
+}  // namespace pcg
+
+extern "C" const char *pcg_status_string(pcg_status s) {
+    switch (s) {
+        case PCG_OK: return "ok";
+        case PCG_ERR_INVALID_ARG: return "invalid argument";
+        case PCG_ERR_INVALID_GROUPS: return "invalid group membership";
+        case PCG_ERR_UNSUPPORTED: return "unsupported size";
+        case PCG_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case PCG_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+extern "C" const char *pcg_last_error(void) { return pcg::g_error; }
+
+namespace {
+
+struct Carver {  // lays arrays out in one allocation, 256-byte aligned
+    size_t off = 0;
+    size_t take(size_t bytes) {
+        size_t at = off;
+        off = (off + bytes + 255) & ~(size_t)255;
+        return at;
+    }
+};
+
+template <typename T>
+cudaError_t upload(char *base, size_t at, const std::vector<T> &v) {
+    if (v.empty()) return cudaSuccess;
+    return cudaMemcpy(base + at, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+}  // namespace
+
+extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg_groups **out) {
+    using namespace pcg;
+    if (out) *out = nullptr;
+    if (!csr || !out || !csr->group_ptr || !csr->tok_degree || (csr->nnz > 0 && !csr->group_tok)) {
+        set_error("pcg_groups_create: null argument");
+        return PCG_ERR_INVALID_ARG;
+    }
+    const int V = csr->V, M = csr->M;
+    const int64_t nnz = csr->nnz;
+    if (V < 1 || M < 1 || nnz < 0 || nnz > INT32_MAX) {
+        set_error("pcg_groups_create: need V >= 1, M >= 1, 0 <= nnz < 2^31 (V=%d M=%d nnz=%lld)", V, M, (long long)nnz);
+        return PCG_ERR_INVALID_ARG;
+    }
+    if (slices_hint != 0 && slices_hint != 1 && slices_hint != 2 && slices_hint != 4 && slices_hint != 8) {
+        set_error("pcg_groups_create: slices_hint must be 0, 1, 2, 4 or 8");
+        return PCG_ERR_INVALID_ARG;
+    }
+    // Without a usable CUDA device the arrays are taken to be host memory, so that the validation below
+    // still reports what is wrong with them; the call then fails with PCG_ERR_CUDA at the allocation.
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    const bool have_device = (e == cudaSuccess);
+    if (!have_device) (void)cudaGetLastError();
+
+    // ---- bring the CSR to the host (with a device present the arrays may be host or device memory) ----
+    std::vector<int32_t> gptr((size_t)M + 1), gtok((size_t)nnz), deg((size_t)V);
+    std::vector<float> w;
+    if (csr->weights && nnz) w.resize((size_t)nnz);
+    if (have_device) {
+        e = cudaMemcpy(gptr.data(), csr->group_ptr, gptr.size() * 4, cudaMemcpyDefault);
+        if (e == cudaSuccess && nnz) e = cudaMemcpy(gtok.data(), csr->group_tok, gtok.size() * 4, cudaMemcpyDefault);
+        if (e == cudaSuccess) e = cudaMemcpy(deg.data(), csr->tok_degree, deg.size() * 4, cudaMemcpyDefault);
+        if (e == cudaSuccess && !w.empty()) e = cudaMemcpy(w.data(), csr->weights, w.size() * 4, cudaMemcpyDefault);
+        if (e != cudaSuccess) return cuda_fail(e, "copying the membership CSR");
+    } else {
+        memcpy(gptr.data(), csr->group_ptr, gptr.size() * 4);
+        if (nnz) memcpy(gtok.data(), csr->group_tok, gtok.size() * 4);
+        memcpy(deg.data(), csr->tok_degree, deg.size() * 4);
+        if (!w.empty()) memcpy(w.data(), csr->weights, w.size() * 4);
+    }
+
+    // ---- validate ----
+    if (gptr[0] != 0 || gptr[M] != nnz) {
+        set_error("group_ptr[0] must be 0 and group_ptr[M] must equal nnz");
+        return PCG_ERR_INVALID_GROUPS;
+    }
+    std::vector<int32_t> count((size_t)V, 0);
+    int max_group = 0;
+    for (int g = 0; g < M; ++g) {
+        if (gptr[g + 1] < gptr[g]) {
+            set_error("group_ptr decreases at group %d", g);
+            return PCG_ERR_INVALID_GROUPS;
+        }
+        for (int32_t k = gptr[g]; k < gptr[g + 1]; ++k) {
+            int32_t t = gtok[k];
+            if (t < 0 || t >= V) {
+                set_error("token id %d of group %d is outside [0,%d)", t, g, V);
+                return PCG_ERR_INVALID_GROUPS;
+            }
+            if (k > gptr[g] && gtok[k - 1] >= t) {
+                set_error("tokens of group %d are not strictly ascending", g);
+                return PCG_ERR_INVALID_GROUPS;
+            }
+            count[t]++;
+        }
+        max_group = std::max(max_group, gptr[g + 1] - gptr[g]);
+    }
+    int max_deg = 0;
+    for (int t = 0; t < V; ++t) {
+        if (deg[t] != count[t] || deg[t] < 1) {
+            set_error("tok_degree[%d] = %d but the token is listed by %d groups (every token needs >= 1)", t, deg[t],
+                      count[t]);
+            return PCG_ERR_INVALID_GROUPS;
+        }
+        max_deg = std::max(max_deg, deg[t]);
+    }
+
+    // ---- reverse membership S(t), ascending group id (counting sort over the CSR) ----
+    std::vector<int32_t> rptr((size_t)V + 1, 0), rgrp((size_t)nnz);
+    std::vector<float> rw;
+    for (int t = 0; t < V; ++t) rptr[t + 1] = rptr[t] + deg[t];
+    {
+        std::vector<int32_t> fill(rptr.begin(), rptr.end() - 1);
+        if (!w.empty()) rw.resize((size_t)nnz);
+        for (int g = 0; g < M; ++g)
+            for (int32_t k = gptr[g]; k < gptr[g + 1]; ++k) {
+                int32_t at = fill[gtok[k]]++;
+                rgrp[at] = g;
+                if (!w.empty()) rw[at] = w[k];
+            }
+    }
+    if (!w.empty()) {
+        for (int64_t k = 0; k < nnz; ++k)
+            if (!(w[k] >= 0.f) || !std::isfinite(w[k])) {
+                set_error("weights[%lld] is negative or not finite", (long long)k);
+                return PCG_ERR_INVALID_GROUPS;
+            }
+        for (int t = 0; t < V; ++t) {
+            double s = 0;
+            for (int32_t k = rptr[t]; k < rptr[t + 1]; ++k) s += rw[k];
+            if (std::fabs(s - 1.0) > 1e-4) {
+                set_error("weights of token %d sum to %.6f over its groups, not 1", t, s);
+                return PCG_ERR_INVALID_GROUPS;
+            }
+        }
+    }
+
+    // ---- choose the token slicing ----
+    int C = slices_hint ? slices_hint : 1;
+    if (!slices_hint)
+        while (C < 8 && (V + C - 1) / C > 8192) C *= 2;
+    int SL = 0;
+    for (;; C *= 2) {
+        SL = (((V + C - 1) / C) + 63) / 64 * 64;
+        if (SL <= 65536 && agg_smem_bytes(SL, M, C) <= kMaxSmem) break;
+        if (C >= 8) {
+            set_error("V=%d, M=%d do not fit the aggregation kernels' shared memory even with 8 slices", V, M);
+            return PCG_ERR_UNSUPPORTED;
+        }
+    }
+
+    // ---- token-sliced copy of the CSR: sub-lists ordered by (slice, group), 16-bit in-slice offsets ----
+    std::vector<int32_t> sptr((size_t)C * (M + 1));
+    std::vector<uint16_t> stok((size_t)nnz);
+    std::vector<float> sw;
+    if (!w.empty()) sw.resize((size_t)nnz);
+    {
+        int32_t at = 0;
+        std::vector<int32_t> cursor(gptr.begin(), gptr.end() - 1);  // tokens ascend, so each slice is a sub-range
+        for (int c = 0; c < C; ++c) {
+            const int32_t t_end = (int32_t)std::min<int64_t>((int64_t)(c + 1) * SL, V);
+            for (int g = 0; g < M; ++g) {
+                sptr[(size_t)c * (M + 1) + g] = at;
+                int32_t k = cursor[g];
+                for (; k < gptr[g + 1] && gtok[k] < t_end; ++k) {
+                    stok[at] = (uint16_t)(gtok[k] - c * SL);
+                    if (!w.empty()) sw[at] = w[k];
+                    ++at;
+                }
+                cursor[g] = k;
+            }
+            sptr[(size_t)c * (M + 1) + M] = at;
+        }
+    }
+    std::vector<float> inv((size_t)V);
+    for (int t = 0; t < V; ++t) inv[t] = 1.0f / (float)deg[t];
+
+    // ---- one device allocation for everything ----
+    Carver cv;
+    const size_t o_gptr = cv.take(gptr.size() * 4), o_gtok = cv.take(gtok.size() * 4), o_inv = cv.take(inv.size() * 4);
+    const size_t o_rptr = cv.take(rptr.size() * 4), o_rgrp = cv.take(rgrp.size() * 4);
+    const size_t o_sptr = cv.take(sptr.size() * 4), o_stok = cv.take(stok.size() * 2);
+    const size_t o_w = cv.take(w.size() * 4), o_sw = cv.take(sw.size() * 4), o_rw = cv.take(rw.size() * 4);
+    const size_t total = cv.off ? cv.off : 256;
+    void *mem = nullptr;
+    if (!have_device) {
+        set_error("no usable CUDA device (the membership itself is valid)");
+        return PCG_ERR_CUDA;
+    }
+    e = cudaMalloc(&mem, total);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc (group handle)");
+    char *base = (char *)mem;
+    e = upload(base, o_gptr, gptr);
+    if (e == cudaSuccess) e = upload(base, o_gtok, gtok);
+    if (e == cudaSuccess) e = upload(base, o_inv, inv);
+    if (e == cudaSuccess) e = upload(base, o_rptr, rptr);
+    if (e == cudaSuccess) e = upload(base, o_rgrp, rgrp);
+    if (e == cudaSuccess) e = upload(base, o_sptr, sptr);
+    if (e == cudaSuccess) e = upload(base, o_stok, stok);
+    if (e == cudaSuccess) e = upload(base, o_w, w);
+    if (e == cudaSuccess) e = upload(base, o_sw, sw);
+    if (e == cudaSuccess) e = upload(base, o_rw, rw);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        cudaFree(mem);
+        return cuda_fail(e, "uploading the group handle");
+    }
+    pcg_groups *h = new (std::nothrow) pcg_groups();
+    if (!h) {
+        cudaFree(mem);
+        set_error("out of host memory");
+        return PCG_ERR_INVALID_ARG;
+    }
+    h->dev.V = V;
+    h->dev.M = M;
+    h->dev.slices = C;
+    h->dev.slice_len = SL;
+    h->dev.groups_per_slice = (M + C - 1) / C;
+    h->dev.group_ptr = (const int32_t *)(base + o_gptr);
+    h->dev.group_tok = (const int32_t *)(base + o_gtok);
+    h->dev.inv_deg = (const float *)(base + o_inv);
+    h->dev.rev_ptr = (const int32_t *)(base + o_rptr);
+    h->dev.rev_grp = (const int32_t *)(base + o_rgrp);
+    h->dev.slice_ptr = (const int32_t *)(base + o_sptr);
+    h->dev.slice_tok = (const uint16_t *)(base + o_stok);
+    h->dev.pair_w = w.empty() ? nullptr : (const float *)(base + o_w);
+    h->dev.slice_w = w.empty() ? nullptr : (const float *)(base + o_sw);
+    h->dev.rev_w = w.empty() ? nullptr : (const float *)(base + o_rw);
+    h->nnz = nnz;
+    h->device = device;
+    h->max_group_size = max_group;
+    h->max_degree = max_deg;
+    h->device_bytes = (int64_t)total;
+    h->allocation = mem;
+    h->agg_smem_bytes = agg_smem_bytes(SL, M, C);
+    *out = h;
+    return PCG_OK;
+}
+
+extern "C" void pcg_groups_destroy(pcg_groups *groups) {
+    if (!groups) return;
+    cudaFree(groups->allocation);
+    delete groups;
+}
+
+extern "C" pcg_status pcg_groups_info(const pcg_groups *groups, pcg_groups_info_t *out) {
+    if (!groups || !out) {
+        pcg::set_error("pcg_groups_info: null argument");
+        return PCG_ERR_INVALID_ARG;
+    }
+    out->V = groups->dev.V;
+    out->M = groups->dev.M;
+    out->nnz = groups->nnz;
+    out->slices = groups->dev.slices;
+    out->slice_len = groups->dev.slice_len;
+    out->max_group_size = groups->max_group_size;
+    out->max_degree = groups->max_degree;
+    out->device = groups->device;
+    out->has_weights = groups->dev.pair_w != nullptr;
+    out->device_bytes = groups->device_bytes;
+    return PCG_OK;
+}

@@ -1,0 +1,270 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the CPU oracle on the same seeded
+inputs.  Integer outputs (accept lengths, group ids, tokens) must be identical except where the first differing
+decision's uniform lies within 1e-6 of its threshold (counted as excused); P and Q must agree within 1e-5
+relative for float32 logits and 1e-3 relative for bf16 logits."""
+import numpy as np
+import pytest
+
+from paper_2511_13732_b200 import workloads as W
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from oracle.compare import compare_verify  # noqa: E402
+
+from gpu_util import logits_to_device, make_handle, run_oracle, run_verify  # noqa: E402
+
+BAND = 1e-6
+
+
+def _assert_parity(got, ref, max_excused=0):
+    n, tok, grp, _ = got
+    cmp = compare_verify(n, tok, grp, ref, band=BAND)
+    assert cmp.hard == 0, f"hard mismatches: {cmp.details[:5]}"
+    assert cmp.excused <= max_excused, f"excused mismatches: {cmp.details[:5]}"
+    return cmp
+
+
+# ------------------------------------------------------------------ pcg_group_probs ----
+@pytest.mark.parametrize("name,rows", [("C1", 9), ("C2", 40), ("C3", 40), ("C4", 26)])
+def test_group_probs_matches_oracle(oracle, name, rows):
+    from paper_2511_13732_b200 import binding
+
+    cfg = W.CONFIGS[name]
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg, B=max(1, rows // (cfg.K + 1) + 1))
+    x = bt.target_logits.reshape(-1, cfg.V)[:rows]
+    want = oracle.group_probs(x, groups.group_ptr, groups.group_tok, groups.tok_degree, cfg.temperature)
+    h = make_handle(groups)
+    got = binding.pcg_group_probs(logits_to_device(x), h, cfg.temperature).cpu().numpy().astype(np.float64)
+    rtol = 1e-5 if cfg.dtype == "f32" else 1e-3
+    np.testing.assert_allclose(got, want, rtol=rtol, atol=1e-37)
+    np.testing.assert_allclose(got.sum(axis=1), 1.0, rtol=2e-6)  # no renormalisation is needed (Sec. 2.2)
+    # in practice the float32 arithmetic is far inside the bf16 allowance
+    assert np.max(np.abs(got - want) / np.maximum(want, 1e-37)) < 1e-5
+
+
+@pytest.mark.parametrize("hint", [1, 2, 4, 8])
+def test_group_probs_any_slicing(oracle, hint):
+    from paper_2511_13732_b200 import binding
+
+    cfg = W.scaled(W.CONFIGS["C4"], V=3000, M=700)  # ragged: V is not a multiple of 64 * slices
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg, B=2)
+    x = bt.draft_logits.reshape(-1, cfg.V)
+    want = oracle.group_probs(x, groups.group_ptr, groups.group_tok, groups.tok_degree, cfg.temperature)
+    h = make_handle(groups, slices_hint=hint)
+    assert h.info.slices == hint
+    got = binding.pcg_group_probs(logits_to_device(x), h, cfg.temperature).cpu().numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-5, atol=1e-37)
+
+
+# ------------------------------------------------------------------------ pcg_verify ----
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4"])
+def test_verify_matches_oracle_on_configs(oracle, name):
+    cfg = W.CONFIGS[name]
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    ref = run_oracle(oracle, bt, groups)
+    got = run_verify(bt, make_handle(groups))
+    _assert_parity(got, ref)
+    assert np.all(got[3] == 0)
+
+
+def test_verify_c5_shape_small_batch(oracle):
+    cfg = W.CONFIGS["C5"]
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg, B=12)
+    ref = run_oracle(oracle, bt, groups)
+    h = make_handle(groups)
+    assert h.info.slices == 8
+    _assert_parity(run_verify(bt, h), ref)
+
+
+@pytest.mark.parametrize("hint", [1, 2, 4, 8])
+def test_verify_any_slicing(oracle, hint):
+    cfg = W.scaled(W.CONFIGS["C3"], B=24, V=5000, M=1200, K=5)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    ref = run_oracle(oracle, bt, groups)
+    _assert_parity(run_verify(bt, make_handle(groups, slices_hint=hint)), ref)
+
+
+@pytest.mark.parametrize("V,dtype", [(1003, "f32"), (1003, "bf16"), (77, "bf16"), (4096 + 8, "bf16"), (5, "f32")])
+def test_verify_ragged_and_misaligned_rows(oracle, V, dtype):
+    """V not a multiple of the vector width: rows start at unaligned addresses and have scalar heads and tails."""
+    cfg = W.scaled(W.CONFIGS["C1"], B=10, K=3, V=V, M=max(2, V // 6), emb_dim=8, dtype=dtype,
+                   degree=min(3, max(2, V // 6)))
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    ref = run_oracle(oracle, bt, groups)
+    _assert_parity(run_verify(bt, make_handle(groups)), ref)
+
+
+@pytest.mark.parametrize("K", [1, 32])
+def test_verify_extreme_k(oracle, K):
+    cfg = W.scaled(W.CONFIGS["C1"], B=6, K=K, V=512, M=100, emb_dim=8)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    bt.draft_logits[:] = bt.target_logits[:, :K] + 0.05 * (bt.draft_logits - bt.target_logits[:, :K])  # long accepts
+    ref = run_oracle(oracle, bt, groups)
+    got = run_verify(bt, make_handle(groups))
+    _assert_parity(got, ref)
+    if K == 32:
+        assert ref.accept_len.max() > 8
+
+
+def _special_groups(kind, V, rng):
+    if kind == "singleton":
+        return W.groups_from_lists(V, [[t] for t in range(V)])
+    if kind == "one_giant":
+        return W.groups_from_lists(V, [list(range(V))])
+    if kind == "giant_plus_small":
+        return W.groups_from_lists(V, [list(range(V))] + [[t, (t + 1) % V] for t in range(0, V, 7)])
+    if kind == "with_empty":
+        lists = [[] for _ in range(40)]
+        for t in range(V):
+            for g in rng.choice(20, size=rng.integers(1, 4), replace=False):
+                lists[2 * g].append(t)  # every odd group stays empty
+        return W.groups_from_lists(V, lists)
+    if kind == "partition":
+        a = rng.integers(0, 50, size=V)
+        return W.groups_from_lists(V, [list(np.nonzero(a == k)[0]) for k in range(50)])
+    raise ValueError(kind)
+
+
+@pytest.mark.parametrize("kind", ["singleton", "one_giant", "giant_plus_small", "with_empty", "partition"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_verify_degenerate_memberships(oracle, kind, dtype):
+    rng = np.random.default_rng(5)
+    V, B, K = 2500, 16, 4
+    groups = _special_groups(kind, V, rng)
+    tl = (2.5 * rng.standard_normal((B, K + 1, V))).astype(np.float32)
+    dl = (tl[:, :K] + rng.standard_normal((B, K, V))).astype(np.float32)
+    if dtype == "bf16":
+        tl, dl = W.f32_to_bf16_bits(tl), W.f32_to_bf16_bits(dl)
+    x = rng.integers(0, V, (B, K)).astype(np.int32)
+    x[:, 0] = np.argmax(dl[:, 0].astype(np.float32) if dtype == "f32" else W.bf16_bits_to_f32(dl[:, 0]), axis=1)
+    u = (rng.integers(0, 1 << 24, (B, K + 1, 2)) * 2.0 ** -24).astype(np.float32)
+    bt = W.Batch(tl, dl, x, u, 0.9, dtype)
+    ref = run_oracle(oracle, bt, groups)
+    for hint in (0, 4):
+        got = run_verify(bt, make_handle(groups, slices_hint=hint))
+        _assert_parity(got, ref)
+    if kind == "one_giant":
+        assert np.all(ref.accept_len == K)  # a single group is always accepted: P = Q = 1
+
+
+def test_verify_all_accept_all_reject_and_masked_logits(oracle):
+    rng = np.random.default_rng(6)
+    cfg = W.scaled(W.CONFIGS["C2"], B=8, K=6, V=2048, M=300, emb_dim=16)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    # identical draft and target: every position accepted, bonus token drawn
+    same = W.Batch(bt.target_logits, bt.target_logits[:, :cfg.K].copy(), bt.draft_tokens, bt.uniforms, 1.0, "f32")
+    ref = run_oracle(oracle, same, groups)
+    assert np.all(ref.accept_len == cfg.K)
+    h = make_handle(groups)
+    _assert_parity(run_verify(same, h), ref)
+    # draft token forced onto a token the target gives no mass (-inf): rejected at position 0
+    tl, dl = bt.target_logits.copy(), bt.draft_logits.copy()
+    for b in range(cfg.B):
+        g_tokens = set()
+        for g in range(groups.M):  # mask, in the target, every token that shares a group with the draft token
+            toks = groups.group_tok[groups.group_ptr[g]:groups.group_ptr[g + 1]]
+            if bt.draft_tokens[b, 0] in toks:
+                g_tokens.update(toks.tolist())
+        tl[b, 0, list(g_tokens)] = -np.inf
+    masked = W.Batch(tl, dl, bt.draft_tokens, bt.uniforms, 1.0, "f32")
+    ref = run_oracle(oracle, masked, groups)
+    assert np.all(ref.accept_len == 0)
+    got = run_verify(masked, h)
+    _assert_parity(got, ref)
+    assert np.all(got[3] == 0)  # -inf logits are legitimate masks, not an error
+    # one dominant logit per row
+    tl2 = bt.target_logits.copy()
+    tl2[:, :, 17] += 60.0
+    dom = W.Batch(tl2, bt.draft_logits, bt.draft_tokens, bt.uniforms, 1.0, "f32")
+    _assert_parity(run_verify(dom, h), run_oracle(oracle, dom, groups))
+
+
+def test_verify_is_bit_reproducible_and_flags_bad_tokens(oracle):
+    cfg = W.scaled(W.CONFIGS["C3"], B=32)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    h = make_handle(groups)
+    first = run_verify(bt, h)
+    for _ in range(5):
+        again = run_verify(bt, h)
+        assert all(np.array_equal(a, b) for a, b in zip(first, again))
+    bad = W.Batch(bt.target_logits, bt.draft_logits, bt.draft_tokens.copy(), bt.uniforms, bt.temperature, bt.dtype)
+    bad.draft_tokens[3, 0] = cfg.V + 5
+    bad.draft_tokens[4, 0] = -1
+    got = run_verify(bad, h)
+    assert got[3][3] & 1 and got[3][4] & 1 and not np.any(np.delete(got[3], [3, 4]) & 1)
+    assert np.all((got[1] >= -1) & (got[1] < cfg.V))
+
+
+def test_verify_host_entry_point_matches_device_entry_point(oracle):
+    from paper_2511_13732_b200 import binding
+
+    cfg = W.scaled(W.CONFIGS["C3"], B=16)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    h = make_handle(groups)
+    dev = run_verify(bt, h)
+    pin = lambda a: torch.from_numpy(a).pin_memory()  # noqa: E731
+    tl = torch.from_numpy(bt.target_logits.view(np.int16)).pin_memory()
+    dl = torch.from_numpy(bt.draft_logits.view(np.int16)).pin_memory()
+    out = (torch.empty(cfg.B, dtype=torch.int32).pin_memory(), torch.empty((cfg.B, cfg.K + 1), dtype=torch.int32).pin_memory(),
+           torch.empty((cfg.B, cfg.K + 1), dtype=torch.int32).pin_memory(), torch.empty(cfg.B, dtype=torch.int32).pin_memory())
+    need = binding.pcg_verify_host_arena_bytes(cfg.B, cfg.K, cfg.V, groups.M, binding.PCG_BF16)
+    arena = torch.empty(need, dtype=torch.uint8, device="cuda")
+    binding.pcg_verify_host(tl, dl, pin(bt.draft_tokens), h, pin(bt.uniforms), bt.temperature, arena, out)
+    for a, b in zip(dev, out):
+        assert np.array_equal(a, b.numpy())
+    with pytest.raises(binding.PcgError) as ei:
+        binding.pcg_verify_host(tl, dl, pin(bt.draft_tokens), h, pin(bt.uniforms), bt.temperature, arena[:1024], out)
+    assert ei.value.status == 4
+
+
+def test_device_side_argument_errors(oracle):
+    from paper_2511_13732_b200 import binding
+
+    cfg = W.scaled(W.CONFIGS["C1"], B=2)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    h = make_handle(groups)
+    tl, dl = logits_to_device(bt.target_logits), logits_to_device(bt.draft_logits)
+    x, u = torch.from_numpy(bt.draft_tokens).cuda(), torch.from_numpy(bt.uniforms).cuda()
+    with pytest.raises(binding.PcgError) as ei:
+        binding.pcg_verify(tl, dl, x, h, u, 0.0)
+    assert ei.value.status == 1
+    with pytest.raises(binding.PcgError) as ei:
+        binding.pcg_verify(tl, dl, x, h, u, 1.0, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert ei.value.status == 4
+    # B = 0 and rows = 0 are no-ops
+    binding.pcg_verify(tl[:0], dl[:0], x[:0], h, u[:0], 1.0)
+    assert binding.pcg_group_probs(tl.reshape(-1, cfg.V)[:0], h).shape == (0, groups.M)
+
+
+def test_full_size_bench_configuration_on_sampled_sequences(oracle):
+    """C5 exactly as bench.py launches it (B=256, K=16, V=65536, bf16): every sequence is checked for structure,
+    and a sample of sequences is checked decision by decision against the oracle."""
+    cfg = W.CONFIGS["C5"]
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    h = make_handle(groups)
+    n, tok, grp, flg = run_verify(bt, h)
+    assert np.all(flg == 0) and np.all((n >= 0) & (n <= cfg.K))
+    for b in range(cfg.B):
+        assert np.array_equal(tok[b, :n[b]], bt.draft_tokens[b, :n[b]])
+        assert np.all(tok[b, n[b] + 1:] == -1) and np.all(grp[b, n[b] + 1:] == -1)
+        for i in range(n[b] + 1):
+            g = grp[b, i]
+            assert tok[b, i] in groups.group_tok[groups.group_ptr[g]:groups.group_ptr[g + 1]]
+    sample = list(range(0, cfg.B, 16)) + [int(np.argmax(n))]
+    sub = W.Batch(bt.target_logits[sample], bt.draft_logits[sample], bt.draft_tokens[sample], bt.uniforms[sample],
+                  bt.temperature, bt.dtype)
+    ref = run_oracle(oracle, sub, groups)
+    _assert_parity((n[sample], tok[sample], grp[sample], flg[sample]), ref)
