@@ -179,10 +179,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C5", choices=sorted(W.CONFIGS))
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (profiling only)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = W.CONFIGS[args.workload]
+    if args.batch > 0:
+        cfg = W.scaled(cfg, B=args.batch, name=f"{cfg.name}[B={args.batch}]")
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

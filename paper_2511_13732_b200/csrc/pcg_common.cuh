@@ -13,6 +13,8 @@
 namespace pcg {
 
 constexpr float kNegInf = -__builtin_huge_valf();
+constexpr int kAggThreads = 512;        // threads per block of the aggregation kernels (fixes the sweep layout)
+constexpr uint32_t kNoGroup = 0xffffu;  // group field of sweep entries that belong to no group
 
 // Device-resident membership, built once by pcg_groups_create.
 struct GroupsDev {
@@ -25,10 +27,16 @@ struct GroupsDev {
     const float *inv_deg;      // [V]     1/N(t)
     const int32_t *rev_ptr;    // [V+1]   reverse membership S(t), ascending group id
     const int32_t *rev_grp;    // [nnz]
-    const int32_t *slice_ptr;  // [C][M+1] start of (slice, group) sub-list in slice_tok
-    const uint16_t *slice_tok; // [nnz]   in-slice token offsets, ordered by (slice, group, token)
+    // Token-sliced copy of the CSR for the aggregation sweep.  Slice c owns entries [ent_off[c], ent_off[c+1]),
+    // a whole number of rows of kAggThreads entries; thread t walks column t (entry j of thread t sits at
+    // row j, so a warp reads consecutive words).  An entry is (group id << 16) | in-slice token offset; all
+    // entries of one (slice, group) pair are consecutive in one thread's column, in CSR order.  Columns are
+    // padded with entries that point at the always-zero slot `slice_len` (group kNoGroup if the thread owns
+    // no group in this slice).
+    const int32_t *ent_off;    // [C+1]
+    const uint32_t *ent;       // [ent_off[C]]
+    const float *ent_w;        // [ent_off[C]] weights in the same layout, or nullptr (equal split)
     const float *pair_w;       // [nnz] CSR-order weights w_{g,t} or nullptr (equal split)
-    const float *slice_w;      // [nnz] the same in slice order, or nullptr
     const float *rev_w;        // [nnz] the same in reverse-membership order, or nullptr
 };
 

@@ -4,7 +4,9 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <algorithm>
 #include <new>
+#include <queue>
 #include <vector>
 
 #include "pcg_common.cuh"
@@ -30,7 +32,7 @@ constexpr size_t kAggScratch = 2048;
 
 size_t agg_smem_bytes(int slice_len, int M, int slices) {
     size_t mc = (size_t)(M + slices - 1) / slices;
-    return (size_t)slice_len * 4 + (size_t)M * 4 + mc * 4 + kAggScratch;
+    return ((size_t)slice_len + 32) * 4 + (size_t)M * 4 + mc * 4 + kAggScratch;
 }
 
 }  // namespace pcg
@@ -179,37 +181,83 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     int C = slices_hint ? slices_hint : 1;
     if (!slices_hint)
         while (C < 8 && (V + C - 1) / C > 8192) C *= 2;
+    if (M >= (int)kNoGroup) {
+        set_error("M=%d: the sweep layout holds group ids in 16 bits (M <= 65534)", M);
+        return PCG_ERR_UNSUPPORTED;
+    }
     int SL = 0;
     for (;; C *= 2) {
         SL = (((V + C - 1) / C) + 63) / 64 * 64;
-        if (SL <= 65536 && agg_smem_bytes(SL, M, C) <= kMaxSmem) break;
+        if (SL <= 65472 && agg_smem_bytes(SL, M, C) <= kMaxSmem) break;
         if (C >= 8) {
             set_error("V=%d, M=%d do not fit the aggregation kernels' shared memory even with 8 slices", V, M);
             return PCG_ERR_UNSUPPORTED;
         }
     }
 
-    // ---- token-sliced copy of the CSR: sub-lists ordered by (slice, group), 16-bit in-slice offsets ----
-    std::vector<int32_t> sptr((size_t)C * (M + 1));
-    std::vector<uint16_t> stok((size_t)nnz);
-    std::vector<float> sw;
-    if (!w.empty()) sw.resize((size_t)nnz);
+    // ---- token-sliced sweep layout (see GroupsDev::ent) ----
+    // Per slice, the groups' sub-lists are dealt to the kAggThreads threads longest first, each to the thread
+    // with the least work so far (ties: lowest thread id), so that the columns are balanced.
+    std::vector<int32_t> eoff((size_t)C + 1, 0);
+    std::vector<uint32_t> ent;
+    std::vector<float> entw;
     {
-        int32_t at = 0;
+        constexpr int NT = kAggThreads;
         std::vector<int32_t> cursor(gptr.begin(), gptr.end() - 1);  // tokens ascend, so each slice is a sub-range
+        std::vector<int32_t> sub_lo((size_t)M), sub_hi((size_t)M), order((size_t)M);
+        std::vector<std::vector<int32_t>> owned(NT);
         for (int c = 0; c < C; ++c) {
             const int32_t t_end = (int32_t)std::min<int64_t>((int64_t)(c + 1) * SL, V);
             for (int g = 0; g < M; ++g) {
-                sptr[(size_t)c * (M + 1) + g] = at;
                 int32_t k = cursor[g];
-                for (; k < gptr[g + 1] && gtok[k] < t_end; ++k) {
-                    stok[at] = (uint16_t)(gtok[k] - c * SL);
-                    if (!w.empty()) sw[at] = w[k];
-                    ++at;
-                }
-                cursor[g] = k;
+                sub_lo[g] = k;
+                while (k < gptr[g + 1] && gtok[k] < t_end) ++k;
+                sub_hi[g] = cursor[g] = k;
+                order[g] = g;
             }
-            sptr[(size_t)c * (M + 1) + M] = at;
+            std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) {
+                return sub_hi[x] - sub_lo[x] > sub_hi[y] - sub_lo[y];
+            });
+            std::priority_queue<std::pair<int64_t, int>, std::vector<std::pair<int64_t, int>>,
+                                std::greater<std::pair<int64_t, int>>> load;
+            for (int t = 0; t < NT; ++t) {
+                owned[t].clear();
+                load.push({0, t});
+            }
+            for (int32_t g : order) {
+                const int32_t len = sub_hi[g] - sub_lo[g];
+                if (len == 0) break;  // the rest is empty in this slice (partial[] is zero-filled by the kernel)
+                auto top = load.top();
+                load.pop();
+                owned[top.second].push_back(g);
+                load.push({top.first + len, top.second});
+            }
+            int64_t rows = 0;
+            for (int t = 0; t < NT; ++t) {
+                int64_t n = 0;
+                for (int32_t g : owned[t]) n += sub_hi[g] - sub_lo[g];
+                rows = std::max(rows, n);
+            }
+            const size_t base = ent.size();
+            if ((int64_t)base + rows * NT > INT32_MAX) {
+                set_error("membership too large for the sweep layout");
+                return PCG_ERR_UNSUPPORTED;
+            }
+            ent.resize(base + (size_t)rows * NT);
+            if (!w.empty()) entw.resize(ent.size(), 0.f);
+            for (int t = 0; t < NT; ++t) {
+                int64_t j = 0;
+                uint32_t last_group = kNoGroup;
+                for (int32_t g : owned[t]) {
+                    last_group = (uint32_t)g;
+                    for (int32_t k = sub_lo[g]; k < sub_hi[g]; ++k, ++j) {
+                        ent[base + (size_t)j * NT + t] = ((uint32_t)g << 16) | (uint32_t)(gtok[k] - c * SL);
+                        if (!w.empty()) entw[base + (size_t)j * NT + t] = w[k];
+                    }
+                }
+                for (; j < rows; ++j) ent[base + (size_t)j * NT + t] = (last_group << 16) | (uint32_t)SL;
+            }
+            eoff[c + 1] = (int32_t)ent.size();
         }
     }
     std::vector<float> inv((size_t)V);
@@ -219,8 +267,8 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     Carver cv;
     const size_t o_gptr = cv.take(gptr.size() * 4), o_gtok = cv.take(gtok.size() * 4), o_inv = cv.take(inv.size() * 4);
     const size_t o_rptr = cv.take(rptr.size() * 4), o_rgrp = cv.take(rgrp.size() * 4);
-    const size_t o_sptr = cv.take(sptr.size() * 4), o_stok = cv.take(stok.size() * 2);
-    const size_t o_w = cv.take(w.size() * 4), o_sw = cv.take(sw.size() * 4), o_rw = cv.take(rw.size() * 4);
+    const size_t o_eoff = cv.take(eoff.size() * 4), o_ent = cv.take(ent.size() * 4);
+    const size_t o_w = cv.take(w.size() * 4), o_entw = cv.take(entw.size() * 4), o_rw = cv.take(rw.size() * 4);
     const size_t total = cv.off ? cv.off : 256;
     void *mem = nullptr;
     if (!have_device) {
@@ -235,10 +283,10 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     if (e == cudaSuccess) e = upload(base, o_inv, inv);
     if (e == cudaSuccess) e = upload(base, o_rptr, rptr);
     if (e == cudaSuccess) e = upload(base, o_rgrp, rgrp);
-    if (e == cudaSuccess) e = upload(base, o_sptr, sptr);
-    if (e == cudaSuccess) e = upload(base, o_stok, stok);
+    if (e == cudaSuccess) e = upload(base, o_eoff, eoff);
+    if (e == cudaSuccess) e = upload(base, o_ent, ent);
     if (e == cudaSuccess) e = upload(base, o_w, w);
-    if (e == cudaSuccess) e = upload(base, o_sw, sw);
+    if (e == cudaSuccess) e = upload(base, o_entw, entw);
     if (e == cudaSuccess) e = upload(base, o_rw, rw);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -261,10 +309,10 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     h->dev.inv_deg = (const float *)(base + o_inv);
     h->dev.rev_ptr = (const int32_t *)(base + o_rptr);
     h->dev.rev_grp = (const int32_t *)(base + o_rgrp);
-    h->dev.slice_ptr = (const int32_t *)(base + o_sptr);
-    h->dev.slice_tok = (const uint16_t *)(base + o_stok);
+    h->dev.ent_off = (const int32_t *)(base + o_eoff);
+    h->dev.ent = (const uint32_t *)(base + o_ent);
     h->dev.pair_w = w.empty() ? nullptr : (const float *)(base + o_w);
-    h->dev.slice_w = w.empty() ? nullptr : (const float *)(base + o_sw);
+    h->dev.ent_w = w.empty() ? nullptr : (const float *)(base + o_entw);
     h->dev.rev_w = w.empty() ? nullptr : (const float *)(base + o_rw);
     h->nnz = nnz;
     h->device = device;

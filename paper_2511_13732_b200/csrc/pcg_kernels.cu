@@ -22,79 +22,120 @@ namespace cg = cooperative_groups;
 namespace pcg {
 
 constexpr int kPosThreads = 256;
-constexpr int kAggThreads = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // ================================================================ position kernel ==========================
+//
+// Per row the kernel needs Z = sum_t 2^(l_t*s - RS) for SOME reference RS (any value works as long as the same
+// RS is used for the group masses: it cancels in P = S/Z), so each thread keeps a lazy reference: the largest
+// logit of its first vector, raised only when a later logit exceeds it by more than 32/s (a factor 2^32 of
+// headroom).  After the first vector the rescale branch is practically never taken, which keeps the special-
+// function unit at exactly one ex2 per logit.  Logits travel global -> shared through a per-thread ring of
+// 16-byte cp.async copies (kStages deep) so that many loads stay in flight without holding registers.
 
-// Online softmax statistics of one row: running maximum m of the raw logits and sum of 2^((l-m)s).
+constexpr int kStages = 8;
+constexpr float kRefInit = -1.0e30f;  // "no logit seen yet"; finite so that -inf logits give 2^-inf = 0, not NaN
+
+struct RefSum {
+    float r;    // raw-logit reference
+    float rs;   // r * s as computed once (the exponent actually subtracted)
+    float thr;  // r + 32/s: logits above this raise the reference
+    float acc;  // sum of 2^(l*s - rs)
+};
+
+__device__ __forceinline__ void raise_ref(RefSum &st, float vm, float s, float headroom) {
+    const float nrs = vm * s;
+    st.acc *= ex2(st.rs - nrs);
+    st.r = vm;
+    st.rs = nrs;
+    st.thr = vm + headroom;
+}
+
 template <int NV>
-__device__ __forceinline__ void absorb(MaxSum &st, const float (&v)[NV], float s) {
+__device__ __forceinline__ void absorb(RefSum &st, const float (&v)[NV], float s, float headroom) {
     float vm = v[0];
 #pragma unroll
     for (int i = 1; i < NV; ++i) vm = fmaxf(vm, v[i]);
-    if (vm > st.m) {  // rare after the first few vectors
-        st.acc *= ex2((st.m - vm) * s);
-        st.m = vm;
-    }
-    if (st.m > kNegInf) {
+    if (vm > st.thr) raise_ref(st, vm, s, headroom);
 #pragma unroll
-        for (int i = 0; i < NV; ++i) st.acc += ex2((v[i] - st.m) * s);
+    for (int i = 0; i < NV; ++i) st.acc += ex2(__fmaf_rn(v[i], s, -st.rs));
+}
+
+__device__ __forceinline__ void absorb1(RefSum &st, float l, float s, float headroom) {
+    if (l > st.thr) raise_ref(st, l, s, headroom);
+    st.acc += ex2(__fmaf_rn(l, s, -st.rs));
+}
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Where the 16-byte vectors of a row start and how many there are.
+template <typename T>
+struct RowSplit {
+    int head, nvec;
+    const uint4 *vp;
+    __device__ __forceinline__ RowSplit(const T *row, int V) {
+        head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
+        if (head > V) head = V;
+        nvec = (V - head) / Elem<T>::kPerVec;
+        vp = reinterpret_cast<const uint4 *>(row + head);
+    }
+};
+
+// Deterministic block-wide combine of (rs, acc) pairs of TWO rows at once: xor butterfly inside a warp, then a
+// fixed-order pass over the warps.  `scratch` holds 4*NWARPS floats.  Every thread returns the same values.
+__device__ __forceinline__ void merge(float &rs, float &acc, float rs2, float acc2) {
+    const float m = fmaxf(rs, rs2);
+    acc = acc * ex2(rs - m) + acc2 * ex2(rs2 - m);
+    rs = m;
+}
+
+template <int NT>
+__device__ __forceinline__ void block_combine2(float &rs_a, float &acc_a, float &rs_b, float &acc_b, float *scratch) {
+    constexpr int NW = NT / 32;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        merge(rs_a, acc_a, __shfl_xor_sync(0xffffffffu, rs_a, o), __shfl_xor_sync(0xffffffffu, acc_a, o));
+        merge(rs_b, acc_b, __shfl_xor_sync(0xffffffffu, rs_b, o), __shfl_xor_sync(0xffffffffu, acc_b, o));
+    }
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) {
+        float *p = scratch + 4 * (threadIdx.x >> 5);
+        p[0] = rs_a, p[1] = acc_a, p[2] = rs_b, p[3] = acc_b;
+    }
+    __syncthreads();
+    rs_a = scratch[0], acc_a = scratch[1], rs_b = scratch[2], acc_b = scratch[3];
+#pragma unroll
+    for (int w = 1; w < NW; ++w) {
+        merge(rs_a, acc_a, scratch[4 * w], scratch[4 * w + 1]);
+        merge(rs_b, acc_b, scratch[4 * w + 2], scratch[4 * w + 3]);
     }
 }
 
-__device__ __forceinline__ void absorb1(MaxSum &st, float l, float s) {
-    if (l > st.m) {
-        st.acc *= ex2((st.m - l) * s);
-        st.m = l;
-    }
-    if (st.m > kNegInf) st.acc += ex2((l - st.m) * s);
-}
-
-template <typename T, int NT>
-__device__ __forceinline__ MaxSum row_stats(const T *__restrict__ row, int V, float s, float *scratch) {
-    constexpr int NV = Elem<T>::kPerVec;
-    constexpr int U = 4;
-    const int tid = threadIdx.x;
-    MaxSum st{kNegInf, 0.f};
-    // elements before the first 16-byte boundary, whole vectors, elements after the last whole vector
-    int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
-    if (head > V) head = V;
-    const int nvec = (V - head) / NV;
-    const uint4 *vp = reinterpret_cast<const uint4 *>(row + head);
-    for (int base = 0; base < nvec; base += NT * U) {
-        uint4 r[U];
+template <int NT>
+__device__ __forceinline__ void block_sum2(float &a, float &b, float *scratch) {
+    constexpr int NW = NT / 32;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int idx = base + u * NT + tid;
-            if (idx < nvec) r[u] = ld_stream(vp + idx);
-        }
+    for (int o = 16; o > 0; o >>= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, o);
+        b += __shfl_xor_sync(0xffffffffu, b, o);
+    }
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) {
+        scratch[2 * (threadIdx.x >> 5)] = a;
+        scratch[2 * (threadIdx.x >> 5) + 1] = b;
+    }
+    __syncthreads();
+    a = scratch[0], b = scratch[1];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int idx = base + u * NT + tid;
-            if (idx < nvec) {
-                float v[NV];
-                Elem<T>::unpack(r[u], v);
-                absorb<NV>(st, v, s);
-            }
-        }
-    }
-    for (int t = tid; t < head; t += NT) absorb1(st, Elem<T>::widen(row[t]), s);
-    for (int t = head + nvec * NV + tid; t < V; t += NT) absorb1(st, Elem<T>::widen(row[t]), s);
-    return block_combine<NT>(st, s, scratch);
-}
-
-// Mass of one group under the row's unnormalised softmax terms: sum_k 2^((l_t - m)s) * w_k, t = tok[k].
-template <typename T, int NT>
-__device__ __forceinline__ float group_mass(const T *__restrict__ row, const GroupsDev &G, int lo, int hi, float m,
-                                            float s, float *scratch) {
-    float part = 0.f;
-    for (int k = lo + (int)threadIdx.x; k < hi; k += NT) {
-        const int t = G.group_tok[k];
-        const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
-        part += __fmul_rn(ex2((Elem<T>::widen(row[t]) - m) * s), w);
-    }
-    return block_sum<NT>(part, scratch);
+    for (int w = 1; w < NW; ++w) a += scratch[2 * w], b += scratch[2 * w + 1];
 }
 
 struct PositionArgs {
@@ -104,25 +145,45 @@ struct PositionArgs {
     const float *uniforms;   // [B, K+1, 2]
     int K;
     float s;                 // log2(e) / temperature
+    float headroom;          // 32 / s
     int32_t *accept;         // [B*K] 1 = accepted
     int32_t *labels;         // [B*K] group label of the draft token
     int32_t *posflags;       // [B*K]
-    float4 *stats;           // [B*K] (m_p, 1/Z_p, m_q, 1/Z_q)
+    float4 *stats;           // [B*K] (RS_p, 1/Z_p, RS_q, 1/Z_q): scaled reference and reciprocal normaliser
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a, GroupsDev G) {
+__global__ void __launch_bounds__(kPosThreads, 5) position_kernel(PositionArgs a, GroupsDev G) {
     constexpr int NT = kPosThreads;
-    __shared__ float scratch[2 * (NT / 32)];
+    constexpr int NV = Elem<T>::kPerVec;
+    constexpr int S = kStages;
+    __shared__ uint4 ring[S][NT];
+    __shared__ float scratch[4 * (NT / 32)];
     __shared__ int sh_label, sh_flag;
+    const int tid = threadIdx.x;
     const int pos = blockIdx.x;
     const int b = pos / a.K, i = pos - b * a.K;
     const int V = G.V;
     const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (a.K + 1) + i) * V;
     const T *qrow = reinterpret_cast<const T *>(a.draft) + (int64_t)pos * V;
     const float *u = a.uniforms + ((int64_t)b * (a.K + 1) + i) * 2;
+    const float s = a.s, headroom = a.headroom;
 
-    if (threadIdx.x == 0) {
+    // ---- start streaming: the two rows form one sequence of 2*nk vector slots per thread ----
+    const RowSplit<T> ts(trow, V), qs(qrow, V);
+    const int nk_t = (ts.nvec + NT - 1) / NT, nk_q = (qs.nvec + NT - 1) / NT, nk = nk_t + nk_q;
+    auto issue = [&](int k) {
+        if (k < nk) {
+            const bool second = k >= nk_t;
+            const int idx = tid + (second ? k - nk_t : k) * NT;
+            if (idx < (second ? qs.nvec : ts.nvec)) cp_async16(&ring[k % S][tid], (second ? qs.vp : ts.vp) + idx);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int k = 0; k < S - 1; ++k) issue(k);
+
+    if (tid == 0) {
         // group-label coupling: the label is drawn from the groups of the draft token with its split weights
         int x = a.draft_tokens[pos], flag = 0;
         if (x < 0 || x >= V) {
@@ -154,26 +215,54 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
         sh_label = G.rev_grp[r0 + j];
         sh_flag = flag;
     }
-    __syncthreads();
+
+    RefSum st_t{kRefInit, kRefInit * s, kRefInit, 0.f}, st_q = st_t;
+    for (int k = 0; k < nk; ++k) {
+        issue(k + S - 1);
+        cp_async_wait<S - 1>();
+        const bool second = k >= nk_t;
+        const int idx = tid + (second ? k - nk_t : k) * NT;
+        if (idx < (second ? qs.nvec : ts.nvec)) {
+            float v[NV];
+            Elem<T>::unpack(ring[k % S][tid], v);
+            if (second)
+                absorb<NV>(st_q, v, s, headroom);
+            else
+                absorb<NV>(st_t, v, s, headroom);
+        }
+    }
+    // elements before the first and after the last whole 16-byte vector of each row
+    for (int t = tid; t < ts.head; t += NT) absorb1(st_t, Elem<T>::widen(trow[t]), s, headroom);
+    for (int t = ts.head + ts.nvec * NV + tid; t < V; t += NT) absorb1(st_t, Elem<T>::widen(trow[t]), s, headroom);
+    for (int t = tid; t < qs.head; t += NT) absorb1(st_q, Elem<T>::widen(qrow[t]), s, headroom);
+    for (int t = qs.head + qs.nvec * NV + tid; t < V; t += NT) absorb1(st_q, Elem<T>::widen(qrow[t]), s, headroom);
+
+    float rs_p = st_t.rs, Zp = st_t.acc, rs_q = st_q.rs, Zq = st_q.acc;
+    block_combine2<NT>(rs_p, Zp, rs_q, Zq, scratch);  // its barriers also publish sh_label
+
+    // ---- masses of the label group under both rows: a handful of gathered logits ----
     const int g = sh_label;
     const int lo = G.group_ptr[g], hi = G.group_ptr[g + 1];
+    float Sp = 0.f, Sq = 0.f;
+    for (int k = lo + tid; k < hi; k += NT) {
+        const int t = G.group_tok[k];
+        const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
+        Sp += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs_p)), w);
+        Sq += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), s, -rs_q)), w);
+    }
+    block_sum2<NT>(Sp, Sq, scratch);
 
-    const MaxSum sp = row_stats<T, NT>(trow, V, a.s, scratch);
-    const float Sp = group_mass<T, NT>(trow, G, lo, hi, sp.m, a.s, scratch);
-    const MaxSum sq = row_stats<T, NT>(qrow, V, a.s, scratch);
-    const float Sq = group_mass<T, NT>(qrow, G, lo, hi, sq.m, a.s, scratch);
-
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         // acceptance u < min(1, P/Q) without a division: P = Sp/Zp, Q = Sq/Zq
-        const float lhs = Sp * sq.acc, rhs = Sq * sp.acc;
+        const float lhs = Sp * Zq, rhs = Sq * Zp;
         const int acc = (lhs >= rhs) || (u[1] * rhs < lhs);
         int flag = sh_flag;
-        if (!(sp.acc > 0.f) || !(sq.acc > 0.f) || isinf(sp.acc) || isinf(sq.acc) || isinf(sp.m) || isinf(sq.m))
+        if (!(Zp > 0.f) || !(Zq > 0.f) || isinf(Zp) || isinf(Zq) || isinf(rs_p) || isinf(rs_q))
             flag |= PCG_FLAG_NONFINITE;
         a.accept[pos] = acc;
         a.labels[pos] = g;
         a.posflags[pos] = flag;
-        a.stats[pos] = make_float4(sp.m, 1.0f / sp.acc, sq.m, 1.0f / sq.acc);
+        a.stats[pos] = make_float4(rs_p, 1.0f / Zp, rs_q, 1.0f / Zq);
     }
 }
 
@@ -197,7 +286,7 @@ struct AggSmem {
 __device__ __forceinline__ AggSmem carve_smem(unsigned char *raw, const GroupsDev &G) {
     AggSmem sm;
     sm.d = reinterpret_cast<float *>(raw);
-    sm.partial = sm.d + G.slice_len;
+    sm.partial = sm.d + G.slice_len + 32;  // d[slice_len] is the always-zero slot of padding entries
     sm.own = sm.partial + G.M;
     unsigned char *tail = reinterpret_cast<unsigned char *>(sm.own + G.groups_per_slice);
     tail = reinterpret_cast<unsigned char *>(((uintptr_t)tail + 15) & ~(uintptr_t)15);
@@ -241,19 +330,49 @@ __device__ __forceinline__ float load_slice_max(const T *__restrict__ row, int n
 }
 
 // Segmented reduction of the slice: partial[g] = sum over the slice's tokens of group g of d[t] (* w).
+// Thread t walks column t of the slice's entry rows (coalesced 32-bit loads, kept several rows ahead in
+// registers), adds d[token] into a register while the group id stays the same and stores the sum when it
+// changes; a group's entries never span two threads, so every partial[g] has exactly one writer and a fixed
+// summation order.  partial[] must be zero-filled and d[slice_len] must be 0 before the call.
 template <int NT>
 __device__ __forceinline__ void sweep_slice(const GroupsDev &G, int c, const float *d, float *partial) {
-    const int32_t *sp = G.slice_ptr + (size_t)c * (G.M + 1);
-    for (int g = threadIdx.x; g < G.M; g += NT) {
-        const int lo = sp[g], hi = sp[g + 1];
-        float acc = 0.f;
-        if (G.slice_w) {
-            for (int k = lo; k < hi; ++k) acc += __fmul_rn(d[G.slice_tok[k]], G.slice_w[k]);
-        } else {
-            for (int k = lo; k < hi; ++k) acc += d[G.slice_tok[k]];
+    constexpr int R = 8;  // rows in flight per thread
+    const int begin = G.ent_off[c], rows = (G.ent_off[c + 1] - begin) / NT;
+    const uint32_t *ep = G.ent + begin + threadIdx.x;
+    const float *wp = G.ent_w ? G.ent_w + begin + threadIdx.x : nullptr;
+    uint32_t cur = kNoGroup;
+    float acc = 0.f;
+    for (int r0 = 0; r0 < rows; r0 += R) {
+        uint32_t e[R];
+        float w[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            const bool in = r0 + j < rows;
+            e[j] = in ? ep[(size_t)(r0 + j) * NT] : 0u;
+            w[j] = (wp && in) ? wp[(size_t)(r0 + j) * NT] : 1.f;
         }
-        partial[g] = acc;
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            if (r0 + j < rows) {
+                const uint32_t g = e[j] >> 16;
+                if (g != cur) {
+                    if (cur != kNoGroup) partial[cur] = acc;
+                    cur = g;
+                    acc = 0.f;
+                }
+                const float v = d[e[j] & 0xffffu];
+                acc += wp ? __fmul_rn(v, w[j]) : v;
+            }
+        }
     }
+    if (cur != kNoGroup) partial[cur] = acc;
+}
+
+// Zero partial[0..M) and the always-zero slot d[slice_len] (block-wide; followed by a barrier at the caller).
+template <int NT>
+__device__ __forceinline__ void clear_partial(const GroupsDev &G, float *d, float *partial) {
+    for (int g = threadIdx.x; g < G.M; g += NT) partial[g] = 0.f;
+    if (threadIdx.x == 0) d[G.slice_len] = 0.f;
 }
 
 // ---------------------------------------------------------------- pcg_group_probs ----------------------------
@@ -264,7 +383,7 @@ struct ProbsArgs {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kAggThreads) group_probs_kernel(ProbsArgs a, GroupsDev G) {
+__global__ void __launch_bounds__(kAggThreads, 2) group_probs_kernel(ProbsArgs a, GroupsDev G) {
     constexpr int NT = kAggThreads;
     extern __shared__ __align__(16) unsigned char raw[];
     AggSmem sm = carve_smem(raw, G);
@@ -277,16 +396,18 @@ __global__ void __launch_bounds__(kAggThreads) group_probs_kernel(ProbsArgs a, G
     const T *rp = reinterpret_cast<const T *>(a.logits) + row * G.V + t0;
 
     // softmax terms of the slice relative to the row maximum (exchanged across the cluster)
+    clear_partial<NT>(G, sm.d, sm.partial);
     const float mloc = load_slice_max<T, NT>(rp, n, sm.d, sm.scratch);
     if (threadIdx.x == 0) sm.xchg[1] = (double)mloc;
     cluster.sync();
     float m = kNegInf;
     for (int r = 0; r < C; ++r) m = fmaxf(m, (float)*cluster.map_shared_rank(&sm.xchg[1], r));
     float zloc = 0.f;
+    const float rs = m * a.s;
     for (int t = threadIdx.x; t < n; t += NT) {
-        const float e = ex2((sm.d[t] - m) * a.s);
+        const float e = ex2(__fmaf_rn(sm.d[t], a.s, -rs));
         zloc += e;
-        sm.d[t] = G.slice_w ? e : __fmul_rn(e, G.inv_deg[t0 + t]);
+        sm.d[t] = G.ent_w ? e : __fmul_rn(e, G.inv_deg[t0 + t]);
     }
     const float zc = block_sum<NT>(zloc, sm.scratch);  // contains the barrier that publishes d
     if (threadIdx.x == 0) sm.xchg[0] = (double)zc;
@@ -322,7 +443,7 @@ struct TerminalArgs {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kAggThreads) terminal_kernel(TerminalArgs a, GroupsDev G) {
+__global__ void __launch_bounds__(kAggThreads, 2) terminal_kernel(TerminalArgs a, GroupsDev G) {
     constexpr int NT = kAggThreads;
     extern __shared__ __align__(16) unsigned char raw[];
     AggSmem sm = carve_smem(raw, G);
@@ -357,15 +478,16 @@ __global__ void __launch_bounds__(kAggThreads) terminal_kernel(TerminalArgs a, G
     const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
 
     bool residual = n < K;  // false: draw from the target's coarse distribution itself (bonus token)
-    float m_tgt = 0.f;
+    float rs_tgt = 0.f;  // scaled reference of the target row's softmax terms
     double Ztot = 0.0, my_off = 0.0, my_excl = 0.0, my_incl = 0.0, my_sum = 0.0;
     const int per = (nown + NT - 1) / NT;
     const int i0 = min(nown, tid * per), i1 = min(nown, i0 + per);
     for (int attempt = 0; attempt < 2; ++attempt) {
         // ---- per-token values of this slice ----
+        clear_partial<NT>(G, sm.d, sm.partial);
         if (residual) {
             const float4 st = a.stats[b * K + n];
-            m_tgt = st.x;
+            rs_tgt = st.x;
             constexpr int NV = Elem<T>::kPerVec;
             const T *tp = trow + t0, *qp = qrow + t0;
             int done = 0;
@@ -377,18 +499,18 @@ __global__ void __launch_bounds__(kAggThreads) terminal_kernel(TerminalArgs a, G
                     Elem<T>::unpack(ld_stream(reinterpret_cast<const uint4 *>(qp) + idx), vq);
 #pragma unroll
                     for (int e = 0; e < NV; ++e) {
-                        const float diff =
-                            __fmul_rn(ex2((vp[e] - st.x) * a.s), st.y) - __fmul_rn(ex2((vq[e] - st.z) * a.s), st.w);
+                        const float diff = __fmul_rn(ex2(__fmaf_rn(vp[e], a.s, -st.x)), st.y) -
+                                           __fmul_rn(ex2(__fmaf_rn(vq[e], a.s, -st.z)), st.w);
                         const int t = idx * NV + e;
-                        sm.d[t] = G.slice_w ? diff : __fmul_rn(diff, G.inv_deg[t0 + t]);
+                        sm.d[t] = G.ent_w ? diff : __fmul_rn(diff, G.inv_deg[t0 + t]);
                     }
                 }
                 done = nvec * NV;
             }
             for (int t = done + tid; t < ns; t += NT) {
-                const float diff = __fmul_rn(ex2((Elem<T>::widen(tp[t]) - st.x) * a.s), st.y) -
-                                   __fmul_rn(ex2((Elem<T>::widen(qp[t]) - st.z) * a.s), st.w);
-                sm.d[t] = G.slice_w ? diff : __fmul_rn(diff, G.inv_deg[t0 + t]);
+                const float diff = __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(tp[t]), a.s, -st.x)), st.y) -
+                                   __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qp[t]), a.s, -st.z)), st.w);
+                sm.d[t] = G.ent_w ? diff : __fmul_rn(diff, G.inv_deg[t0 + t]);
             }
             __syncthreads();
         } else {
@@ -397,10 +519,10 @@ __global__ void __launch_bounds__(kAggThreads) terminal_kernel(TerminalArgs a, G
             cluster.sync();
             float m = kNegInf;
             for (int r = 0; r < C; ++r) m = fmaxf(m, (float)*cluster.map_shared_rank(&sm.xchg[1], r));
-            m_tgt = m;
+            rs_tgt = m * a.s;
             for (int t = tid; t < ns; t += NT) {
-                const float e = ex2((sm.d[t] - m) * a.s);
-                sm.d[t] = G.slice_w ? e : __fmul_rn(e, G.inv_deg[t0 + t]);
+                const float e = ex2(__fmaf_rn(sm.d[t], a.s, -rs_tgt));
+                sm.d[t] = G.ent_w ? e : __fmul_rn(e, G.inv_deg[t0 + t]);
             }
             __syncthreads();
         }
@@ -490,7 +612,7 @@ __global__ void __launch_bounds__(kAggThreads) terminal_kernel(TerminalArgs a, G
             auto omega = [&](int k) -> float {
                 const int t = G.group_tok[lo + k];
                 const float w = G.pair_w ? G.pair_w[lo + k] : G.inv_deg[t];
-                return __fmul_rn(ex2((Elem<T>::widen(trow[t]) - m_tgt) * a.s), w);
+                return __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs_tgt)), w);
             };
             double wsum = 0.0;
             int wlast = -1;
@@ -565,8 +687,8 @@ static pcg_status check_common(const pcg_groups *groups, pcg_dtype dtype, float 
         set_error("%s: dtype must be PCG_F32 or PCG_BF16", who);
         return PCG_ERR_INVALID_ARG;
     }
-    if (!(temperature > 0.f) || !std::isfinite(temperature)) {
-        set_error("%s: temperature must be positive and finite", who);
+    if (!(temperature >= 1e-6f) || !std::isfinite(temperature)) {
+        set_error("%s: temperature must be finite and at least 1e-6", who);
         return PCG_ERR_INVALID_ARG;
     }
     int dev = -1;
@@ -714,7 +836,8 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
     if (stage_events) e = cudaEventRecord((cudaEvent_t)stage_events[0], cs);
     if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
 
-    PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, w.accept, w.labels, w.posflags, w.stats};
+    PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K,       s,
+                    32.0f / s,     w.accept,     w.labels,     w.posflags, w.stats};
     if (dtype == PCG_F32)
         position_kernel<float><<<B * K, kPosThreads, 0, cs>>>(pa, G);
     else
