@@ -46,6 +46,7 @@ struct pcg_groups {
     pcg::GroupsDev dev;
     int64_t nnz;
     int device;
+    int sm_count;
     int max_group_size;
     int max_degree;
     int64_t device_bytes;

@@ -316,6 +316,8 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     h->dev.rev_w = w.empty() ? nullptr : (const float *)(base + o_rw);
     h->nnz = nnz;
     h->device = device;
+    h->sm_count = 1;
+    cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device);
     h->max_group_size = max_group;
     h->max_degree = max_deg;
     h->device_bytes = (int64_t)total;

@@ -13,6 +13,7 @@
 // pcg_group_probs uses the same token-sliced aggregation to write P of every row.
 #include <cooperative_groups.h>
 
+#include <algorithm>
 #include <cmath>
 
 #include "pcg_common.cuh"
@@ -21,121 +22,70 @@ namespace cg = cooperative_groups;
 
 namespace pcg {
 
-constexpr int kPosThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // ================================================================ position kernel ==========================
 //
-// Per row the kernel needs Z = sum_t 2^(l_t*s - RS) for SOME reference RS (any value works as long as the same
-// RS is used for the group masses: it cancels in P = S/Z), so each thread keeps a lazy reference: the largest
-// logit of its first vector, raised only when a later logit exceeds it by more than 32/s (a factor 2^32 of
-// headroom).  After the first vector the rescale branch is practically never taken, which keeps the special-
-// function unit at exactly one ex2 per logit.  Logits travel global -> shared through a per-thread ring of
-// 16-byte cp.async copies (kStages deep) so that many loads stay in flight without holding registers.
+// Per row the kernel needs Z = sum_t 2^(l_t*s - RS) for SOME reference RS: any value works as long as the same
+// RS is used for the group masses, because it cancels in P = S/Z.  So no running maximum is kept.  Each thread
+// holds a reference rs; it adds the terms of a 16-byte vector relative to rs and only then looks at their
+// sum: a sum above 2^32 (or an overflow to +inf) means some logit sits far above the reference, and the thread
+// redoes that one vector after raising rs to the vector's maximum (rescaling what it has summed so far).
+// That happens on a thread's first vector and practically never again, so the fast path costs exactly one
+// ex2 per logit and no max instructions.  Terms therefore stay below 2^32 and Z below V * 2^32.
+//
+// A block handles one drafted position: its first half streams the target row, its second half the draft row,
+// with 128-bit loads issued one batch (kBatch vectors per thread) ahead of the arithmetic.  The chain of
+// dependent loads that leads from the draft token to the label group's logits (token -> its groups -> label ->
+// group's token list -> logits) is spread over the streaming loop, one hop per batch, so its latency is hidden.
 
-constexpr int kStages = 8;
-constexpr float kRefInit = -1.0e30f;  // "no logit seen yet"; finite so that -inf logits give 2^-inf = 0, not NaN
+constexpr int kPosThreads = 256;
+constexpr int kHalf = kPosThreads / 2;
+constexpr int kBatch = 4;
+constexpr float kRefInit = -1.0e30f;     // "no logit seen yet": finite, so that -inf logits give 2^-inf = 0, not NaN
+constexpr float kVecSumLimit = 4294967296.f;  // 2^32
 
 struct RefSum {
-    float r;    // raw-logit reference
-    float rs;   // r * s as computed once (the exponent actually subtracted)
-    float thr;  // r + 32/s: logits above this raise the reference
+    float rs;   // scaled reference: the exponent subtracted from l*s
     float acc;  // sum of 2^(l*s - rs)
 };
 
-__device__ __forceinline__ void raise_ref(RefSum &st, float vm, float s, float headroom) {
-    const float nrs = vm * s;
-    st.acc *= ex2(st.rs - nrs);
-    st.r = vm;
-    st.rs = nrs;
-    st.thr = vm + headroom;
-}
-
 template <int NV>
-__device__ __forceinline__ void absorb(RefSum &st, const float (&v)[NV], float s, float headroom) {
+__device__ __forceinline__ void absorb_slow(RefSum &st, const float (&v)[NV], float s) {
     float vm = v[0];
 #pragma unroll
     for (int i = 1; i < NV; ++i) vm = fmaxf(vm, v[i]);
-    if (vm > st.thr) raise_ref(st, vm, s, headroom);
-#pragma unroll
-    for (int i = 0; i < NV; ++i) st.acc += ex2(__fmaf_rn(v[i], s, -st.rs));
-}
-
-__device__ __forceinline__ void absorb1(RefSum &st, float l, float s, float headroom) {
-    if (l > st.thr) raise_ref(st, l, s, headroom);
-    st.acc += ex2(__fmaf_rn(l, s, -st.rs));
-}
-
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
-    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-// Where the 16-byte vectors of a row start and how many there are.
-template <typename T>
-struct RowSplit {
-    int head, nvec;
-    const uint4 *vp;
-    __device__ __forceinline__ RowSplit(const T *row, int V) {
-        head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
-        if (head > V) head = V;
-        nvec = (V - head) / Elem<T>::kPerVec;
-        vp = reinterpret_cast<const uint4 *>(row + head);
+    if (vm > kNegInf) {  // (a vector of -inf only adds zeros and cannot get here)
+        const float nrs = vm * s;
+        st.acc *= ex2(st.rs - nrs);
+        st.rs = nrs;
     }
-};
+    float vs = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) vs += ex2(__fmaf_rn(v[i], s, -st.rs));
+    st.acc += vs;
+}
 
-// Deterministic block-wide combine of (rs, acc) pairs of TWO rows at once: xor butterfly inside a warp, then a
-// fixed-order pass over the warps.  `scratch` holds 4*NWARPS floats.  Every thread returns the same values.
+template <int NV>
+__device__ __forceinline__ void absorb(RefSum &st, const float (&v)[NV], float s) {
+    float vs = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) vs += ex2(__fmaf_rn(v[i], s, -st.rs));
+    if (vs <= kVecSumLimit)
+        st.acc += vs;
+    else  // reference too low for this vector (always so for a thread's first vector): raise it and redo
+        absorb_slow<NV>(st, v, s);
+}
+
+__device__ __forceinline__ void absorb1(RefSum &st, float l, float s) {
+    const float v[1] = {l};
+    absorb<1>(st, v, s);
+}
+
 __device__ __forceinline__ void merge(float &rs, float &acc, float rs2, float acc2) {
     const float m = fmaxf(rs, rs2);
     acc = acc * ex2(rs - m) + acc2 * ex2(rs2 - m);
     rs = m;
-}
-
-template <int NT>
-__device__ __forceinline__ void block_combine2(float &rs_a, float &acc_a, float &rs_b, float &acc_b, float *scratch) {
-    constexpr int NW = NT / 32;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        merge(rs_a, acc_a, __shfl_xor_sync(0xffffffffu, rs_a, o), __shfl_xor_sync(0xffffffffu, acc_a, o));
-        merge(rs_b, acc_b, __shfl_xor_sync(0xffffffffu, rs_b, o), __shfl_xor_sync(0xffffffffu, acc_b, o));
-    }
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) {
-        float *p = scratch + 4 * (threadIdx.x >> 5);
-        p[0] = rs_a, p[1] = acc_a, p[2] = rs_b, p[3] = acc_b;
-    }
-    __syncthreads();
-    rs_a = scratch[0], acc_a = scratch[1], rs_b = scratch[2], acc_b = scratch[3];
-#pragma unroll
-    for (int w = 1; w < NW; ++w) {
-        merge(rs_a, acc_a, scratch[4 * w], scratch[4 * w + 1]);
-        merge(rs_b, acc_b, scratch[4 * w + 2], scratch[4 * w + 3]);
-    }
-}
-
-template <int NT>
-__device__ __forceinline__ void block_sum2(float &a, float &b, float *scratch) {
-    constexpr int NW = NT / 32;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        a += __shfl_xor_sync(0xffffffffu, a, o);
-        b += __shfl_xor_sync(0xffffffffu, b, o);
-    }
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) {
-        scratch[2 * (threadIdx.x >> 5)] = a;
-        scratch[2 * (threadIdx.x >> 5) + 1] = b;
-    }
-    __syncthreads();
-    a = scratch[0], b = scratch[1];
-#pragma unroll
-    for (int w = 1; w < NW; ++w) a += scratch[2 * w], b += scratch[2 * w + 1];
 }
 
 struct PositionArgs {
@@ -145,7 +95,6 @@ struct PositionArgs {
     const float *uniforms;   // [B, K+1, 2]
     int K;
     float s;                 // log2(e) / temperature
-    float headroom;          // 32 / s
     int32_t *accept;         // [B*K] 1 = accepted
     int32_t *labels;         // [B*K] group label of the draft token
     int32_t *posflags;       // [B*K]
@@ -153,114 +102,167 @@ struct PositionArgs {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kPosThreads, 5) position_kernel(PositionArgs a, GroupsDev G) {
-    constexpr int NT = kPosThreads;
+__global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a, GroupsDev G) {
+    constexpr int NT = kPosThreads, H = kHalf, NW = NT / 32, HW = H / 32;
     constexpr int NV = Elem<T>::kPerVec;
-    constexpr int S = kStages;
-    __shared__ uint4 ring[S][NT];
-    __shared__ float scratch[4 * (NT / 32)];
-    __shared__ int sh_label, sh_flag;
+    constexpr int U = kBatch;
+    constexpr int kChainSteps = 6;
+    __shared__ float red_z[2 * NW];
+    __shared__ float red_s[NW];
     const int tid = threadIdx.x;
+    const int half = tid / H, htid = tid - half * H;  // 0: target row, 1: draft row (warp-uniform)
+    const int V = G.V, K = a.K;
+    const float s = a.s;
     const int pos = blockIdx.x;
-    const int b = pos / a.K, i = pos - b * a.K;
-    const int V = G.V;
-    const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (a.K + 1) + i) * V;
-    const T *qrow = reinterpret_cast<const T *>(a.draft) + (int64_t)pos * V;
-    const float *u = a.uniforms + ((int64_t)b * (a.K + 1) + i) * 2;
-    const float s = a.s, headroom = a.headroom;
+    const int b = pos / K, i = pos - b * K;
+    const T *row = half ? reinterpret_cast<const T *>(a.draft) + (int64_t)pos * V
+                        : reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + i) * V;
+    const float *u = a.uniforms + ((int64_t)b * (K + 1) + i) * 2;
 
-    // ---- start streaming: the two rows form one sequence of 2*nk vector slots per thread ----
-    const RowSplit<T> ts(trow, V), qs(qrow, V);
-    const int nk_t = (ts.nvec + NT - 1) / NT, nk_q = (qs.nvec + NT - 1) / NT, nk = nk_t + nk_q;
-    auto issue = [&](int k) {
-        if (k < nk) {
-            const bool second = k >= nk_t;
-            const int idx = tid + (second ? k - nk_t : k) * NT;
-            if (idx < (second ? qs.nvec : ts.nvec)) cp_async16(&ring[k % S][tid], (second ? qs.vp : ts.vp) + idx);
-        }
-        cp_async_commit();
-    };
-#pragma unroll
-    for (int k = 0; k < S - 1; ++k) issue(k);
-
-    if (tid == 0) {
-        // group-label coupling: the label is drawn from the groups of the draft token with its split weights
-        int x = a.draft_tokens[pos], flag = 0;
-        if (x < 0 || x >= V) {
-            x = 0;
-            flag = PCG_FLAG_BAD_DRAFT_TOKEN;
-        }
-        const int r0 = G.rev_ptr[x], N = G.rev_ptr[x + 1] - r0;
-        int j;
-        if (!G.rev_w) {
-            j = (int)floor((double)u[0] * (double)N);  // exact: a float times a small integer fits a double
-            j = min(max(j, 0), N - 1);
-        } else {
-            double tot = 0.0, run = 0.0;
-            for (int e = 0; e < N; ++e) tot += (double)G.rev_w[r0 + e];
-            const double target = (double)u[0] * tot;
-            j = -1;
-            int last_pos = 0;
-            for (int e = 0; e < N; ++e) {
-                const double w = (double)G.rev_w[r0 + e];
-                if (w > 0.0) last_pos = e;
-                run += w;
-                if (run > target) {
-                    j = e;
-                    break;
+    // ---- dependent-load chain towards the label group's logits (every thread, redundantly) ----
+    int c_x = 0, c_r0 = 0, c_n = 1, c_g = 0, c_lo = 0, c_hi = 0, c_t = 0, c_flag = 0;
+    float c_u0 = 0.f, c_u1 = 0.f, c_l = kNegInf, c_w = 0.f;
+    auto chain = [&](int step) {
+        switch (step) {
+            case 0:
+                c_x = a.draft_tokens[pos];
+                c_u0 = u[0];
+                c_u1 = u[1];
+                break;
+            case 1:
+                if (c_x < 0 || c_x >= V) {
+                    c_x = 0;
+                    c_flag = PCG_FLAG_BAD_DRAFT_TOKEN;
                 }
+                c_r0 = G.rev_ptr[c_x];
+                c_n = G.rev_ptr[c_x + 1] - c_r0;
+                break;
+            case 2: {
+                // group-label coupling: the label is drawn from the groups of the draft token
+                int j;
+                if (!G.rev_w) {
+                    j = (int)floor((double)c_u0 * (double)c_n);  // exact: float times small integer in double
+                    j = min(max(j, 0), c_n - 1);
+                } else {
+                    double tot = 0.0, run = 0.0;
+                    for (int e = 0; e < c_n; ++e) tot += (double)G.rev_w[c_r0 + e];
+                    const double target = (double)c_u0 * tot;
+                    j = -1;
+                    int last_pos = 0;
+                    for (int e = 0; e < c_n; ++e) {
+                        const double w = (double)G.rev_w[c_r0 + e];
+                        if (w > 0.0) last_pos = e;
+                        run += w;
+                        if (run > target) {
+                            j = e;
+                            break;
+                        }
+                    }
+                    if (j < 0) j = last_pos;
+                }
+                c_g = G.rev_grp[c_r0 + j];
+                break;
             }
-            if (j < 0) j = last_pos;
+            case 3:
+                c_lo = G.group_ptr[c_g];
+                c_hi = G.group_ptr[c_g + 1];
+                break;
+            case 4:
+                if (c_lo + htid < c_hi) c_t = G.group_tok[c_lo + htid];
+                break;
+            case 5:
+                if (c_lo + htid < c_hi) {
+                    c_l = Elem<T>::widen(row[c_t]);
+                    c_w = G.pair_w ? G.pair_w[c_lo + htid] : G.inv_deg[c_t];
+                }
+                break;
         }
-        sh_label = G.rev_grp[r0 + j];
-        sh_flag = flag;
-    }
+    };
 
-    RefSum st_t{kRefInit, kRefInit * s, kRefInit, 0.f}, st_q = st_t;
-    for (int k = 0; k < nk; ++k) {
-        issue(k + S - 1);
-        cp_async_wait<S - 1>();
-        const bool second = k >= nk_t;
-        const int idx = tid + (second ? k - nk_t : k) * NT;
-        if (idx < (second ? qs.nvec : ts.nvec)) {
+    // ---- stream the row: elements before the first 16-byte boundary, whole vectors, the rest ----
+    RefSum st{kRefInit * s, 0.f};
+    int chained = 0;
+    int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
+    if (head > V) head = V;
+    const int nvec = (V - head) / NV;
+    const int nfull = nvec / (H * U);  // batches in which every thread has all U vectors
+    {
+        const uint4 *p = reinterpret_cast<const uint4 *>(row + head) + htid;
+        uint4 cur[U], nxt[U];
+        if (nfull > 0) {
+#pragma unroll
+            for (int j = 0; j < U; ++j) cur[j] = ld_stream(p + j * H);
+        }
+        for (int bi = 0; bi < nfull; ++bi) {
+            p += H * U;
+            if (bi + 1 < nfull) {
+#pragma unroll
+                for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * H);
+            }
+            if (chained < kChainSteps) chain(chained++);
+#pragma unroll
+            for (int j = 0; j < U; ++j) {
+                float v[NV];
+                Elem<T>::unpack(cur[j], v);
+                absorb<NV>(st, v, s);
+            }
+#pragma unroll
+            for (int j = 0; j < U; ++j) cur[j] = nxt[j];
+        }
+        // remaining whole vectors (fewer than H*U), then the scalar head and tail
+        for (int idx = nfull * H * U + htid; idx < nvec; idx += H) {
             float v[NV];
-            Elem<T>::unpack(ring[k % S][tid], v);
-            if (second)
-                absorb<NV>(st_q, v, s, headroom);
-            else
-                absorb<NV>(st_t, v, s, headroom);
+            Elem<T>::unpack(ld_stream(reinterpret_cast<const uint4 *>(row + head) + idx), v);
+            absorb<NV>(st, v, s);
         }
+        for (int t = htid; t < head; t += H) absorb1(st, Elem<T>::widen(row[t]), s);
+        for (int t = head + nvec * NV + htid; t < V; t += H) absorb1(st, Elem<T>::widen(row[t]), s);
     }
-    // elements before the first and after the last whole 16-byte vector of each row
-    for (int t = tid; t < ts.head; t += NT) absorb1(st_t, Elem<T>::widen(trow[t]), s, headroom);
-    for (int t = ts.head + ts.nvec * NV + tid; t < V; t += NT) absorb1(st_t, Elem<T>::widen(trow[t]), s, headroom);
-    for (int t = tid; t < qs.head; t += NT) absorb1(st_q, Elem<T>::widen(qrow[t]), s, headroom);
-    for (int t = qs.head + qs.nvec * NV + tid; t < V; t += NT) absorb1(st_q, Elem<T>::widen(qrow[t]), s, headroom);
+    while (chained < kChainSteps) chain(chained++);
 
-    float rs_p = st_t.rs, Zp = st_t.acc, rs_q = st_q.rs, Zq = st_q.acc;
-    block_combine2<NT>(rs_p, Zp, rs_q, Zq, scratch);  // its barriers also publish sh_label
+    // ---- per-row (rs, Z): xor butterfly inside a warp, then a fixed-order pass over each half's warps ----
+    float rs = st.rs, Z = st.acc;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) merge(rs, Z, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, Z, o));
+    if ((tid & 31) == 0) {
+        red_z[2 * (tid >> 5)] = rs;
+        red_z[2 * (tid >> 5) + 1] = Z;
+    }
+    __syncthreads();
+    float rs_p = red_z[0], Zp = red_z[1], rs_q = red_z[2 * HW], Zq = red_z[2 * HW + 1];
+#pragma unroll
+    for (int w = 1; w < HW; ++w) {
+        merge(rs_p, Zp, red_z[2 * w], red_z[2 * w + 1]);
+        merge(rs_q, Zq, red_z[2 * (HW + w)], red_z[2 * (HW + w) + 1]);
+    }
 
-    // ---- masses of the label group under both rows: a handful of gathered logits ----
-    const int g = sh_label;
-    const int lo = G.group_ptr[g], hi = G.group_ptr[g + 1];
-    float Sp = 0.f, Sq = 0.f;
-    for (int k = lo + tid; k < hi; k += NT) {
+    // ---- mass of the label group under this half's row (first element prefetched by the chain) ----
+    const float rs_mine = half ? rs_q : rs_p;
+    float part = __fmul_rn(ex2(__fmaf_rn(c_l, s, -rs_mine)), c_w);
+    for (int k = c_lo + htid + H; k < c_hi; k += H) {  // groups larger than half a block
         const int t = G.group_tok[k];
         const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
-        Sp += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs_p)), w);
-        Sq += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), s, -rs_q)), w);
+        part += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(row[t]), s, -rs_mine)), w);
     }
-    block_sum2<NT>(Sp, Sq, scratch);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if ((tid & 31) == 0) red_s[tid >> 5] = part;
+    __syncthreads();
 
     if (tid == 0) {
+        float Sp = red_s[0], Sq = red_s[HW];
+        for (int w = 1; w < HW; ++w) {
+            Sp += red_s[w];
+            Sq += red_s[HW + w];
+        }
         // acceptance u < min(1, P/Q) without a division: P = Sp/Zp, Q = Sq/Zq
         const float lhs = Sp * Zq, rhs = Sq * Zp;
-        const int acc = (lhs >= rhs) || (u[1] * rhs < lhs);
-        int flag = sh_flag;
+        const int acc = (lhs >= rhs) || (c_u1 * rhs < lhs);
+        int flag = c_flag;
         if (!(Zp > 0.f) || !(Zq > 0.f) || isinf(Zp) || isinf(Zq) || isinf(rs_p) || isinf(rs_q))
             flag |= PCG_FLAG_NONFINITE;
         a.accept[pos] = acc;
-        a.labels[pos] = g;
+        a.labels[pos] = c_g;
         a.posflags[pos] = flag;
         a.stats[pos] = make_float4(rs_p, 1.0f / Zp, rs_q, 1.0f / Zq);
     }
@@ -836,8 +838,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
     if (stage_events) e = cudaEventRecord((cudaEvent_t)stage_events[0], cs);
     if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
 
-    PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K,       s,
-                    32.0f / s,     w.accept,     w.labels,     w.posflags, w.stats};
+    PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, w.accept, w.labels, w.posflags, w.stats};
     if (dtype == PCG_F32)
         position_kernel<float><<<B * K, kPosThreads, 0, cs>>>(pa, G);
     else
