@@ -180,6 +180,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C5", choices=sorted(W.CONFIGS))
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (profiling only)")
+    ap.add_argument("--mode", default="default", choices=["default", "dense", "cluster"],
+                    help="pcg_verify mode of the timed steps (the headline is 'default')")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -231,13 +233,16 @@ def main():
     x, u = h_x.cuda(), h_u.cuda()
     B, K, V, M = cfg.B, cfg.K, cfg.V, groups.M
     dt_code = binding.PCG_BF16 if bf16 else binding.PCG_F32
-    ws = torch.empty(binding.pcg_verify_workspace_bytes(B, K, V, M, dt_code), dtype=torch.uint8, device="cuda")
+    mode = {"default": binding.VERIFY_DEFAULT, "dense": binding.VERIFY_DENSE,
+            "cluster": binding.VERIFY_CLUSTER_TERMINAL}[args.mode]
+    ws = torch.empty(binding.pcg_verify_workspace_bytes(B, K, V, M, dt_code, mode), dtype=torch.uint8, device="cuda")
     out = (torch.empty(B, dtype=torch.int32, device="cuda"), torch.empty((B, K + 1), dtype=torch.int32, device="cuda"),
            torch.empty((B, K + 1), dtype=torch.int32, device="cuda"), torch.empty(B, dtype=torch.int32, device="cuda"))
     esz = 2 if bf16 else 4
 
     def step(events=None):
-        binding.pcg_verify(tl, dl, x, handle, u, cfg.temperature, workspace=ws, out=out, stage_events=events)
+        binding.pcg_verify(tl, dl, x, handle, u, cfg.temperature, workspace=ws, out=out, stage_events=events,
+                           mode=mode)
 
     def barrier():
         if dist is not None:
@@ -287,6 +292,11 @@ def main():
     h2d = (B * (2 * K + 1) * V * esz) + B * K * 4 + B * (K + 1) * 8
     d2h = B * 4 * 2 + B * (K + 1) * 4 * 2
 
+    # kernels launched by one pcg_verify call (see pcg_verify in csrc/pcg_kernels.cu)
+    info = handle.info
+    chunk_unit = 128 if B >= 128 else 32
+    chunk = min(-(-B // chunk_unit) * chunk_unit, max(chunk_unit, ((64 << 20) // (V * 4)) // chunk_unit * chunk_unit))
+    launches_per_step = {"default": 1 + 1 + 2 * (-(-B // chunk)) + 1, "cluster": 2, "dense": 2 + 1 + 1 + 1}[args.mode]
     if rank == 0:
         peak, peak_src = hbm_peak()
         alg_bytes = B * K * 2 * V * esz  # per drafted position: one target and one draft row, read once
@@ -304,11 +314,12 @@ def main():
                          "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": alg_bytes,
                          "avg_launch_ms": pos_ms},
-            "stages_ms": {"position_kernel": pos_ms, "terminal_kernel": term_ms},
+            "stages_ms": {"per_position_stage": pos_ms, "per_sequence_stage": term_ms},
+            "mode": args.mode,
             "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
                     "api": "pcg_verify_host (pinned host tensors)"},
-            "gpu_launches": 2 * args.steps,
+            "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
             "mean_accept_len": float(accept_len.mean()),
         }

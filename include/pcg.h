@@ -52,8 +52,13 @@ typedef struct CUevent_st *pcg_event;
 #define PCG_FLAG_NONFINITE 4       /* a row's maximum or normaliser was not finite (NaN/+inf logits, or all -inf) */
 
 /* Bits of the `mode` argument of pcg_verify. */
-#define PCG_VERIFY_DEFAULT 0u
-#define PCG_VERIFY_DENSE 1u /* form P and Q of ALL groups at EVERY position (through the workspace) */
+#define PCG_VERIFY_DEFAULT 0u /* per position only the label group's P and Q are formed (what the accept test
+                                 needs); all groups are aggregated once per sequence, at its terminal position */
+#define PCG_VERIFY_DENSE 1u   /* form P and Q of ALL groups at EVERY position (stored in the workspace), then take
+                                 the same decisions from the stored vectors */
+#define PCG_VERIFY_CLUSTER_TERMINAL 2u /* default mode, but the per-sequence stage runs as one thread-block cluster
+                                 per sequence instead of the batched transpose / sparse-product / draw kernels
+                                 (lower latency for a handful of sequences); not combinable with DENSE */
 
 /*
  * Group membership: the Acoustic Similarity Groups as a group->token CSR plus

@@ -23,6 +23,7 @@ namespace cg = cooperative_groups;
 namespace pcg {
 
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr size_t kMaxDynSmem = 227 * 1024;  // dynamic shared memory a block may opt in to
 
 // ================================================================ position kernel ==========================
 //
@@ -101,6 +102,33 @@ struct PositionArgs {
     float4 *stats;           // [B*K] (RS_p, 1/Z_p, RS_q, 1/Z_q): scaled reference and reciprocal normaliser
 };
 
+// Group-label coupling: the label of draft token x is drawn from the groups containing x (reverse membership
+// entries [r0, r0+n), ascending group id) -- uniformly for the equal split, by inverse CDF over w_{.,x} otherwise.
+__device__ __forceinline__ int draw_label(const GroupsDev &G, int r0, int n, float u0) {
+    int j;
+    if (!G.rev_w) {
+        j = (int)floor((double)u0 * (double)n);  // exact: float times small integer in double
+        j = min(max(j, 0), n - 1);
+    } else {
+        double tot = 0.0, run = 0.0;
+        for (int e = 0; e < n; ++e) tot += (double)G.rev_w[r0 + e];
+        const double target = (double)u0 * tot;
+        j = -1;
+        int last_pos = 0;
+        for (int e = 0; e < n; ++e) {
+            const double w = (double)G.rev_w[r0 + e];
+            if (w > 0.0) last_pos = e;
+            run += w;
+            if (run > target) {
+                j = e;
+                break;
+            }
+        }
+        if (j < 0) j = last_pos;
+    }
+    return G.rev_grp[r0 + j];
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a, GroupsDev G) {
     constexpr int NT = kPosThreads, H = kHalf, NW = NT / 32, HW = H / 32;
@@ -137,32 +165,9 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
                 c_r0 = G.rev_ptr[c_x];
                 c_n = G.rev_ptr[c_x + 1] - c_r0;
                 break;
-            case 2: {
-                // group-label coupling: the label is drawn from the groups of the draft token
-                int j;
-                if (!G.rev_w) {
-                    j = (int)floor((double)c_u0 * (double)c_n);  // exact: float times small integer in double
-                    j = min(max(j, 0), c_n - 1);
-                } else {
-                    double tot = 0.0, run = 0.0;
-                    for (int e = 0; e < c_n; ++e) tot += (double)G.rev_w[c_r0 + e];
-                    const double target = (double)c_u0 * tot;
-                    j = -1;
-                    int last_pos = 0;
-                    for (int e = 0; e < c_n; ++e) {
-                        const double w = (double)G.rev_w[c_r0 + e];
-                        if (w > 0.0) last_pos = e;
-                        run += w;
-                        if (run > target) {
-                            j = e;
-                            break;
-                        }
-                    }
-                    if (j < 0) j = last_pos;
-                }
-                c_g = G.rev_grp[c_r0 + j];
+            case 2:
+                c_g = draw_label(G, c_r0, c_n, c_u0);
                 break;
-            }
             case 3:
                 c_lo = G.group_ptr[c_g];
                 c_hi = G.group_ptr[c_g + 1];
@@ -678,6 +683,545 @@ __global__ void __launch_bounds__(kAggThreads, 2) terminal_kernel(TerminalArgs a
     cluster.sync();  // no block may exit while another still reads its shared memory
 }
 
+// ================================================================ batched terminal stage ====================
+//
+// The terminal draw of a sequence needs the residual (P - Q)_+ of ALL groups at one position (the first
+// rejection, or the bonus row).  Over a batch that is one sparse-matrix product: R[b, g] = sum_{t in G_g}
+// D[b, t], with D[b, t] = (p(t) - q(t)) / N(t) at sequence b's terminal position.  Four kernels:
+//   terminal_prepare_kernel    one block per sequence: warp ballot over the accept bits -> first rejection n_b;
+//                              if everything was accepted, the softmax statistics of the bonus row
+//   residual_transpose_kernel  re-reads the two rows of every sequence's terminal position and writes D
+//                              TRANSPOSED, Dt[t, b]: the sequences of a chunk side by side in one line
+//   group_spmm_kernel          one warp per (4 groups, block of sequences): walks the groups' token lists once
+//                              and adds one fully used line of Dt per token (Dt stays in L2)
+//   terminal_draw_kernel       one block per sequence: prefix scan over the M residual masses, group draw,
+//                              within-group token draw, outputs
+// Sequences are processed in chunks whose Dt fits in L2.
+
+constexpr int kPrepThreads = 256;  // terminal_prepare_kernel
+constexpr int kTrThreads = 256;    // residual_transpose_kernel
+constexpr int kSpmmThreads = 256;  // group_spmm_kernel: 8 warps, one group each
+#ifndef PCG_SPMM_SPL
+#define PCG_SPMM_SPL 4    // sequences per lane of the sparse product for batches of at least 32 * PCG_SPMM_SPL
+#endif
+#ifndef PCG_SPMM_DEPTH
+#define PCG_SPMM_DEPTH 8  // loads of Dt in flight per lane
+#endif
+constexpr int kSpmmWide = PCG_SPMM_SPL;
+constexpr int kSpmmDepth = PCG_SPMM_DEPTH;
+constexpr int kDrawThreads = 512;  // terminal_draw_kernel
+
+struct PrepareArgs {
+    const void *target;
+    int K;
+    float s;
+    int want_bonus_stats;  // 0 in dense mode (the stored P of the bonus row is used instead)
+    const int32_t *accept;
+    const int32_t *posflags;
+    const float4 *stats;
+    int32_t *term_n;      // [B] first rejected position, K if none
+    int32_t *term_flags;  // [B] flags of the positions up to and including n
+    float4 *term_stats;   // [B] (RS_p, 1/Z_p, RS_q, 1/Z_q) of the terminal position; (RS_p, 1/Z_p, 0, 0) for a bonus row
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kPrepThreads) terminal_prepare_kernel(PrepareArgs a, GroupsDev G) {
+    constexpr int NT = kPrepThreads, NW = NT / 32, NV = Elem<T>::kPerVec;
+    __shared__ int s_n, s_flags;
+    __shared__ float red[2 * NW];
+    const int b = blockIdx.x, tid = threadIdx.x, K = a.K, V = G.V;
+    // ---- first rejected position: one ballot over the K <= 32 accept bits ----
+    if (tid < 32) {
+        const int rej = (tid < K) && (a.accept[b * K + tid] == 0);
+        const unsigned mask = __ballot_sync(0xffffffffu, rej);
+        const int n = mask ? (__ffs(mask) - 1) : K;
+        const int f = (tid < K && tid <= n) ? a.posflags[b * K + tid] : 0;
+        const int flags = __reduce_or_sync(0xffffffffu, f);
+        if (tid == 0) {
+            s_n = n;
+            s_flags = flags;
+        }
+    }
+    __syncthreads();
+    const int n = s_n;
+    if (n < K || !a.want_bonus_stats) {
+        if (tid == 0) {
+            a.term_n[b] = n;
+            a.term_flags[b] = s_flags;
+            a.term_stats[b] = n < K ? a.stats[b * K + n] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        return;
+    }
+    // ---- every position accepted: softmax statistics of the bonus row (target row K) ----
+    const T *row = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + K) * V;
+    RefSum st{kRefInit * a.s, 0.f};
+    int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
+    if (head > V) head = V;
+    const int nvec = (V - head) / NV;
+    const uint4 *vp = reinterpret_cast<const uint4 *>(row + head);
+    int idx = tid;
+    for (; idx + 3 * NT < nvec; idx += 4 * NT) {
+        uint4 r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) r[j] = ld_stream(vp + idx + j * NT);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float v[NV];
+            Elem<T>::unpack(r[j], v);
+            absorb<NV>(st, v, a.s);
+        }
+    }
+    for (; idx < nvec; idx += NT) {
+        float v[NV];
+        Elem<T>::unpack(ld_stream(vp + idx), v);
+        absorb<NV>(st, v, a.s);
+    }
+    for (int t = tid; t < head; t += NT) absorb1(st, Elem<T>::widen(row[t]), a.s);
+    for (int t = head + nvec * NV + tid; t < V; t += NT) absorb1(st, Elem<T>::widen(row[t]), a.s);
+    float rs = st.rs, Z = st.acc;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) merge(rs, Z, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, Z, o));
+    if ((tid & 31) == 0) {
+        red[2 * (tid >> 5)] = rs;
+        red[2 * (tid >> 5) + 1] = Z;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        rs = red[0];
+        Z = red[1];
+        for (int w = 1; w < NW; ++w) merge(rs, Z, red[2 * w], red[2 * w + 1]);
+        int flags = s_flags;
+        if (!(Z > 0.f) || isinf(Z) || isinf(rs)) flags |= PCG_FLAG_NONFINITE;
+        a.term_n[b] = n;
+        a.term_flags[b] = flags;
+        a.term_stats[b] = make_float4(rs, 1.0f / Z, 0.f, 0.f);
+    }
+}
+
+// Loads of Dt: cached in L2 only (.cg).  Every line of Dt is read once per group its token belongs to, at
+// unrelated times, so it has to survive in L2 between those reads; the streaming form used for the logits
+// (ld.global.nc.L1::no_allocate) is retained in L2 for too short a time for that.
+__device__ __forceinline__ float ld_l2_f32(const float *p) {
+    float r;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(r) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ float4 ld_l2_f32x4(const float *p) {
+    float4 r;
+    asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w)
+                 : "l"(p));
+    return r;
+}
+#ifdef PCG_DT_STORE_EVICT_LAST
+__device__ __forceinline__ void st_dt(float *p, float v) {
+    uint64_t pol;
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(v), "l"(pol) : "memory");
+}
+#else
+__device__ __forceinline__ void st_dt(float *p, float v) { *p = v; }
+#endif
+
+struct TransposeArgs {
+    const void *target;
+    const void *draft;
+    int B, K;
+    int b0;             // first sequence of this chunk
+    int bpad;           // sequences per line of Dt (row stride of Dt, a multiple of 32)
+    float s;
+    const int32_t *term_n;
+    const float4 *term_stats;
+    float *Dt;          // [V, bpad]
+};
+
+// Grid (ceil(V / TT), bpad / 32): a tile of TT tokens x 32 sequences.  Warp w loads the row segments of
+// sequences w, w+8, w+16, w+24 (one 16-byte vector per lane), the tile is turned in shared memory (column
+// rotated by the vector index, so that both sides are free of bank conflicts) and written out one 128-byte
+// line per token.  Sequences past the end of the batch get zeros.
+template <typename T>
+__global__ void __launch_bounds__(kTrThreads) residual_transpose_kernel(TransposeArgs a, GroupsDev G) {
+    constexpr int NV = Elem<T>::kPerVec, TT = 32 * NV;
+    __shared__ float tile[TT * 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int V = G.V, K = a.K;
+    const int t0 = blockIdx.x * TT;
+    const int bbase = a.b0 + blockIdx.y * 32;
+    const int t = t0 + lane * NV;  // first token of this lane's vector
+    float invd[NV];
+#pragma unroll
+    for (int e = 0; e < NV; ++e) invd[e] = (!G.ent_w && t + e < V) ? G.inv_deg[t + e] : 1.f;
+    // all of this thread's loads first (4 sequences x 2 rows), then the arithmetic
+    int n[4];
+    float4 st[4];
+    uint4 rp[4], rq[4];
+    bool fast[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int b = bbase + warp + 8 * q;
+        n[q] = b < a.B ? a.term_n[b] : -1;
+        st[q] = b < a.B ? a.term_stats[b] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int b = bbase + warp + 8 * q;
+        const T *tp = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + max(n[q], 0)) * V + t;
+        const T *qp = reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(max(n[q], 0), K - 1)) * V + t;
+        fast[q] = n[q] >= 0 && t + NV <= V && (((uintptr_t)tp | (uintptr_t)qp) & 15u) == 0;
+        rp[q] = rq[q] = make_uint4(0u, 0u, 0u, 0u);
+        if (fast[q]) {
+            rp[q] = ld_stream(reinterpret_cast<const uint4 *>(tp));
+            if (n[q] < K) rq[q] = ld_stream(reinterpret_cast<const uint4 *>(qp));
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const int sl = warp + 8 * q;
+        float d[NV];
+#pragma unroll
+        for (int e = 0; e < NV; ++e) d[e] = 0.f;
+        if (n[q] >= 0 && t < V) {
+            const int b = bbase + sl;
+            float lp[NV], lq[NV];
+            const bool resid = n[q] < K;
+            if (fast[q]) {
+                Elem<T>::unpack(rp[q], lp);
+                Elem<T>::unpack(rq[q], lq);
+            } else {  // ragged end of the row or rows that are not 16-byte aligned
+                const T *tp = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n[q]) * V + t;
+                const T *qp = reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(n[q], K - 1)) * V + t;
+#pragma unroll
+                for (int e = 0; e < NV; ++e) {
+                    const bool in = t + e < V;
+                    lp[e] = in ? Elem<T>::widen(tp[e]) : kNegInf;
+                    lq[e] = (in && resid) ? Elem<T>::widen(qp[e]) : kNegInf;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < NV; ++e) {
+                float v = __fmul_rn(ex2(__fmaf_rn(lp[e], a.s, -st[q].x)), st[q].y);
+                if (resid) v -= __fmul_rn(ex2(__fmaf_rn(lq[e], a.s, -st[q].z)), st[q].w);
+                d[e] = __fmul_rn(v, invd[e]);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < NV; ++e) tile[(lane * NV + e) * 32 + ((sl + lane) & 31)] = d[e];
+    }
+    __syncthreads();
+    float *out = a.Dt + (size_t)blockIdx.y * 32 + lane;
+    for (int r = warp; r < TT; r += kTrThreads / 32) {
+        const int tok = t0 + r;
+        if (tok < V) st_dt(out + (size_t)tok * a.bpad, tile[r * 32 + ((lane + r / NV) & 31)]);
+    }
+}
+
+struct SpmmArgs {
+    const float *Dt;  // [V, bpad]
+    int B;
+    int b0;           // first sequence of this chunk
+    int bpad;
+    float *R;         // [B, M] (raw sums; the consumer clamps at zero)
+};
+
+template <int SPL>
+struct SeqVec;
+template <>
+struct SeqVec<1> {
+    float v[1];
+    __device__ __forceinline__ void load(const float *p) { v[0] = ld_l2_f32(p); }
+};
+template <>
+struct SeqVec<2> {
+    float v[2];
+    __device__ __forceinline__ void load(const float *p) {
+        asm volatile("ld.global.cg.v2.f32 {%0,%1}, [%2];" : "=f"(v[0]), "=f"(v[1]) : "l"(p));
+    }
+};
+template <>
+struct SeqVec<4> {
+    float v[4];
+    __device__ __forceinline__ void load(const float *p) {
+        const float4 r = ld_l2_f32x4(p);
+        v[0] = r.x, v[1] = r.y, v[2] = r.z, v[3] = r.w;
+    }
+};
+
+// Grid (ceil(M / 8), bpad / (32 * SPL)).  A warp owns one group and a block of 32 * SPL sequences; a lane
+// holds SPL consecutive sequences (one 4-, 8- or 16-byte load per token).  The warp fetches the group's token
+// list with coalesced loads (the next 32 tokens while the current ones are processed), then adds the tokens'
+// lines of Dt in CSR order, DEPTH loads in flight at a time.  The 8 x (32 * SPL) block of sums is turned in
+// shared memory so that R is written along the group index.
+#ifndef PCG_SPMM_MINBLOCKS
+#define PCG_SPMM_MINBLOCKS 4  // caps the registers so that 32 warps per SM are resident
+#endif
+template <int SPL, int DEPTH>
+__global__ void __launch_bounds__(kSpmmThreads, PCG_SPMM_MINBLOCKS) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
+    constexpr int NS = 32 * SPL;            // sequences per block
+    constexpr int GPB = kSpmmThreads / 32;  // groups per block
+    __shared__ float tile[GPB * (NS + 1)];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gblock = blockIdx.x * GPB;
+    const float *col = a.Dt + (size_t)blockIdx.y * NS + lane * SPL;
+    const int g = gblock + warp;
+    float acc[SPL];
+#pragma unroll
+    for (int q = 0; q < SPL; ++q) acc[q] = 0.f;
+    if (g < G.M) {  // warp-uniform
+        const int lo = G.group_ptr[g], hi = G.group_ptr[g + 1];
+        int tok_next = lo + lane < hi ? G.group_tok[lo + lane] : 0;
+        float w_next = (G.pair_w && lo + lane < hi) ? G.pair_w[lo + lane] : 1.f;
+        for (int k0 = lo; k0 < hi; k0 += 32) {
+            const int cnt = min(32, hi - k0);
+            const int tokv = tok_next;
+            const float wv = w_next;
+            if (k0 + 32 + lane < hi) {
+                tok_next = G.group_tok[k0 + 32 + lane];
+                if (G.pair_w) w_next = G.pair_w[k0 + 32 + lane];
+            }
+            for (int j0 = 0; j0 < cnt; j0 += DEPTH) {
+                SeqVec<SPL> x[DEPTH];
+#pragma unroll
+                for (int j = 0; j < DEPTH; ++j) {
+                    const int tok = __shfl_sync(0xffffffffu, tokv, (j0 + j) & 31);
+                    if (j0 + j < cnt) x[j].load(col + (size_t)tok * a.bpad);
+                }
+#pragma unroll
+                for (int j = 0; j < DEPTH; ++j) {
+                    const float w = __shfl_sync(0xffffffffu, wv, (j0 + j) & 31);
+                    if (j0 + j < cnt) {
+#pragma unroll
+                        for (int q = 0; q < SPL; ++q) acc[q] += G.pair_w ? __fmul_rn(x[j].v[q], w) : x[j].v[q];
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < SPL; ++q) tile[warp * (NS + 1) + lane * SPL + q] = acc[q];
+    __syncthreads();
+    // 8 consecutive threads write the 8 groups of one sequence (32 contiguous bytes of R)
+    const int gl = tid % GPB;
+    for (int sq = tid / GPB; sq < NS; sq += kSpmmThreads / GPB) {
+        const int b = a.b0 + blockIdx.y * NS + sq;
+        if (b < a.B && gblock + gl < G.M) a.R[(size_t)b * G.M + gblock + gl] = tile[gl * (NS + 1) + sq];
+    }
+}
+
+struct DrawArgs {
+    const void *target;
+    const int32_t *draft_tokens;
+    const float *uniforms;
+    int K;
+    float s;
+    const int32_t *labels;
+    const int32_t *term_n;
+    const int32_t *term_flags;
+    const float4 *term_stats;
+    const float *R;    // default mode: [B, M] residual sums
+    const float *Pws;  // dense mode: [B*(K+1), M] target group masses
+    const float *Qws;  // dense mode: [B*K, M] draft group masses
+    int32_t *out_accept_len;
+    int32_t *out_tokens;
+    int32_t *out_groups;  // may be null
+    int32_t *out_flags;   // may be null
+};
+
+__device__ __forceinline__ int own_slot(int j) { return j + (j >> 5); }  // one pad word per 32: chunked reads spread over banks
+
+// One block per sequence.  Shared memory: the M clamped residual masses (padded), then scratch.
+template <typename T, bool DENSE>
+__global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a, GroupsDev G) {
+    constexpr int NT = kDrawThreads;
+    extern __shared__ __align__(16) unsigned char raw[];
+    const int M = G.M, V = G.V, K = a.K;
+    float *own = reinterpret_cast<float *>(raw);
+    unsigned char *tail = raw + (((size_t)own_slot(M) + 1) * 4 + 15) / 16 * 16;
+    double *dscratch = reinterpret_cast<double *>(tail);      // 32 doubles
+    float *scratch = reinterpret_cast<float *>(dscratch + 32);  // 64 floats
+    int *ibox = reinterpret_cast<int *>(scratch + 64);          // 8 ints
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int n = a.term_n[b];
+    int flags = a.term_flags[b];
+    const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
+    const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
+    const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
+    bool residual = n < K;  // false: draw from the target's coarse distribution itself (bonus token)
+    const float *Pn = DENSE ? a.Pws + ((size_t)b * (K + 1) + n) * M : nullptr;
+    const float *Qn = DENSE ? a.Qws + ((size_t)b * K + min(n, K - 1)) * M : nullptr;
+
+    const int per = (M + NT - 1) / NT;
+    const int i0 = min(M, tid * per), i1 = min(M, i0 + per);
+    double Ztot = 0.0, my_excl = 0.0, my_incl = 0.0, my_sum = 0.0;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        if (DENSE) {
+            for (int g = tid; g < M; g += NT)
+                own[own_slot(g)] = fmaxf(residual ? Pn[g] - Qn[g] : Pn[g], 0.f);  // (P - Q)_+ ; NaN becomes 0
+        } else if (attempt == 0) {
+            // R holds sum_t (p - q)/N for a rejection and sum_t p/N for the bonus row
+            const float *Rb = a.R + (size_t)b * M;
+            for (int g = tid; g < M; g += NT) own[own_slot(g)] = fmaxf(Rb[g], 0.f);
+        } else {
+            // slow path of the zero-residual fallback: the target masses straight from the row
+            const float rs = a.term_stats[b].x;
+            for (int g = tid; g < M; g += NT) {
+                float acc = 0.f;
+                for (int k = G.group_ptr[g]; k < G.group_ptr[g + 1]; ++k) {
+                    const int t = G.group_tok[k];
+                    const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
+                    acc += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs)), w);
+                }
+                own[own_slot(g)] = fmaxf(acc, 0.f);
+            }
+        }
+        __syncthreads();
+        // ---- prefix sums over the groups (double): a contiguous chunk per thread, then a block scan ----
+        my_sum = 0.0;
+        for (int j = i0; j < i1; ++j) my_sum += (double)own[own_slot(j)];
+        block_scan<NT>(my_sum, dscratch, &my_excl, &my_incl, &Ztot);
+        if (Ztot > 0.0 || !residual) break;
+        // a rejection whose residual vanished (P == Q to rounding): draw from P instead
+        flags |= PCG_FLAG_ZERO_RESIDUAL;
+        residual = false;
+        __syncthreads();
+    }
+
+    // ---- group draw: first group whose inclusive prefix exceeds u * Z ----
+    const double target = (double)u_group * Ztot;
+    if (tid == 0) {
+        ibox[2] = NT;  // selected thread (minimum)
+        ibox[3] = -1;  // last group with mass (maximum)
+        ibox[4] = -1;  // drawn group
+    }
+    __syncthreads();
+    int my_last = -1;
+    for (int j = i0; j < i1; ++j)
+        if (own[own_slot(j)] > 0.f) my_last = j;
+    if (my_last >= 0) atomicMax(&ibox[3], my_last);
+    if (my_sum > 0.0 && my_incl > target) atomicMin(&ibox[2], tid);
+    __syncthreads();
+    if (ibox[2] == tid) {
+        double loc = 0.0;
+        int pick = my_last;
+        for (int j = i0; j < i1; ++j) {
+            loc += (double)own[own_slot(j)];
+            if (my_excl + loc > target) {
+                pick = j;
+                break;
+            }
+        }
+        ibox[4] = pick;
+    }
+    __syncthreads();
+    int gsel = ibox[4] >= 0 ? ibox[4] : ibox[3];  // rounding left no prefix above the target: last group with mass
+    int z = 0;
+    if (gsel < 0) {  // no mass anywhere (non-finite inputs): emit group 0 / token 0 and flag it
+        gsel = 0;
+        flags |= PCG_FLAG_NONFINITE;
+    } else {
+        // ---- token inside the drawn group: target-conditional p(t) w / P[g] over the group's CSR order.
+        // Only ratios inside the group matter, so the terms are taken relative to the group's largest logit.
+        const int lo = G.group_ptr[gsel], hi = G.group_ptr[gsel + 1], len = hi - lo;
+        const int per2 = (len + NT - 1) / NT;
+        const int k0 = min(len, tid * per2), k1 = min(len, k0 + per2);
+        float mloc = kNegInf;
+        for (int k = k0; k < k1; ++k) mloc = fmaxf(mloc, Elem<T>::widen(trow[G.group_tok[lo + k]]));
+        const float mg = block_max<NT>(mloc, scratch);
+        const float rs = mg > kNegInf ? mg * a.s : 0.f;
+        auto omega = [&](int k) -> float {
+            const int t = G.group_tok[lo + k];
+            const float w = G.pair_w ? G.pair_w[lo + k] : G.inv_deg[t];
+            return __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs)), w);
+        };
+        double wsum = 0.0;
+        int wlast = -1;
+        for (int k = k0; k < k1; ++k) {
+            const float w = omega(k);
+            wsum += (double)w;
+            if (w > 0.f) wlast = k;
+        }
+        double excl, incl, wtot;
+        block_scan<NT>(wsum, dscratch, &excl, &incl, &wtot);
+        if (tid == 0) {
+            ibox[2] = NT;
+            ibox[3] = -1;
+            ibox[4] = -1;
+        }
+        __syncthreads();
+        const double target2 = (double)u_token * wtot;
+        if (wlast >= 0) atomicMax(&ibox[3], wlast);
+        if (wsum > 0.0 && incl > target2) atomicMin(&ibox[2], tid);
+        __syncthreads();
+        if (ibox[2] == tid) {
+            double loc = 0.0;
+            int pick = wlast;
+            for (int k = k0; k < k1; ++k) {
+                loc += (double)omega(k);
+                if (excl + loc > target2) {
+                    pick = k;
+                    break;
+                }
+            }
+            ibox[4] = pick;
+        }
+        __syncthreads();
+        const int ksel = ibox[4] >= 0 ? ibox[4] : ibox[3];
+        if (ksel >= 0) {
+            z = G.group_tok[lo + ksel];
+        } else {  // the drawn group has no token with target mass (non-finite inputs)
+            z = len > 0 ? G.group_tok[lo] : 0;
+            flags |= PCG_FLAG_NONFINITE;
+        }
+    }
+    // ---- emit: accepted draft tokens, the drawn token, then filler ----
+    if (tid <= K) {
+        int tok = -1, grp = -1;
+        if (tid < n) {
+            tok = a.draft_tokens[b * K + tid];
+            if (tok < 0 || tok >= V) tok = 0;  // verified as token 0 (and flagged), so emitted as token 0
+            grp = a.labels[b * K + tid];
+        } else if (tid == n) {
+            tok = z;
+            grp = gsel;
+        }
+        a.out_tokens[(int64_t)b * (K + 1) + tid] = tok;
+        if (a.out_groups) a.out_groups[(int64_t)b * (K + 1) + tid] = grp;
+    }
+    if (tid == 0) {
+        a.out_accept_len[b] = n;
+        if (a.out_flags) a.out_flags[b] = flags;
+    }
+}
+
+// ---------------------------------------------------------------- dense mode: accept test from full P, Q -----
+struct DenseAcceptArgs {
+    const int32_t *draft_tokens;
+    const float *uniforms;
+    int B, K;
+    const float *Pws;  // [B*(K+1), M]
+    const float *Qws;  // [B*K, M]
+    int32_t *accept, *labels, *posflags;
+};
+
+// One thread per drafted position: label draw, then u < min(1, P[g]/Q[g]) on the stored group masses.
+__global__ void dense_accept_kernel(DenseAcceptArgs a, GroupsDev G) {
+    const int pos = blockIdx.x * blockDim.x + threadIdx.x;
+    if (pos >= a.B * a.K) return;
+    const int b = pos / a.K, i = pos - b * a.K;
+    int x = a.draft_tokens[pos], flag = 0;
+    if (x < 0 || x >= G.V) {
+        x = 0;
+        flag = PCG_FLAG_BAD_DRAFT_TOKEN;
+    }
+    const float *u = a.uniforms + ((int64_t)b * (a.K + 1) + i) * 2;
+    const int r0 = G.rev_ptr[x];
+    const int g = draw_label(G, r0, G.rev_ptr[x + 1] - r0, u[0]);
+    const float P = a.Pws[((size_t)b * (a.K + 1) + i) * G.M + g], Q = a.Qws[(size_t)pos * G.M + g];
+    if (isnan(P) || isnan(Q)) flag |= PCG_FLAG_NONFINITE;
+    a.accept[pos] = (P >= Q) || (u[1] * Q < P);
+    a.labels[pos] = g;
+    a.posflags[pos] = flag;
+}
+
 // ================================================================ host side ================================
 
 static pcg_status check_common(const pcg_groups *groups, pcg_dtype dtype, float temperature, const char *who) {
@@ -723,14 +1267,33 @@ static cudaError_t launch_cluster(Kern kern, int blocks, int cluster, size_t sme
     return cudaLaunchKernelEx(&cfg, kern, args, G);
 }
 
+#ifndef PCG_DT_BUDGET_MB
+#define PCG_DT_BUDGET_MB 64
+#endif
+constexpr size_t kDtBudgetBytes = (size_t)PCG_DT_BUDGET_MB << 20;  // Dt of one chunk of sequences must stay inside the L2
+
+// Sequences per chunk of the batched terminal stage: a multiple of 32 * kSpmmWide (one warp of the sparse
+// product covers that many sequences with vector loads) once the batch has that many, of 32 below that.
+static int terminal_chunk(int B, int V) {
+    const int64_t unit = B >= 32 * kSpmmWide ? 32 * kSpmmWide : 32;
+    const int64_t bpad = ((int64_t)B + unit - 1) / unit * unit;
+    int64_t fit = (int64_t)(kDtBudgetBytes / ((size_t)V * 4)) / unit * unit;
+    if (fit < unit) fit = unit;
+    return (int)(fit < bpad ? fit : bpad);
+}
+
+static size_t draw_smem_bytes(int M) { return (((size_t)M + (size_t)(M >> 5) + 1) * 4 + 15) / 16 * 16 + 32 * 8 + 64 * 4 + 8 * 4; }
+
 struct VerifyWorkspace {
-    int32_t *accept, *labels, *posflags;
-    float4 *stats;
+    int32_t *accept, *labels, *posflags, *term_n, *term_flags;
+    float4 *stats, *term_stats;
+    float *Dt, *R;     // default mode
+    float *Pws, *Qws;  // dense mode
     size_t bytes;
 };
 
-static VerifyWorkspace carve_workspace(void *base, int64_t positions) {
-    VerifyWorkspace w;
+static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t V, int64_t M, uint32_t mode) {
+    VerifyWorkspace w = {};
     size_t off = 0;
     auto take = [&](size_t bytes) {
         size_t at = off;
@@ -738,10 +1301,21 @@ static VerifyWorkspace carve_workspace(void *base, int64_t positions) {
         return at;
     };
     char *p = (char *)base;
+    const int64_t positions = B * K;
     w.stats = (float4 *)(p + take((size_t)positions * 16));
     w.accept = (int32_t *)(p + take((size_t)positions * 4));
     w.labels = (int32_t *)(p + take((size_t)positions * 4));
     w.posflags = (int32_t *)(p + take((size_t)positions * 4));
+    w.term_stats = (float4 *)(p + take((size_t)B * 16));
+    w.term_n = (int32_t *)(p + take((size_t)B * 4));
+    w.term_flags = (int32_t *)(p + take((size_t)B * 4));
+    if (mode & PCG_VERIFY_DENSE) {
+        w.Pws = (float *)(p + take((size_t)(B * (K + 1) * M) * 4));
+        w.Qws = (float *)(p + take((size_t)(B * K * M) * 4));
+    } else if (!(mode & PCG_VERIFY_CLUSTER_TERMINAL)) {
+        w.Dt = (float *)(p + take((size_t)V * (size_t)terminal_chunk((int)B, (int)V) * 4));
+        w.R = (float *)(p + take((size_t)(B * M) * 4));
+    }
     w.bytes = off ? off : 256;
     return w;
 }
@@ -778,12 +1352,9 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
 
 extern "C" size_t pcg_verify_workspace_bytes(int32_t B, int32_t K, int32_t V, int32_t M, pcg_dtype dtype,
                                              uint32_t mode) {
-    (void)V;
-    (void)M;
     (void)dtype;
-    (void)mode;
-    if (B < 0 || K < 0) return 256;
-    return carve_workspace(nullptr, (int64_t)B * K).bytes;
+    if (B < 0 || K < 0 || V < 1 || M < 1) return 256;
+    return carve_workspace(nullptr, B, K, V, M, mode).bytes;
 }
 
 extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_logits, pcg_dtype dtype, int32_t B,
@@ -802,8 +1373,9 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         set_error("pcg_verify: K=%d exceeds the 32 positions one ballot covers", K);
         return PCG_ERR_UNSUPPORTED;
     }
-    if (mode & ~PCG_VERIFY_DENSE) {
-        set_error("pcg_verify: unknown mode bits 0x%x", mode);
+    if ((mode & ~(PCG_VERIFY_DENSE | PCG_VERIFY_CLUSTER_TERMINAL)) ||
+        mode == (PCG_VERIFY_DENSE | PCG_VERIFY_CLUSTER_TERMINAL)) {
+        set_error("pcg_verify: unknown or contradictory mode bits 0x%x", mode);
         return PCG_ERR_INVALID_ARG;
     }
     if (B == 0) return PCG_OK;
@@ -817,7 +1389,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         set_error("pcg_verify: logits pointers must be aligned to their element size");
         return PCG_ERR_INVALID_ARG;
     }
-    if ((int64_t)B * K > INT32_MAX / 8) {
+    if ((int64_t)B * (K + 1) > INT32_MAX / 8) {
         set_error("pcg_verify: B*K too large for one launch");
         return PCG_ERR_UNSUPPORTED;
     }
@@ -827,36 +1399,103 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
                   workspace_bytes);
         return PCG_ERR_WORKSPACE;
     }
-    if (mode & PCG_VERIFY_DENSE) {
-        set_error("pcg_verify: dense mode is not built yet");
+    const bool dense = mode & PCG_VERIFY_DENSE, cluster_terminal = mode & PCG_VERIFY_CLUSTER_TERMINAL;
+    const size_t draw_smem = draw_smem_bytes(G.M);
+    if (!cluster_terminal && draw_smem > kMaxDynSmem) {
+        set_error("pcg_verify: M=%d needs %zu bytes of shared memory in the terminal draw (limit %zu)", G.M, draw_smem,
+                  kMaxDynSmem);
         return PCG_ERR_UNSUPPORTED;
     }
     cudaStream_t cs = (cudaStream_t)stream;
-    const VerifyWorkspace w = carve_workspace(workspace, (int64_t)B * K);
+    const VerifyWorkspace w = carve_workspace(workspace, B, K, G.V, G.M, mode);
     const float s = (float)((double)kLog2e / (double)temperature);
     cudaError_t e = cudaSuccess;
     if (stage_events) e = cudaEventRecord((cudaEvent_t)stage_events[0], cs);
     if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
 
-    PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, w.accept, w.labels, w.posflags, w.stats};
-    if (dtype == PCG_F32)
-        position_kernel<float><<<B * K, kPosThreads, 0, cs>>>(pa, G);
-    else
-        position_kernel<uint16_t><<<B * K, kPosThreads, 0, cs>>>(pa, G);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
+    // ---- per-position stage: statistics, label, accept bit ----
+    if (dense) {
+        // P and Q of ALL groups at EVERY position, then the accept test on the stored masses
+        pcg_status st2 = pcg_group_probs(target_logits, dtype, (int64_t)B * (K + 1), temperature, groups, w.Pws, stream);
+        if (st2 == PCG_OK) st2 = pcg_group_probs(draft_logits, dtype, (int64_t)B * K, temperature, groups, w.Qws, stream);
+        if (st2 != PCG_OK) return st2;
+        DenseAcceptArgs da{draft_tokens, uniforms, B, K, w.Pws, w.Qws, w.accept, w.labels, w.posflags};
+        dense_accept_kernel<<<(B * K + 127) / 128, 128, 0, cs>>>(da, G);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e, "launching dense_accept_kernel");
+    } else {
+        PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, w.accept, w.labels, w.posflags, w.stats};
+        if (dtype == PCG_F32)
+            position_kernel<float><<<B * K, kPosThreads, 0, cs>>>(pa, G);
+        else
+            position_kernel<uint16_t><<<B * K, kPosThreads, 0, cs>>>(pa, G);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
+    }
     if (stage_events) {
         e = cudaEventRecord((cudaEvent_t)stage_events[1], cs);
         if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
     }
 
-    TerminalArgs ta{target_logits, draft_logits, draft_tokens, uniforms,       K,          s,         w.accept,
-                    w.labels,      w.posflags,   w.stats,      out_accept_len, out_tokens, out_groups, out_flags};
-    if (dtype == PCG_F32)
-        e = launch_cluster(terminal_kernel<float>, B * G.slices, G.slices, groups->agg_smem_bytes, cs, ta, G);
-    else
-        e = launch_cluster(terminal_kernel<uint16_t>, B * G.slices, G.slices, groups->agg_smem_bytes, cs, ta, G);
-    if (e != cudaSuccess) return cuda_fail(e, "launching terminal_kernel");
+    // ---- per-sequence stage: first rejection, residual over all groups, group and token draw ----
+    if (cluster_terminal) {
+        TerminalArgs ta{target_logits, draft_logits, draft_tokens, uniforms,       K,          s,         w.accept,
+                        w.labels,      w.posflags,   w.stats,      out_accept_len, out_tokens, out_groups, out_flags};
+        if (dtype == PCG_F32)
+            e = launch_cluster(terminal_kernel<float>, B * G.slices, G.slices, groups->agg_smem_bytes, cs, ta, G);
+        else
+            e = launch_cluster(terminal_kernel<uint16_t>, B * G.slices, G.slices, groups->agg_smem_bytes, cs, ta, G);
+        if (e != cudaSuccess) return cuda_fail(e, "launching terminal_kernel");
+    } else {
+        PrepareArgs pr{target_logits, K, s, dense ? 0 : 1, w.accept, w.posflags, w.stats, w.term_n, w.term_flags, w.term_stats};
+        if (dtype == PCG_F32)
+            terminal_prepare_kernel<float><<<B, kPrepThreads, 0, cs>>>(pr, G);
+        else
+            terminal_prepare_kernel<uint16_t><<<B, kPrepThreads, 0, cs>>>(pr, G);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e, "launching terminal_prepare_kernel");
+        if (!dense) {
+            const int chunk = terminal_chunk(B, G.V);
+            const int tt = 32 * (dtype == PCG_F32 ? 4 : 8);
+            const bool wide = B >= 32 * kSpmmWide;  // several sequences per lane in the sparse product
+            for (int b0 = 0; b0 < B; b0 += chunk) {
+                // blocks of 32 sequences in this chunk, rounded up to what one block of the sparse product reads
+                const int unit = wide ? 32 * kSpmmWide : 32;
+                const int nb = (std::min(B - b0, chunk) + unit - 1) / unit * (unit / 32);
+                TransposeArgs tr{target_logits, draft_logits, B, K, b0, chunk, s, w.term_n, w.term_stats, w.Dt};
+                const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
+                if (dtype == PCG_F32)
+                    residual_transpose_kernel<float><<<tgrid, kTrThreads, 0, cs>>>(tr, G);
+                else
+                    residual_transpose_kernel<uint16_t><<<tgrid, kTrThreads, 0, cs>>>(tr, G);
+                e = cudaGetLastError();
+                if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
+                SpmmArgs sp{w.Dt, B, b0, chunk, w.R};
+                const unsigned gx = (unsigned)((G.M + kSpmmThreads / 32 - 1) / (kSpmmThreads / 32));
+                if (wide)
+                    group_spmm_kernel<kSpmmWide, kSpmmDepth>
+                        <<<dim3(gx, (unsigned)(nb / kSpmmWide)), kSpmmThreads, 0, cs>>>(sp, G);
+                else
+                    group_spmm_kernel<1, 16><<<dim3(gx, (unsigned)nb), kSpmmThreads, 0, cs>>>(sp, G);
+                e = cudaGetLastError();
+                if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
+            }
+        }
+        DrawArgs dr{target_logits, draft_tokens, uniforms, K,     s,     w.labels,       w.term_n,   w.term_flags,
+                    w.term_stats,  w.R,          w.Pws,    w.Qws, out_accept_len, out_tokens, out_groups, out_flags};
+        auto launch_draw = [&](auto kern) -> cudaError_t {
+            cudaError_t le = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)draw_smem);
+            if (le != cudaSuccess) return le;
+            kern<<<B, kDrawThreads, draw_smem, cs>>>(dr, G);
+            return cudaGetLastError();
+        };
+        if (dtype == PCG_F32)
+            e = dense ? launch_draw(terminal_draw_kernel<float, true>) : launch_draw(terminal_draw_kernel<float, false>);
+        else
+            e = dense ? launch_draw(terminal_draw_kernel<uint16_t, true>)
+                      : launch_draw(terminal_draw_kernel<uint16_t, false>);
+        if (e != cudaSuccess) return cuda_fail(e, "launching terminal_draw_kernel");
+    }
     if (stage_events) {
         e = cudaEventRecord((cudaEvent_t)stage_events[2], cs);
         if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");

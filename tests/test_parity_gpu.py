@@ -15,6 +15,9 @@ from oracle.compare import compare_verify  # noqa: E402
 from gpu_util import logits_to_device, make_handle, run_oracle, run_verify  # noqa: E402
 
 BAND = 1e-6
+# pcg_verify modes: default (label group per position, batched per-sequence stage), dense (P and Q of all groups at
+# every position), cluster terminal (default per-position stage, one thread-block cluster per sequence afterwards)
+MODES = [pytest.param(0, id="default"), pytest.param(1, id="dense"), pytest.param(2, id="cluster")]
 
 
 def _assert_parity(got, ref, max_excused=0):
@@ -60,58 +63,108 @@ def test_group_probs_any_slicing(oracle, hint):
 
 
 # ------------------------------------------------------------------------ pcg_verify ----
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4"])
-def test_verify_matches_oracle_on_configs(oracle, name):
+def test_verify_matches_oracle_on_configs(oracle, name, mode):
     cfg = W.CONFIGS[name]
     groups = W.make_groups(cfg)
     bt = W.make_batch(cfg)
     ref = run_oracle(oracle, bt, groups)
-    got = run_verify(bt, make_handle(groups))
+    got = run_verify(bt, make_handle(groups), mode=mode)
     _assert_parity(got, ref)
     assert np.all(got[3] == 0)
 
 
-def test_verify_c5_shape_small_batch(oracle):
+@pytest.mark.parametrize("mode", MODES)
+def test_verify_c5_shape_small_batch(oracle, mode):
     cfg = W.CONFIGS["C5"]
     groups = W.make_groups(cfg)
     bt = W.make_batch(cfg, B=12)
     ref = run_oracle(oracle, bt, groups)
     h = make_handle(groups)
     assert h.info.slices == 8
-    _assert_parity(run_verify(bt, h), ref)
+    _assert_parity(run_verify(bt, h, mode=mode), ref)
 
 
+def test_verify_batch_spanning_several_sequence_blocks(oracle):
+    """The batched per-sequence stage handles 32 sequences per line: 70 sequences = two full blocks and a ragged one,
+    with a group count that is not a multiple of the 32 groups a block of the sparse product owns."""
+    cfg = W.scaled(W.CONFIGS["C3"], B=70, V=3000, M=1001, K=3)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    bt.draft_logits[::3] = bt.target_logits[::3, :cfg.K]  # every third sequence accepts everything: bonus rows
+    ref = run_oracle(oracle, bt, groups)
+    assert np.any(ref.accept_len == cfg.K) and np.any(ref.accept_len == 0)
+    h = make_handle(groups)
+    for mode in (0, 1, 2):
+        _assert_parity(run_verify(bt, h, mode=mode), ref)
+
+
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("hint", [1, 2, 4, 8])
-def test_verify_any_slicing(oracle, hint):
+def test_verify_any_slicing(oracle, hint, mode):
     cfg = W.scaled(W.CONFIGS["C3"], B=24, V=5000, M=1200, K=5)
     groups = W.make_groups(cfg)
     bt = W.make_batch(cfg)
     ref = run_oracle(oracle, bt, groups)
-    _assert_parity(run_verify(bt, make_handle(groups, slices_hint=hint)), ref)
+    _assert_parity(run_verify(bt, make_handle(groups, slices_hint=hint), mode=mode), ref)
 
 
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("V,dtype", [(1003, "f32"), (1003, "bf16"), (77, "bf16"), (4096 + 8, "bf16"), (5, "f32")])
-def test_verify_ragged_and_misaligned_rows(oracle, V, dtype):
+def test_verify_ragged_and_misaligned_rows(oracle, V, dtype, mode):
     """V not a multiple of the vector width: rows start at unaligned addresses and have scalar heads and tails."""
     cfg = W.scaled(W.CONFIGS["C1"], B=10, K=3, V=V, M=max(2, V // 6), emb_dim=8, dtype=dtype,
                    degree=min(3, max(2, V // 6)))
     groups = W.make_groups(cfg)
     bt = W.make_batch(cfg)
     ref = run_oracle(oracle, bt, groups)
-    _assert_parity(run_verify(bt, make_handle(groups)), ref)
+    _assert_parity(run_verify(bt, make_handle(groups), mode=mode), ref)
 
 
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("K", [1, 32])
-def test_verify_extreme_k(oracle, K):
+def test_verify_extreme_k(oracle, K, mode):
     cfg = W.scaled(W.CONFIGS["C1"], B=6, K=K, V=512, M=100, emb_dim=8)
     groups = W.make_groups(cfg)
     bt = W.make_batch(cfg)
     bt.draft_logits[:] = bt.target_logits[:, :K] + 0.05 * (bt.draft_logits - bt.target_logits[:, :K])  # long accepts
     ref = run_oracle(oracle, bt, groups)
-    got = run_verify(bt, make_handle(groups))
+    got = run_verify(bt, make_handle(groups), mode=mode)
     _assert_parity(got, ref)
     if K == 32:
         assert ref.accept_len.max() > 8
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_verify_general_split_weights(oracle, dtype, mode):
+    """General weights w_{k,t} (non-negative, summing to one over the groups of each token) in place of the equal
+    split: the reduction, the label draw and the within-group draw all use them."""
+    rng = np.random.default_rng(11)
+    cfg = W.scaled(W.CONFIGS["C4"], B=20, K=4, V=3000, M=500, dtype=dtype)
+    groups = W.make_groups(cfg)
+    raw = rng.random(groups.nnz) + 0.05
+    raw[rng.random(groups.nnz) < 0.1] = 0.0  # some memberships carry no mass at all
+    tot = np.zeros(cfg.V)
+    np.add.at(tot, groups.group_tok, raw)
+    dead = tot[groups.group_tok] == 0
+    raw[dead] = 1.0
+    tot = np.zeros(cfg.V)
+    np.add.at(tot, groups.group_tok, raw)
+    w = (raw / tot[groups.group_tok]).astype(np.float32)
+    bt = W.make_batch(cfg)
+    ref = run_oracle(oracle, bt, groups, weights=w.astype(np.float64))
+    got = run_verify(bt, make_handle(groups, weights=w), mode=mode)
+    _assert_parity(got, ref)
+    if mode == 0:
+        from paper_2511_13732_b200 import binding
+
+        x = bt.target_logits.reshape(-1, cfg.V)[:7]
+        want = oracle.group_probs(x, groups.group_ptr, groups.group_tok, groups.tok_degree, cfg.temperature,
+                                  weights=w.astype(np.float64))
+        P = binding.pcg_group_probs(logits_to_device(x), make_handle(groups, weights=w), cfg.temperature)
+        np.testing.assert_allclose(P.cpu().numpy(), want, rtol=1e-5, atol=1e-37)
 
 
 def _special_groups(kind, V, rng):
@@ -148,8 +201,8 @@ def test_verify_degenerate_memberships(oracle, kind, dtype):
     u = (rng.integers(0, 1 << 24, (B, K + 1, 2)) * 2.0 ** -24).astype(np.float32)
     bt = W.Batch(tl, dl, x, u, 0.9, dtype)
     ref = run_oracle(oracle, bt, groups)
-    for hint in (0, 4):
-        got = run_verify(bt, make_handle(groups, slices_hint=hint))
+    for hint, mode in ((0, 0), (0, 1), (0, 2), (4, 1), (4, 2)):
+        got = run_verify(bt, make_handle(groups, slices_hint=hint), mode=mode)
         _assert_parity(got, ref)
     if kind == "one_giant":
         assert np.all(ref.accept_len == K)  # a single group is always accepted: P = Q = 1
@@ -165,7 +218,8 @@ def test_verify_all_accept_all_reject_and_masked_logits(oracle):
     ref = run_oracle(oracle, same, groups)
     assert np.all(ref.accept_len == cfg.K)
     h = make_handle(groups)
-    _assert_parity(run_verify(same, h), ref)
+    for mode in (0, 1, 2):
+        _assert_parity(run_verify(same, h, mode=mode), ref)
     # draft token forced onto a token the target gives no mass (-inf): rejected at position 0
     tl, dl = bt.target_logits.copy(), bt.draft_logits.copy()
     for b in range(cfg.B):
@@ -178,14 +232,17 @@ def test_verify_all_accept_all_reject_and_masked_logits(oracle):
     masked = W.Batch(tl, dl, bt.draft_tokens, bt.uniforms, 1.0, "f32")
     ref = run_oracle(oracle, masked, groups)
     assert np.all(ref.accept_len == 0)
-    got = run_verify(masked, h)
-    _assert_parity(got, ref)
-    assert np.all(got[3] == 0)  # -inf logits are legitimate masks, not an error
+    for mode in (0, 1, 2):
+        got = run_verify(masked, h, mode=mode)
+        _assert_parity(got, ref)
+        assert np.all(got[3] == 0)  # -inf logits are legitimate masks, not an error
     # one dominant logit per row
     tl2 = bt.target_logits.copy()
     tl2[:, :, 17] += 60.0
     dom = W.Batch(tl2, bt.draft_logits, bt.draft_tokens, bt.uniforms, 1.0, "f32")
-    _assert_parity(run_verify(dom, h), run_oracle(oracle, dom, groups))
+    ref = run_oracle(oracle, dom, groups)
+    for mode in (0, 1, 2):
+        _assert_parity(run_verify(dom, h, mode=mode), ref)
 
 
 def test_verify_is_bit_reproducible_and_flags_bad_tokens(oracle):
@@ -248,14 +305,15 @@ def test_device_side_argument_errors(oracle):
     assert binding.pcg_group_probs(tl.reshape(-1, cfg.V)[:0], h).shape == (0, groups.M)
 
 
-def test_full_size_bench_configuration_on_sampled_sequences(oracle):
+@pytest.mark.parametrize("mode", [pytest.param(0, id="default"), pytest.param(1, id="dense")])
+def test_full_size_bench_configuration_on_sampled_sequences(oracle, mode):
     """C5 exactly as bench.py launches it (B=256, K=16, V=65536, bf16): every sequence is checked for structure,
     and a sample of sequences is checked decision by decision against the oracle."""
     cfg = W.CONFIGS["C5"]
     groups = W.make_groups(cfg)
     bt = W.make_batch(cfg)
     h = make_handle(groups)
-    n, tok, grp, flg = run_verify(bt, h)
+    n, tok, grp, flg = run_verify(bt, h, mode=mode)
     assert np.all(flg == 0) and np.all((n >= 0) & (n <= cfg.K))
     for b in range(cfg.B):
         assert np.array_equal(tok[b, :n[b]], bt.draft_tokens[b, :n[b]])
