@@ -200,6 +200,34 @@ pcg_status pcg_verify_host(const void *target_logits, const void *draft_logits, 
                            int32_t *out_flags, void *device_arena, size_t device_arena_bytes, uint32_t mode,
                            pcg_stream stream);
 
+/*
+ * pcg_verify for callers that have no workspace to give.  (The paper has no counterpart to this entry point;
+ * it exists for the library's users only.)
+ *
+ * Who needs it: code that runs after its host application has handed out all device memory and forbids
+ * further allocation -- an inference server whose memory pool was carved up at start-up, a plug-in running
+ * inside someone else's process, a latency-critical loop that must never meet cudaMalloc (which may stall the
+ * whole device, or fail once the pool owns all memory).  Such a caller cannot size and allocate the workspace
+ * pcg_verify asks for, so this variant keeps its scratch in an array that is part of the library image: 1 MiB
+ * of device memory on every GPU that loads libpcg.so, held until the process exits.  The call allocates and
+ * frees nothing, on the host side of CUDA or through any library.
+ *
+ * Same arguments, results and errors as pcg_verify in PCG_VERIFY_CLUSTER_TERMINAL mode, without workspace,
+ * mode and stage events.  Limits: the per-position bookkeeping of the call must fit the array -- 28 bytes per
+ * drafted position plus 24 per sequence (each array rounded up to 256 bytes), i.e. roughly B*K <= 35,000; larger calls return
+ * PCG_ERR_UNSUPPORTED with a message that says so, before anything is launched.
+ *
+ * The first call on each device looks up the array's device address (with that device current) and remembers
+ * it; make that first call outside any stream capture.  All calls on one device share the one array, which
+ * keeps whatever the previous call left in it (nothing in it needs clearing: every field is written before it
+ * is read within a call).  Two calls whose kernels can overlap on the same GPU -- different streams, or different
+ * host threads -- race on it: serialise them, or use pcg_verify with separate workspaces.
+ */
+pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits, pcg_dtype dtype, int32_t B, int32_t K,
+                             const int32_t *draft_tokens, const pcg_groups *groups, const float *uniforms,
+                             float temperature, int32_t *out_accept_len, int32_t *out_tokens, int32_t *out_groups,
+                             int32_t *out_flags, pcg_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,6 +25,7 @@ STATUS_NAMES = {0: "PCG_OK", 1: "PCG_ERR_INVALID_ARG", 2: "PCG_ERR_INVALID_GROUP
 EXPORTS = [
     "pcg_status_string", "pcg_last_error", "pcg_groups_create", "pcg_groups_destroy", "pcg_groups_info",
     "pcg_group_probs", "pcg_verify_workspace_bytes", "pcg_verify", "pcg_verify_host_arena_bytes", "pcg_verify_host",
+    "pcg_verify_static",
 ]
 
 
@@ -84,6 +85,8 @@ def load(build_if_missing: bool = True):
     lib.pcg_verify_host_arena_bytes.restype = sz
     lib.pcg_verify_host.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, f32, vp, vp, vp, vp, vp, sz, u32, vp]
     lib.pcg_verify_host.restype = ctypes.c_int
+    lib.pcg_verify_static.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, f32, vp, vp, vp, vp, vp]
+    lib.pcg_verify_static.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -223,4 +226,17 @@ def pcg_verify_host(target_logits, draft_logits, draft_tokens, groups: Groups, u
                                   _dev_ptr(draft_tokens), groups.handle, _dev_ptr(uniforms), float(temperature),
                                   _dev_ptr(accept_len), _dev_ptr(tokens), _dev_ptr(grp), _dev_ptr(flags),
                                   _dev_ptr(arena), arena.numel() * arena.element_size(), mode, _stream_ptr(stream)))
+    return out
+
+
+def pcg_verify_static(target_logits, draft_logits, draft_tokens, groups: Groups, uniforms, temperature: float,
+                      out, stream=None):
+    """``pcg_verify_static``: verification with the library's built-in scratch.  Every tensor, the four outputs
+    in ``out`` included (groups and flags may be None), is supplied by the caller; nothing is allocated here."""
+    B, K1, V = target_logits.shape
+    accept_len, tokens, grp, flags = out
+    _check(load().pcg_verify_static(_dev_ptr(target_logits), _dev_ptr(draft_logits), dtype_code(target_logits), B,
+                                    K1 - 1, _dev_ptr(draft_tokens), groups.handle, _dev_ptr(uniforms),
+                                    float(temperature), _dev_ptr(accept_len), _dev_ptr(tokens), _dev_ptr(grp),
+                                    _dev_ptr(flags), _stream_ptr(stream)))
     return out

@@ -15,10 +15,15 @@
 
 #include <algorithm>
 #include <cmath>
+#include <mutex>
 
 #include "pcg_common.cuh"
 
 namespace cg = cooperative_groups;
+
+#ifndef PCG_STATIC_SCRATCH_BYTES
+#define PCG_STATIC_SCRATCH_BYTES (1u << 20)  // built-in scratch of pcg_verify_static, per GPU
+#endif
 
 namespace pcg {
 
@@ -1501,4 +1506,63 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
     }
     return PCG_OK;
+}
+
+// ================================================================ verification without caller scratch ======
+//
+// Built-in scratch of pcg_verify_static: one array per GPU that loads the library, held until the process
+// exits.  In host code `g_static_scratch` is only a stand-in for the symbol, never a device address; the
+// address a kernel may use comes from cudaGetSymbolAddress, asked once per device and remembered here.
+namespace pcg {
+constexpr size_t kStaticScratchBytes = PCG_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+constexpr int kMaxStaticDevices = 64;
+static void *g_static_scratch_addr[kMaxStaticDevices];  // zero-initialised; written once per device
+static std::mutex g_static_scratch_mutex;
+}  // namespace pcg
+
+extern "C" pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits, pcg_dtype dtype,
+                                        int32_t B, int32_t K, const int32_t *draft_tokens, const pcg_groups *groups,
+                                        const float *uniforms, float temperature, int32_t *out_accept_len,
+                                        int32_t *out_tokens, int32_t *out_groups, int32_t *out_flags,
+                                        pcg_stream stream) {
+    if (!groups) {
+        set_error("pcg_verify_static: null group handle");
+        return PCG_ERR_INVALID_ARG;
+    }
+    if (B < 0 || K < 1) {
+        set_error("pcg_verify_static: need B >= 0 and K >= 1 (B=%d K=%d)", B, K);
+        return PCG_ERR_INVALID_ARG;
+    }
+    const uint32_t mode = PCG_VERIFY_CLUSTER_TERMINAL;  // the mode whose scratch is a few bytes per position
+    const size_t need = pcg_verify_workspace_bytes(B, K, groups->dev.V, groups->dev.M, dtype, mode);
+    if (need > kStaticScratchBytes) {
+        set_error("pcg_verify_static: B=%d, K=%d need %zu bytes of scratch but the built-in array holds %zu "
+                  "(about %zu positions); use pcg_verify with a workspace of your own",
+                  B, K, need, kStaticScratchBytes, kStaticScratchBytes / 29);
+        return PCG_ERR_UNSUPPORTED;
+    }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= kMaxStaticDevices) {
+        set_error("pcg_verify_static: device ordinal %d is beyond the %d devices the address table covers", dev,
+                  kMaxStaticDevices);
+        return PCG_ERR_UNSUPPORTED;
+    }
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+        if (!g_static_scratch_addr[dev]) {  // first call on this device: resolve the symbol with it current
+            void *addr = nullptr;
+            e = cudaGetSymbolAddress(&addr, g_static_scratch);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress (built-in scratch)");
+            g_static_scratch_addr[dev] = addr;
+        }
+        scratch = g_static_scratch_addr[dev];
+    }
+    // Nothing in the scratch has to start at zero: every field a kernel reads is written earlier in the same call.
+    return pcg_verify(target_logits, draft_logits, dtype, B, K, draft_tokens, groups, uniforms, temperature,
+                      out_accept_len, out_tokens, out_groups, out_flags, scratch, kStaticScratchBytes, mode, stream,
+                      nullptr);
 }
