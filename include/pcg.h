@@ -53,12 +53,17 @@ typedef struct CUevent_st *pcg_event;
 
 /* Bits of the `mode` argument of pcg_verify. */
 #define PCG_VERIFY_DEFAULT 0u /* per position only the label group's P and Q are formed (what the accept test
-                                 needs); all groups are aggregated once per sequence, at its terminal position */
+                                 needs); all groups are aggregated once per sequence, at its terminal position.
+                                 The per-sequence stage runs as CLUSTER_TERMINAL for a handful of sequences
+                                 (B * slices <= 2 * SM count) and as BATCHED_TERMINAL beyond that */
 #define PCG_VERIFY_DENSE 1u   /* form P and Q of ALL groups at EVERY position (stored in the workspace), then take
                                  the same decisions from the stored vectors */
-#define PCG_VERIFY_CLUSTER_TERMINAL 2u /* default mode, but the per-sequence stage runs as one thread-block cluster
-                                 per sequence instead of the batched transpose / sparse-product / draw kernels
-                                 (lower latency for a handful of sequences); not combinable with DENSE */
+#define PCG_VERIFY_CLUSTER_TERMINAL 2u /* default per-position stage; per-sequence stage as one thread-block
+                                 cluster per sequence (shared-memory aggregation; lowest latency for small batches) */
+#define PCG_VERIFY_BATCHED_TERMINAL 4u /* default per-position stage; per-sequence stage as the batched kernels
+                                 (transposed residual, sparse product over L2, draw; best throughput for large
+                                 batches) */
+/* The modes are alternatives, not flags to combine; all four take the same decisions. */
 
 /*
  * Group membership: the Acoustic Similarity Groups as a group->token CSR plus

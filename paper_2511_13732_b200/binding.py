@@ -18,7 +18,7 @@ from . import build as _build
 
 PCG_F32, PCG_BF16 = 0, 1
 FLAG_BAD_DRAFT_TOKEN, FLAG_ZERO_RESIDUAL, FLAG_NONFINITE = 1, 2, 4
-VERIFY_DEFAULT, VERIFY_DENSE, VERIFY_CLUSTER_TERMINAL = 0, 1, 2
+VERIFY_DEFAULT, VERIFY_DENSE, VERIFY_CLUSTER_TERMINAL, VERIFY_BATCHED_TERMINAL = 0, 1, 2, 4
 STATUS_NAMES = {0: "PCG_OK", 1: "PCG_ERR_INVALID_ARG", 2: "PCG_ERR_INVALID_GROUPS", 3: "PCG_ERR_UNSUPPORTED",
                 4: "PCG_ERR_WORKSPACE", 5: "PCG_ERR_CUDA"}
 

@@ -705,13 +705,20 @@ __global__ void __launch_bounds__(kAggThreads, 2) terminal_kernel(TerminalArgs a
 
 constexpr int kPrepThreads = 256;  // terminal_prepare_kernel
 constexpr int kTrThreads = 256;    // residual_transpose_kernel
-constexpr int kSpmmThreads = 256;  // group_spmm_kernel: 8 warps, one group each
+#ifndef PCG_SPMM_THREADS
+#define PCG_SPMM_THREADS 128
+#endif
+constexpr int kSpmmThreads = PCG_SPMM_THREADS;  // group_spmm_kernel: warps of 8 groups each
 #ifndef PCG_SPMM_SPL
 #define PCG_SPMM_SPL 4    // sequences per lane of the sparse product for batches of at least 32 * PCG_SPMM_SPL
 #endif
 #ifndef PCG_SPMM_DEPTH
-#define PCG_SPMM_DEPTH 8  // loads of Dt in flight per lane
+#define PCG_SPMM_DEPTH 8  // tokens per batch of the sparse product; two batches of loads are in flight per lane
 #endif
+#ifndef PCG_SPMM_GW
+#define PCG_SPMM_GW 8  // consecutive groups per warp of the sparse product
+#endif
+constexpr int kSpmmGroupsPerWarp = PCG_SPMM_GW;
 constexpr int kSpmmWide = PCG_SPMM_SPL;
 constexpr int kSpmmDepth = PCG_SPMM_DEPTH;
 constexpr int kDrawThreads = 512;  // terminal_draw_kernel
@@ -840,12 +847,15 @@ struct TransposeArgs {
     float *Dt;          // [V, bpad]
 };
 
+#ifndef PCG_TR_MINBLOCKS
+#define PCG_TR_MINBLOCKS 3  // caps the registers so that 24 warps per SM are resident (measured best)
+#endif
 // Grid (ceil(V / TT), bpad / 32): a tile of TT tokens x 32 sequences.  Warp w loads the row segments of
 // sequences w, w+8, w+16, w+24 (one 16-byte vector per lane), the tile is turned in shared memory (column
 // rotated by the vector index, so that both sides are free of bank conflicts) and written out one 128-byte
 // line per token.  Sequences past the end of the batch get zeros.
 template <typename T>
-__global__ void __launch_bounds__(kTrThreads) residual_transpose_kernel(TransposeArgs a, GroupsDev G) {
+__global__ void __launch_bounds__(kTrThreads, PCG_TR_MINBLOCKS) residual_transpose_kernel(TransposeArgs a, GroupsDev G) {
     constexpr int NV = Elem<T>::kPerVec, TT = 32 * NV;
     __shared__ float tile[TT * 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -951,64 +961,109 @@ struct SeqVec<4> {
     }
 };
 
-// Grid (ceil(M / 8), bpad / (32 * SPL)).  A warp owns one group and a block of 32 * SPL sequences; a lane
-// holds SPL consecutive sequences (one 4-, 8- or 16-byte load per token).  The warp fetches the group's token
-// list with coalesced loads (the next 32 tokens while the current ones are processed), then adds the tokens'
-// lines of Dt in CSR order, DEPTH loads in flight at a time.  The 8 x (32 * SPL) block of sums is turned in
-// shared memory so that R is written along the group index.
-#ifndef PCG_SPMM_MINBLOCKS
-#define PCG_SPMM_MINBLOCKS 4  // caps the registers so that 32 warps per SM are resident
-#endif
-template <int SPL, int DEPTH>
-__global__ void __launch_bounds__(kSpmmThreads, PCG_SPMM_MINBLOCKS) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
-    constexpr int NS = 32 * SPL;            // sequences per block
-    constexpr int GPB = kSpmmThreads / 32;  // groups per block
-    __shared__ float tile[GPB * (NS + 1)];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int gblock = blockIdx.x * GPB;
+// Grid (ceil(M / (8 * warps per block)), bpad / (32 * SPL)).  A warp owns 8 consecutive groups -- their token
+// lists are one contiguous range of the CSR -- and a block of 32 * SPL sequences; a lane holds SPL consecutive
+// sequences (one 4-, 8- or 16-byte load per token).  The range is walked in batches of DEPTH tokens with two
+// register buffers: the loads of batch i+1 are issued before batch i is added, so a warp keeps up to 2 * DEPTH
+// lines of Dt in flight at all times (random L2 gathers need on the order of 150 KB in flight per SM to
+// reach the L2's bandwidth).  Token ids are fetched 32 at a time, one block of 32 ahead.  Sums run in CSR
+// order; a group ends where the running entry index reaches the next group pointer.  The warp's 8 x (32 * SPL)
+// sums are turned in shared memory so that R is written along the group index, 32 bytes per sequence.
+template <int SPL, int DEPTH, bool HAS_W>
+__global__ void __launch_bounds__(kSpmmThreads) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
+    constexpr int NS = 32 * SPL;  // sequences per warp
+    constexpr int GW = kSpmmGroupsPerWarp;
+    constexpr int TS = NS + 4;    // row stride of the result tile (keeps 16-byte alignment, spreads banks)
+    static_assert(32 % DEPTH == 0, "a batch never straddles two blocks of 32 token ids");
+    __shared__ __align__(16) float tiles[(kSpmmThreads / 32) * GW * TS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float *tile = tiles + warp * GW * TS;
+    const int g0 = (blockIdx.x * (kSpmmThreads / 32) + warp) * GW;
+    if (g0 >= G.M) return;  // warp-uniform; the kernel has no block-wide barrier
+    const int ng = min(GW, G.M - g0);
     const float *col = a.Dt + (size_t)blockIdx.y * NS + lane * SPL;
-    const int g = gblock + warp;
+    const int ptr_l = lane <= ng ? G.group_ptr[g0 + lane] : 0;  // lane i: group_ptr[g0 + i]
+    const int e0 = __shfl_sync(0xffffffffu, ptr_l, 0), e1 = __shfl_sync(0xffffffffu, ptr_l, ng);
+    const int nbatch = (e1 - e0 + DEPTH - 1) / DEPTH;
+
+    // token ids (and weights) of entries e0 + 32*blk + lane; entries past the end repeat the last one
+    auto load_ids = [&](int blk, int &tok, float &w) {
+        const int k = min(e0 + blk * 32 + lane, e1 - 1);
+        tok = (e1 > e0) ? G.group_tok[k] : 0;
+        w = (HAS_W && e1 > e0) ? G.pair_w[k] : 1.f;
+    };
+    int ids_cur, ids_nxt;
+    float w_cur, w_nxt;
+    load_ids(0, ids_cur, w_cur);
+    load_ids(1, ids_nxt, w_nxt);
+    // issue the loads of batch i (its ids live in ids_cur if it belongs to block `blk_cur`, else in ids_nxt)
+    int blk_cur = 0;
+    auto issue = [&](int i, SeqVec<SPL>(&x)[DEPTH]) {
+        const int off = i * DEPTH;  // entry offset from e0
+        const bool in_cur = (off >> 5) == blk_cur;
+        const int src = in_cur ? ids_cur : ids_nxt;
+#pragma unroll
+        for (int j = 0; j < DEPTH; ++j) {
+            const int tok = __shfl_sync(0xffffffffu, src, (off + j) & 31);
+            x[j].load(col + (size_t)tok * a.bpad);  // past the end: a repeat of the last line, never added
+        }
+    };
     float acc[SPL];
 #pragma unroll
     for (int q = 0; q < SPL; ++q) acc[q] = 0.f;
-    if (g < G.M) {  // warp-uniform
-        const int lo = G.group_ptr[g], hi = G.group_ptr[g + 1];
-        int tok_next = lo + lane < hi ? G.group_tok[lo + lane] : 0;
-        float w_next = (G.pair_w && lo + lane < hi) ? G.pair_w[lo + lane] : 1.f;
-        for (int k0 = lo; k0 < hi; k0 += 32) {
-            const int cnt = min(32, hi - k0);
-            const int tokv = tok_next;
-            const float wv = w_next;
-            if (k0 + 32 + lane < hi) {
-                tok_next = G.group_tok[k0 + 32 + lane];
-                if (G.pair_w) w_next = G.pair_w[k0 + 32 + lane];
+    int gi = 0;
+    int gend = __shfl_sync(0xffffffffu, ptr_l, 1);
+    auto close_groups = [&](int k) {  // the entry index reached k: close every group that ends at or before k
+        while (gi < ng && gend <= k) {
+#pragma unroll
+            for (int q = 0; q < SPL; ++q) {
+                tile[gi * TS + lane * SPL + q] = acc[q];
+                acc[q] = 0.f;
             }
-            for (int j0 = 0; j0 < cnt; j0 += DEPTH) {
-                SeqVec<SPL> x[DEPTH];
+            ++gi;
+            gend = __shfl_sync(0xffffffffu, ptr_l, min(gi + 1, 31));
+        }
+    };
+    auto consume = [&](int i, const SeqVec<SPL>(&x)[DEPTH]) {
+        const int off = i * DEPTH;
+        // advance the id blocks once the first batch of a new block is consumed (its loads were issued from ids_nxt)
+        if ((off >> 5) != blk_cur) {
+            blk_cur = off >> 5;
+            ids_cur = ids_nxt;
+            w_cur = w_nxt;
+            load_ids(blk_cur + 1, ids_nxt, w_nxt);
+        }
+        const int n = min(DEPTH, e1 - e0 - off);
 #pragma unroll
-                for (int j = 0; j < DEPTH; ++j) {
-                    const int tok = __shfl_sync(0xffffffffu, tokv, (j0 + j) & 31);
-                    if (j0 + j < cnt) x[j].load(col + (size_t)tok * a.bpad);
+        for (int j = 0; j < DEPTH; ++j) {
+            if (j < n) {
+                if (HAS_W) {
+                    const float w = __shfl_sync(0xffffffffu, w_cur, (off + j) & 31);
+#pragma unroll
+                    for (int q = 0; q < SPL; ++q) acc[q] += __fmul_rn(x[j].v[q], w);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < SPL; ++q) acc[q] += x[j].v[q];
                 }
-#pragma unroll
-                for (int j = 0; j < DEPTH; ++j) {
-                    const float w = __shfl_sync(0xffffffffu, wv, (j0 + j) & 31);
-                    if (j0 + j < cnt) {
-#pragma unroll
-                        for (int q = 0; q < SPL; ++q) acc[q] += G.pair_w ? __fmul_rn(x[j].v[q], w) : x[j].v[q];
-                    }
-                }
+                close_groups(e0 + off + j + 1);
             }
         }
+    };
+    close_groups(e0);  // leading empty groups
+    SeqVec<SPL> xa[DEPTH], xb[DEPTH];
+    if (nbatch > 0) issue(0, xa);
+    for (int i = 0; i < nbatch; i += 2) {
+        if (i + 1 < nbatch) issue(i + 1, xb);
+        consume(i, xa);
+        if (i + 2 < nbatch) issue(i + 2, xa);
+        if (i + 1 < nbatch) consume(i + 1, xb);
     }
-#pragma unroll
-    for (int q = 0; q < SPL; ++q) tile[warp * (NS + 1) + lane * SPL + q] = acc[q];
-    __syncthreads();
-    // 8 consecutive threads write the 8 groups of one sequence (32 contiguous bytes of R)
-    const int gl = tid % GPB;
-    for (int sq = tid / GPB; sq < NS; sq += kSpmmThreads / GPB) {
-        const int b = a.b0 + blockIdx.y * NS + sq;
-        if (b < a.B && gblock + gl < G.M) a.R[(size_t)b * G.M + gblock + gl] = tile[gl * (NS + 1) + sq];
+    close_groups(e1);  // trailing empty groups (gi reaches ng)
+    __syncwarp();
+    const int bbase = a.b0 + blockIdx.y * NS;
+    for (int i = lane; i < NS * GW; i += 32) {  // 8 consecutive lanes: the 8 groups of one sequence
+        const int sq = i / GW, t = i - sq * GW;
+        if (bbase + sq < a.B && t < ng) a.R[(size_t)(bbase + sq) * G.M + g0 + t] = tile[t * TS + sq];
     }
 }
 
@@ -1314,10 +1369,10 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
     w.term_stats = (float4 *)(p + take((size_t)B * 16));
     w.term_n = (int32_t *)(p + take((size_t)B * 4));
     w.term_flags = (int32_t *)(p + take((size_t)B * 4));
-    if (mode & PCG_VERIFY_DENSE) {
+    if (mode == PCG_VERIFY_DENSE) {
         w.Pws = (float *)(p + take((size_t)(B * (K + 1) * M) * 4));
         w.Qws = (float *)(p + take((size_t)(B * K * M) * 4));
-    } else if (!(mode & PCG_VERIFY_CLUSTER_TERMINAL)) {
+    } else if (mode != PCG_VERIFY_CLUSTER_TERMINAL) {
         w.Dt = (float *)(p + take((size_t)V * (size_t)terminal_chunk((int)B, (int)V) * 4));
         w.R = (float *)(p + take((size_t)(B * M) * 4));
     }
@@ -1378,8 +1433,8 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         set_error("pcg_verify: K=%d exceeds the 32 positions one ballot covers", K);
         return PCG_ERR_UNSUPPORTED;
     }
-    if ((mode & ~(PCG_VERIFY_DENSE | PCG_VERIFY_CLUSTER_TERMINAL)) ||
-        mode == (PCG_VERIFY_DENSE | PCG_VERIFY_CLUSTER_TERMINAL)) {
+    if (mode != PCG_VERIFY_DEFAULT && mode != PCG_VERIFY_DENSE && mode != PCG_VERIFY_CLUSTER_TERMINAL &&
+        mode != PCG_VERIFY_BATCHED_TERMINAL) {
         set_error("pcg_verify: unknown or contradictory mode bits 0x%x", mode);
         return PCG_ERR_INVALID_ARG;
     }
@@ -1404,7 +1459,11 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
                   workspace_bytes);
         return PCG_ERR_WORKSPACE;
     }
-    const bool dense = mode & PCG_VERIFY_DENSE, cluster_terminal = mode & PCG_VERIFY_CLUSTER_TERMINAL;
+    const bool dense = mode == PCG_VERIFY_DENSE;
+    // Default: one cluster per sequence while all clusters are resident in about one wave (a handful of
+    // sequences: fewer launches, lower latency), the batched kernels beyond that.
+    const bool cluster_terminal = mode == PCG_VERIFY_CLUSTER_TERMINAL ||
+                                  (mode == PCG_VERIFY_DEFAULT && (int64_t)B * G.slices <= 2 * (int64_t)groups->sm_count);
     const size_t draw_smem = draw_smem_bytes(G.M);
     if (!cluster_terminal && draw_smem > kMaxDynSmem) {
         set_error("pcg_verify: M=%d needs %zu bytes of shared memory in the terminal draw (limit %zu)", G.M, draw_smem,
@@ -1476,12 +1535,22 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
                 SpmmArgs sp{w.Dt, B, b0, chunk, w.R};
-                const unsigned gx = (unsigned)((G.M + kSpmmThreads / 32 - 1) / (kSpmmThreads / 32));
-                if (wide)
-                    group_spmm_kernel<kSpmmWide, kSpmmDepth>
-                        <<<dim3(gx, (unsigned)(nb / kSpmmWide)), kSpmmThreads, 0, cs>>>(sp, G);
-                else
-                    group_spmm_kernel<1, 16><<<dim3(gx, (unsigned)nb), kSpmmThreads, 0, cs>>>(sp, G);
+                const int gpb = kSpmmGroupsPerWarp * (kSpmmThreads / 32);  // groups per block
+                const unsigned gx = (unsigned)((G.M + gpb - 1) / gpb);
+                const bool has_w = G.pair_w != nullptr;
+                if (wide) {
+                    const dim3 grid(gx, (unsigned)(nb / kSpmmWide));
+                    if (has_w)
+                        group_spmm_kernel<kSpmmWide, kSpmmDepth, true><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
+                    else
+                        group_spmm_kernel<kSpmmWide, kSpmmDepth, false><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
+                } else {
+                    const dim3 grid(gx, (unsigned)nb);
+                    if (has_w)
+                        group_spmm_kernel<1, 16, true><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
+                    else
+                        group_spmm_kernel<1, 16, false><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
+                }
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
             }

@@ -15,9 +15,11 @@ from oracle.compare import compare_verify  # noqa: E402
 from gpu_util import logits_to_device, make_handle, run_oracle, run_verify  # noqa: E402
 
 BAND = 1e-6
-# pcg_verify modes: default (label group per position, batched per-sequence stage), dense (P and Q of all groups at
-# every position), cluster terminal (default per-position stage, one thread-block cluster per sequence afterwards)
-MODES = [pytest.param(0, id="default"), pytest.param(1, id="dense"), pytest.param(2, id="cluster")]
+# pcg_verify modes: default (label group per position; per-sequence stage chosen by batch size), dense (P and Q of
+# all groups at every position), cluster terminal (one thread-block cluster per sequence), batched terminal
+# (transposed residual + sparse product + draw kernels)
+MODES = [pytest.param(0, id="default"), pytest.param(1, id="dense"), pytest.param(2, id="cluster"),
+         pytest.param(4, id="batched")]
 
 
 def _assert_parity(got, ref, max_excused=0):
@@ -96,7 +98,7 @@ def test_verify_batch_spanning_several_sequence_blocks(oracle):
     ref = run_oracle(oracle, bt, groups)
     assert np.any(ref.accept_len == cfg.K) and np.any(ref.accept_len == 0)
     h = make_handle(groups)
-    for mode in (0, 1, 2):
+    for mode in (0, 1, 2, 4):
         _assert_parity(run_verify(bt, h, mode=mode), ref)
 
 
@@ -157,7 +159,7 @@ def test_verify_general_split_weights(oracle, dtype, mode):
     ref = run_oracle(oracle, bt, groups, weights=w.astype(np.float64))
     got = run_verify(bt, make_handle(groups, weights=w), mode=mode)
     _assert_parity(got, ref)
-    if mode == 0:
+    if mode == 4:
         from paper_2511_13732_b200 import binding
 
         x = bt.target_logits.reshape(-1, cfg.V)[:7]
@@ -201,7 +203,7 @@ def test_verify_degenerate_memberships(oracle, kind, dtype):
     u = (rng.integers(0, 1 << 24, (B, K + 1, 2)) * 2.0 ** -24).astype(np.float32)
     bt = W.Batch(tl, dl, x, u, 0.9, dtype)
     ref = run_oracle(oracle, bt, groups)
-    for hint, mode in ((0, 0), (0, 1), (0, 2), (4, 1), (4, 2)):
+    for hint, mode in ((0, 4), (0, 1), (0, 2), (4, 1), (4, 2), (4, 0)):
         got = run_verify(bt, make_handle(groups, slices_hint=hint), mode=mode)
         _assert_parity(got, ref)
     if kind == "one_giant":
@@ -218,7 +220,7 @@ def test_verify_all_accept_all_reject_and_masked_logits(oracle):
     ref = run_oracle(oracle, same, groups)
     assert np.all(ref.accept_len == cfg.K)
     h = make_handle(groups)
-    for mode in (0, 1, 2):
+    for mode in (0, 1, 2, 4):
         _assert_parity(run_verify(same, h, mode=mode), ref)
     # draft token forced onto a token the target gives no mass (-inf): rejected at position 0
     tl, dl = bt.target_logits.copy(), bt.draft_logits.copy()
@@ -232,7 +234,7 @@ def test_verify_all_accept_all_reject_and_masked_logits(oracle):
     masked = W.Batch(tl, dl, bt.draft_tokens, bt.uniforms, 1.0, "f32")
     ref = run_oracle(oracle, masked, groups)
     assert np.all(ref.accept_len == 0)
-    for mode in (0, 1, 2):
+    for mode in (0, 1, 2, 4):
         got = run_verify(masked, h, mode=mode)
         _assert_parity(got, ref)
         assert np.all(got[3] == 0)  # -inf logits are legitimate masks, not an error
@@ -241,7 +243,7 @@ def test_verify_all_accept_all_reject_and_masked_logits(oracle):
     tl2[:, :, 17] += 60.0
     dom = W.Batch(tl2, bt.draft_logits, bt.draft_tokens, bt.uniforms, 1.0, "f32")
     ref = run_oracle(oracle, dom, groups)
-    for mode in (0, 1, 2):
+    for mode in (0, 1, 2, 4):
         _assert_parity(run_verify(dom, h, mode=mode), ref)
 
 
@@ -305,7 +307,8 @@ def test_device_side_argument_errors(oracle):
     assert binding.pcg_group_probs(tl.reshape(-1, cfg.V)[:0], h).shape == (0, groups.M)
 
 
-@pytest.mark.parametrize("mode", [pytest.param(0, id="default"), pytest.param(1, id="dense")])
+@pytest.mark.parametrize("mode", [pytest.param(0, id="default"), pytest.param(1, id="dense"),
+                                  pytest.param(2, id="cluster")])
 def test_full_size_bench_configuration_on_sampled_sequences(oracle, mode):
     """C5 exactly as bench.py launches it (B=256, K=16, V=65536, bf16): every sequence is checked for structure,
     and a sample of sequences is checked decision by decision against the oracle."""
