@@ -206,6 +206,38 @@ pcg_status pcg_verify_host(const void *target_logits, const void *draft_logits, 
                            pcg_stream stream);
 
 /*
+ * Group construction on the GPU (the group-construction equation of Sec. 2.1): the neighbourhood of token t is
+ *     G(t) = { t' : cos(Emb(t), Emb(t')) > theta },
+ * and the DISTINCT neighbourhoods form the groups.  One-time set-up ("precomputed once and cached", Sec. 2.2
+ * "Complexity and memory"), not part of the verification hot path.
+ *
+ *   emb    [V, d] DEVICE memory, row-major, PCG_BF16 or PCG_F32 (a float32 table is rounded to bfloat16,
+ *          nearest even, first: the similarity is defined on bfloat16 values, with products and sums in float32
+ *          and cos = dot * (1/|a|) * (1/|b|))
+ *   theta  threshold (strict >).  t is always a member of G(t); a zero embedding is similar to nothing else.
+ * Groups are numbered by the smallest token whose neighbourhood equals the set; tokens inside a group ascend;
+ * tok_degree counts the distinct groups containing a token.
+ * The call allocates device memory (V*V/8 bytes of scratch, freed before it returns, plus the result),
+ * synchronises the device, and returns an object that owns the result until pcg_asg_destroy.
+ * pcg_asg_csr fills a pcg_csr whose arrays are DEVICE pointers owned by the object (valid until destroy); it can
+ * be handed to pcg_groups_create as is.
+ * Errors: INVALID_ARG (null, V < 1, d < 1, bad dtype, theta not finite), UNSUPPORTED (V > 2^20), CUDA.
+ */
+typedef struct pcg_asg pcg_asg;
+typedef struct {
+    int32_t V, M;
+    int64_t nnz;
+    int32_t max_group_size;
+    int32_t max_degree;
+    float similarity_ms; /* device time of the similarity (tensor-core) kernel */
+    float total_ms;      /* device time of the whole construction */
+} pcg_asg_info_t;
+pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V, int32_t d, float theta, pcg_asg **out);
+pcg_status pcg_asg_info(const pcg_asg *asg, pcg_asg_info_t *out);
+pcg_status pcg_asg_csr(const pcg_asg *asg, pcg_csr *out);
+void pcg_asg_destroy(pcg_asg *asg);
+
+/*
  * pcg_verify for callers that have no workspace to give.  (The paper has no counterpart to this entry point;
  * it exists for the library's users only.)
  *

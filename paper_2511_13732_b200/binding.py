@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "PCG_OK", 1: "PCG_ERR_INVALID_ARG", 2: "PCG_ERR_INVALID_GROUP
 EXPORTS = [
     "pcg_status_string", "pcg_last_error", "pcg_groups_create", "pcg_groups_destroy", "pcg_groups_info",
     "pcg_group_probs", "pcg_verify_workspace_bytes", "pcg_verify", "pcg_verify_host_arena_bytes", "pcg_verify_host",
-    "pcg_verify_static",
+    "pcg_verify_static", "pcg_asg_create", "pcg_asg_info", "pcg_asg_csr", "pcg_asg_destroy",
 ]
 
 
@@ -45,6 +45,12 @@ class GroupsInfo(ctypes.Structure):
     _fields_ = [("V", ctypes.c_int32), ("M", ctypes.c_int32), ("nnz", ctypes.c_int64), ("slices", ctypes.c_int32),
                 ("slice_len", ctypes.c_int32), ("max_group_size", ctypes.c_int32), ("max_degree", ctypes.c_int32),
                 ("device", ctypes.c_int32), ("has_weights", ctypes.c_int32), ("device_bytes", ctypes.c_int64)]
+
+
+class AsgInfo(ctypes.Structure):
+    _fields_ = [("V", ctypes.c_int32), ("M", ctypes.c_int32), ("nnz", ctypes.c_int64),
+                ("max_group_size", ctypes.c_int32), ("max_degree", ctypes.c_int32),
+                ("similarity_ms", ctypes.c_float), ("total_ms", ctypes.c_float)]
 
 
 _lib = None
@@ -87,6 +93,11 @@ def load(build_if_missing: bool = True):
     lib.pcg_verify_host.restype = ctypes.c_int
     lib.pcg_verify_static.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, f32, vp, vp, vp, vp, vp]
     lib.pcg_verify_static.restype = ctypes.c_int
+    lib.pcg_asg_create.argtypes = [vp, ctypes.c_int, i32, i32, f32, ctypes.POINTER(vp)]
+    lib.pcg_asg_create.restype = ctypes.c_int
+    lib.pcg_asg_info.argtypes, lib.pcg_asg_info.restype = [vp, ctypes.POINTER(AsgInfo)], ctypes.c_int
+    lib.pcg_asg_csr.argtypes, lib.pcg_asg_csr.restype = [vp, ctypes.POINTER(_Csr)], ctypes.c_int
+    lib.pcg_asg_destroy.argtypes, lib.pcg_asg_destroy.restype = [vp], None
     _lib = lib
     return lib
 
@@ -240,3 +251,59 @@ def pcg_verify_static(target_logits, draft_logits, draft_tokens, groups: Groups,
                                     float(temperature), _dev_ptr(accept_len), _dev_ptr(tokens), _dev_ptr(grp),
                                     _dev_ptr(flags), _stream_ptr(stream)))
     return out
+
+
+class Asg:
+    """Owner of a ``pcg_asg`` object: groups built on the GPU from an embedding table (``pcg_asg_create``).
+
+    ``emb`` is a contiguous CUDA tensor [V, d], bfloat16 or float32.  ``csr_arrays()`` downloads the result;
+    ``groups()`` hands the device-resident CSR straight to ``pcg_groups_create``."""
+
+    def __init__(self, emb, theta: float):
+        if emb.dim() != 2 or not emb.is_cuda or not emb.is_contiguous():
+            raise ValueError("emb must be a contiguous CUDA tensor [V, d]")
+        self.handle = ctypes.c_void_p()
+        _check(load().pcg_asg_create(_dev_ptr(emb), dtype_code(emb), emb.shape[0], emb.shape[1], float(theta),
+                                     ctypes.byref(self.handle)))
+        self.info = AsgInfo()
+        _check(load().pcg_asg_info(self.handle, ctypes.byref(self.info)))
+        self._csr = _Csr()
+        _check(load().pcg_asg_csr(self.handle, ctypes.byref(self._csr)))
+
+    def csr_arrays(self):
+        """(group_ptr [M+1], group_tok [nnz], tok_degree [V]) as numpy int32 arrays (copied from the device)."""
+        import torch
+
+        def fetch(ptr, n):
+            if n == 0:
+                return np.zeros(0, np.int32)
+
+            class _View:  # zero-copy view of library-owned device memory
+                __cuda_array_interface__ = {"shape": (int(n),), "typestr": "<i4", "data": (int(ptr), False), "version": 2}
+
+            return torch.as_tensor(_View(), device="cuda").cpu().numpy().copy()
+
+        i = self.info
+        return fetch(self._csr.group_ptr, i.M + 1), fetch(self._csr.group_tok, i.nnz), fetch(self._csr.tok_degree, i.V)
+
+    def groups(self, slices_hint: int = 0) -> "Groups":
+        """A verification handle built directly from the device-resident result."""
+        g = Groups.__new__(Groups)
+        g._keep = (self,)
+        g.handle = ctypes.c_void_p()
+        _check(load().pcg_groups_create(ctypes.byref(self._csr), int(slices_hint), ctypes.byref(g.handle)))
+        g.info = GroupsInfo()
+        _check(load().pcg_groups_info(g.handle, ctypes.byref(g.info)))
+        g.V, g.M = g.info.V, g.info.M
+        return g
+
+    def close(self):
+        if getattr(self, "handle", None):
+            load().pcg_asg_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpcg.so")
-SOURCES = ["pcg_groups.cu", "pcg_kernels.cu", "pcg_host.cu"]
+SOURCES = ["pcg_groups.cu", "pcg_kernels.cu", "pcg_host.cu", "pcg_asg.cu"]
 HEADERS = [os.path.join(CSRC, "pcg_common.cuh"), os.path.join(ROOT, "include", "pcg.h")]
 
 

@@ -1,0 +1,507 @@
+// Group construction on the GPU: cosine-threshold neighbourhoods of an embedding table, distinct sets, CSR.
+// One-time set-up (the groups are precomputed once and cached); not part of the verification hot path.
+//
+// Stages (all on the device):
+//   asg_prepare_kernel      rows to bfloat16 (zero-padded to a multiple of 32 columns and 128 rows), 1/|row| in fp32
+//   asg_similarity_kernel   E * E^T on the tensor cores, 128 x 128 tiles; the epilogue turns each dot product
+//                           into cos = dot * rn_i * rn_j, compares with theta and packs the decisions into a
+//                           V x V BIT matrix (the V x V similarities are never stored)
+//   asg_row_kernel          per row: population count and a position-aware 64-bit hash of its bit row
+//   asg_representative_kernel  rep(t) = smallest t' with G(t') == G(t).  Such a t' is itself a member of G(t)
+//                           (t' is in G(t') = G(t)), so only the set bits below t are candidates: hash, then
+//                           a full comparison of the two bit rows
+//   scans, asg_fill_kernel  group numbers by ascending representative, group_ptr, token lists from the bit rows,
+//                           token degrees by counting
+#include <cuda_bf16.h>
+
+#include <cmath>
+#include <new>
+#include <vector>
+
+#include "pcg_common.cuh"
+
+struct pcg_asg {
+    int32_t V, M;
+    int64_t nnz;
+    int32_t max_group_size, max_degree;
+    float similarity_ms, total_ms;
+    int32_t *group_ptr, *group_tok, *tok_degree;  // device
+};
+
+namespace pcg {
+
+constexpr int kAsgTile = 128;  // rows and columns of a similarity tile
+constexpr int kAsgBK = 32;     // embedding columns per pipeline step
+constexpr int kAsgLd = 40;     // shared-memory row stride in bf16 (80 bytes: 16-byte aligned, conflict-free ldmatrix)
+constexpr int kAsgThreads = 256;
+
+// ---------------------------------------------------------------------------------------------- prepare
+// One warp per padded row.  out[r, :] = bf16(emb[r, :]) (exact for bf16 input), zero beyond d and beyond V;
+// rnorm[r] = 1 / sqrt(sum of squares of the bf16 values) in fp32, 0 for a zero row.
+template <typename T>
+__global__ void asg_prepare_kernel(const T *emb, int V, int d, int dp, int Vp, __nv_bfloat16 *out, float *rnorm) {
+    const int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (r >= Vp) return;
+    float ss = 0.f;
+    for (int c = lane; c < dp; c += 32) {
+        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+        if (r < V && c < d) {
+            if (sizeof(T) == 2)
+                v = reinterpret_cast<const __nv_bfloat16 *>(emb)[(size_t)r * d + c];
+            else
+                v = __float2bfloat16_rn(reinterpret_cast<const float *>(emb)[(size_t)r * d + c]);
+        }
+        out[(size_t)r * dp + c] = v;
+        const float f = __bfloat162float(v);
+        ss = __fmaf_rn(f, f, ss);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (lane == 0) rnorm[r] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
+}
+
+// ---------------------------------------------------------------------------------------------- similarity
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void *smem) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"((uint32_t)__cvta_generic_to_shared(smem)));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void asg_cp_async16(void *smem, const void *g) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(g)
+                 : "memory");
+}
+
+// Grid (Vp/128, Vp/128), 256 threads = 8 warps as 2 x 4; a warp owns 64 x 32 of the tile (4 x 4 mma tiles).
+// Both operands are row blocks of the same matrix E (the "B" operand is E^T, i.e. rows of E with the
+// embedding index contiguous, which is the column-major form mma expects).  bits[V, W]: bit j of word w of row i
+// says j' = 32 w + j is in G(i).
+__global__ void __launch_bounds__(kAsgThreads) asg_similarity_kernel(const __nv_bfloat16 *E, const float *rnorm, int V,
+                                                                    int dp, float theta, int W, uint32_t *bits) {
+    constexpr int T = kAsgTile, BK = kAsgBK, LD = kAsgLd;
+    __shared__ __align__(16) unsigned char smem_raw[2 * 2 * T * LD * 2];  // [stage][A|B][T][LD] bf16; reused for the decisions
+    __nv_bfloat16 *sm = reinterpret_cast<__nv_bfloat16 *>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int wm = warp >> 2, wn = warp & 3;
+    const int i0 = blockIdx.y * T, j0 = blockIdx.x * T;
+    auto tile_ptr = [&](int stage, int which) { return sm + ((size_t)stage * 2 + which) * T * LD; };
+    auto load_stage = [&](int stage, int k0) {
+        // 128 rows x 32 bf16 = 4 chunks of 16 bytes per row, per operand: 512 chunks, 2 per thread
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            const int idx = tid + c * kAsgThreads, row = idx >> 2, ch = idx & 3;
+            asg_cp_async16(tile_ptr(stage, 0) + row * LD + ch * 8, E + (size_t)(i0 + row) * dp + k0 + ch * 8);
+            asg_cp_async16(tile_ptr(stage, 1) + row * LD + ch * 8, E + (size_t)(j0 + row) * dp + k0 + ch * 8);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    float acc[4][4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
+    const int nk = dp / BK;
+    load_stage(0, 0);
+    for (int kt = 0; kt < nk; ++kt) {
+        if (kt + 1 < nk) {
+            load_stage((kt + 1) & 1, (kt + 1) * BK);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncthreads();
+        const __nv_bfloat16 *A = tile_ptr(kt & 1, 0) + (wm * 64) * LD, *B = tile_ptr(kt & 1, 1) + (wn * 32) * LD;
+#pragma unroll
+        for (int ks = 0; ks < BK; ks += 16) {
+            uint32_t af[4][4], bf[2][4];
+#pragma unroll
+            for (int mi = 0; mi < 4; ++mi) ldmatrix_x4(af[mi], A + (mi * 16 + (lane & 15)) * LD + ks + (lane >> 4) * 8);
+#pragma unroll
+            for (int nj = 0; nj < 2; ++nj)  // two n8 tiles per ldmatrix: lanes 0-15 first tile (k 0-7, 8-15), 16-31 second
+                ldmatrix_x4(bf[nj], B + (nj * 16 + (lane >> 4) * 8 + (lane & 7)) * LD + ks + ((lane >> 3) & 1) * 8);
+#pragma unroll
+            for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+                for (int ni = 0; ni < 4; ++ni) mma_bf16_16816(acc[mi][ni], af[mi], bf[ni >> 1][(ni & 1) * 2], bf[ni >> 1][(ni & 1) * 2 + 1]);
+        }
+        __syncthreads();  // the stage is overwritten by the load after next
+    }
+    // ---- decisions: one byte per (row, column) of the tile in shared memory, then 32 of them per word ----
+    constexpr int PS = T + 16;  // byte stride of a decision row
+    unsigned char *dec = smem_raw;
+    float rni[4][2], rnj[4][2];
+#pragma unroll
+    for (int mi = 0; mi < 4; ++mi) {
+        rni[mi][0] = rnorm[i0 + wm * 64 + mi * 16 + (lane >> 2)];
+        rni[mi][1] = rnorm[i0 + wm * 64 + mi * 16 + (lane >> 2) + 8];
+    }
+#pragma unroll
+    for (int ni = 0; ni < 4; ++ni) {
+        rnj[ni][0] = rnorm[j0 + wn * 32 + ni * 8 + (lane & 3) * 2];
+        rnj[ni][1] = rnorm[j0 + wn * 32 + ni * 8 + (lane & 3) * 2 + 1];
+    }
+#pragma unroll
+    for (int mi = 0; mi < 4; ++mi)
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int r = wm * 64 + mi * 16 + (lane >> 2) + (c >> 1) * 8;
+                const int q = wn * 32 + ni * 8 + (lane & 3) * 2 + (c & 1);
+                const float cosv = __fmul_rn(__fmul_rn(acc[mi][ni][c], rni[mi][c >> 1]), rnj[ni][c & 1]);
+                const bool in = (j0 + q < V) && (cosv > theta || i0 + r == j0 + q);
+                dec[r * PS + q] = in ? 1 : 0;
+            }
+    __syncthreads();
+    {
+        const int r = tid >> 1;
+        if (i0 + r < V) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int w = (tid & 1) * 2 + h;
+                const uint4 *p = reinterpret_cast<const uint4 *>(dec + r * PS + w * 32);
+                uint32_t word = 0;
+#pragma unroll
+                for (int v = 0; v < 2; ++v) {
+                    const uint4 x = p[v];
+                    const uint32_t q4[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+#pragma unroll
+                        for (int bb = 0; bb < 4; ++bb) word |= ((q4[k] >> (8 * bb)) & 1u) << (v * 16 + k * 4 + bb);
+                }
+                bits[(size_t)(i0 + r) * W + (j0 >> 5) + w] = word;
+            }
+        }
+    }
+}
+
+
+// ---------------------------------------------------------------------------------------------- rows
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {  // splitmix64 finaliser
+    x ^= x >> 30;
+    x *= 0xbf58476d1ce4e5b9ull;
+    x ^= x >> 27;
+    x *= 0x94d049bb133111ebull;
+    x ^= x >> 31;
+    return x;
+}
+
+// One warp per row: number of members and a hash of the bit row (sum of mixed (word, position) pairs, so it
+// does not depend on the order in which the lanes visit the words).
+__global__ void asg_row_kernel(const uint32_t *bits, int V, int W, int32_t *count, uint64_t *hash) {
+    const int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (t >= V) return;
+    const uint32_t *row = bits + (size_t)t * W;
+    int n = 0;
+    uint64_t h = 0;
+    for (int w = lane; w < W; w += 32) {
+        const uint32_t x = row[w];
+        n += __popc(x);
+        if (x) h += mix64(((uint64_t)(uint32_t)w << 32) | x);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        n += __shfl_xor_sync(0xffffffffu, n, o);
+        h += __shfl_xor_sync(0xffffffffu, h, o);
+    }
+    if (lane == 0) {
+        count[t] = n;
+        hash[t] = h;
+    }
+}
+
+// One warp per row t: the smallest member t' < t of G(t) whose bit row equals row t, else t itself.
+__global__ void asg_representative_kernel(const uint32_t *bits, int V, int W, const int32_t *count,
+                                          const uint64_t *hash, int32_t *rep) {
+    const int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (t >= V) return;
+    const uint32_t *row = bits + (size_t)t * W;
+    const uint64_t ht = hash[t];
+    const int ct = count[t];
+    int found = t;
+    for (int w0 = 0; w0 * 32 < t && found == t; w0 += 32) {  // 32 words = 1024 candidate tokens per round
+        const int w = w0 + lane;
+        uint32_t x = (w < W) ? row[w] : 0u;
+        if (w * 32 + 31 >= t) {  // keep candidates below t only
+            const int keep = t - w * 32;
+            x = keep <= 0 ? 0u : (keep >= 32 ? x : (x & ((1u << keep) - 1u)));
+        }
+        while (true) {
+            // smallest remaining candidate of this round whose hash and size match
+            int cand = 0x7fffffff;
+            while (x) {
+                const int j = w * 32 + __ffs(x) - 1;
+                if (hash[j] == ht && count[j] == ct) {
+                    cand = j;
+                    break;
+                }
+                x &= x - 1;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cand = min(cand, __shfl_xor_sync(0xffffffffu, cand, o));
+            if (cand == 0x7fffffff) break;
+            const uint32_t *other = bits + (size_t)cand * W;
+            bool same = true;
+            for (int k = lane; k < W; k += 32) same = same && (row[k] == other[k]);
+            if (__all_sync(0xffffffffu, same)) {
+                found = cand;
+                break;
+            }
+            if ((cand >> 5) == w) x &= ~(1u << (cand & 31));  // a hash collision: drop it and look on
+        }
+    }
+    if (lane == 0) rep[t] = found;
+}
+
+// Exclusive prefix sum of n ints by one block (set-up sizes: n <= 2^20), total to out[n].
+__global__ void asg_scan_kernel(const int32_t *in, int n, int32_t *out) {
+    __shared__ int32_t part[1024];
+    const int tid = threadIdx.x, per = (n + 1023) / 1024;
+    const int lo = min(n, tid * per), hi = min(n, lo + per);
+    int32_t s = 0;
+    for (int i = lo; i < hi; ++i) s += in[i];
+    part[tid] = s;
+    __syncthreads();
+    if (tid == 0) {
+        int32_t run = 0;
+        for (int i = 0; i < 1024; ++i) {
+            const int32_t v = part[i];
+            part[i] = run;
+            run += v;
+        }
+        out[n] = run;
+    }
+    __syncthreads();
+    int32_t run = part[tid];
+    for (int i = lo; i < hi; ++i) {
+        const int32_t v = in[i];
+        out[i] = run;
+        run += v;
+    }
+}
+
+__global__ void asg_flag_kernel(const int32_t *rep, int V, int32_t *is_rep) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < V) is_rep[t] = rep[t] == t;
+}
+
+// sizes[g] = |G(t)| for the representative t of group g = gid[t]
+__global__ void asg_sizes_kernel(const int32_t *rep, const int32_t *gid, const int32_t *count, int V, int32_t *sizes) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < V && rep[t] == t) sizes[gid[t]] = count[t];
+}
+
+// One warp per representative row: its set bits, ascending, into group_tok[group_ptr[g] ...]; degrees by counting.
+__global__ void asg_fill_kernel(const uint32_t *bits, int V, int W, const int32_t *rep, const int32_t *gid,
+                                const int32_t *group_ptr, int32_t *group_tok, int32_t *degree) {
+    const int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (t >= V || rep[t] != t) return;
+    const uint32_t *row = bits + (size_t)t * W;
+    int base = group_ptr[gid[t]];
+    for (int w0 = 0; w0 < W; w0 += 32) {
+        const int w = w0 + lane;
+        uint32_t x = w < W ? row[w] : 0u;
+        const int n = __popc(x);
+        int incl = n;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        int at = base + incl - n;
+        while (x) {
+            const int j = w * 32 + __ffs(x) - 1;
+            group_tok[at++] = j;
+            atomicAdd(&degree[j], 1);
+            x &= x - 1;
+        }
+        base += __shfl_sync(0xffffffffu, incl, 31);
+    }
+}
+
+__global__ void asg_max_kernel(const int32_t *a, int n, int32_t *out) {  // out must hold 0 on entry
+    int m = 0;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) m = max(m, a[i]);
+    atomicMax(out, m);
+}
+
+}  // namespace pcg
+
+// ================================================================================================ host side
+using namespace pcg;
+
+namespace {
+struct DeviceBuffers {  // frees whatever was allocated when it goes out of scope
+    std::vector<void *> ptrs;
+    cudaError_t alloc(void **p, size_t bytes) {
+        cudaError_t e = cudaMalloc(p, bytes ? bytes : 1);
+        if (e == cudaSuccess) ptrs.push_back(*p);
+        return e;
+    }
+    void release(void *keep) {  // forget one pointer (it now belongs to the result)
+        for (auto &q : ptrs)
+            if (q == keep) q = nullptr;
+    }
+    ~DeviceBuffers() {
+        for (void *q : ptrs)
+            if (q) cudaFree(q);
+    }
+};
+}  // namespace
+
+extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V, int32_t d, float theta,
+                                     pcg_asg **out) {
+    if (out) *out = nullptr;
+    if (!emb || !out || V < 1 || d < 1 || (dtype != PCG_F32 && dtype != PCG_BF16) || !std::isfinite(theta)) {
+        set_error("pcg_asg_create: null pointer, V < 1, d < 1, bad dtype or a threshold that is not finite");
+        return PCG_ERR_INVALID_ARG;
+    }
+    if (V > (1 << 20)) {
+        set_error("pcg_asg_create: V=%d exceeds 2^20 (the bit matrix would need %lld GB)", V,
+                  (long long)((int64_t)V * V / 8 >> 30));
+        return PCG_ERR_UNSUPPORTED;
+    }
+    const int Vp = (V + kAsgTile - 1) / kAsgTile * kAsgTile, dp = (d + kAsgBK - 1) / kAsgBK * kAsgBK, W = Vp / 32;
+    DeviceBuffers buf;
+    __nv_bfloat16 *E = nullptr;
+    float *rnorm = nullptr;
+    uint32_t *bits = nullptr;
+    int32_t *count = nullptr, *rep = nullptr, *flag = nullptr, *gid = nullptr, *sizes = nullptr, *gptr = nullptr;
+    int32_t *gtok = nullptr, *deg = nullptr, *maxes = nullptr;
+    uint64_t *hash = nullptr;
+    cudaError_t e = buf.alloc((void **)&E, (size_t)Vp * dp * 2);
+    if (e == cudaSuccess) e = buf.alloc((void **)&rnorm, (size_t)Vp * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&bits, (size_t)V * W * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&count, (size_t)V * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&hash, (size_t)V * 8);
+    if (e == cudaSuccess) e = buf.alloc((void **)&rep, (size_t)V * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&flag, (size_t)V * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&gid, ((size_t)V + 1) * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&sizes, (size_t)V * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&gptr, ((size_t)V + 1) * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&deg, (size_t)V * 4);
+    if (e == cudaSuccess) e = buf.alloc((void **)&maxes, 8);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc (group construction)");
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    for (auto &x : ev)
+        if (e == cudaSuccess) e = cudaEventCreate(&x);
+    auto drop_events = [&]() {
+        for (auto &x : ev)
+            if (x) cudaEventDestroy(x);
+    };
+    if (e != cudaSuccess) {
+        drop_events();
+        return cuda_fail(e, "cudaEventCreate");
+    }
+    const int rows_per_block = 8, row_blocks = (V + rows_per_block - 1) / rows_per_block;
+    cudaEventRecord(ev[0], 0);
+    if (dtype == PCG_BF16)
+        asg_prepare_kernel<uint16_t><<<(Vp + 7) / 8, 256>>>((const uint16_t *)emb, V, d, dp, Vp, E, rnorm);
+    else
+        asg_prepare_kernel<float><<<(Vp + 7) / 8, 256>>>((const float *)emb, V, d, dp, Vp, E, rnorm);
+    cudaEventRecord(ev[1], 0);
+    asg_similarity_kernel<<<dim3(Vp / kAsgTile, Vp / kAsgTile), kAsgThreads>>>(E, rnorm, V, dp, theta, W, bits);
+    cudaEventRecord(ev[2], 0);
+    asg_row_kernel<<<row_blocks, 256>>>(bits, V, W, count, hash);
+    asg_representative_kernel<<<row_blocks, 256>>>(bits, V, W, count, hash, rep);
+    asg_flag_kernel<<<(V + 255) / 256, 256>>>(rep, V, flag);
+    asg_scan_kernel<<<1, 1024>>>(flag, V, gid);  // gid[t] = group number of a representative t; gid[V] = M
+    int32_t M = 0;
+    e = cudaMemcpy(&M, gid + V, 4, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) {
+        asg_sizes_kernel<<<(V + 255) / 256, 256>>>(rep, gid, count, V, sizes);
+        asg_scan_kernel<<<1, 1024>>>(sizes, M, gptr);
+    }
+    int32_t nnz = 0;
+    if (e == cudaSuccess) e = cudaMemcpy(&nnz, gptr + M, 4, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = buf.alloc((void **)&gtok, (size_t)nnz * 4);
+    if (e == cudaSuccess) e = cudaMemsetAsync(deg, 0, (size_t)V * 4, 0);
+    if (e == cudaSuccess) e = cudaMemsetAsync(maxes, 0, 8, 0);
+    int32_t mx[2] = {0, 0};
+    float sim_ms = 0.f, total_ms = 0.f;
+    if (e == cudaSuccess) {
+        asg_fill_kernel<<<row_blocks, 256>>>(bits, V, W, rep, gid, gptr, gtok, deg);
+        asg_max_kernel<<<64, 256>>>(sizes, M, maxes);
+        asg_max_kernel<<<64, 256>>>(deg, V, maxes + 1);
+        cudaEventRecord(ev[3], 0);
+        e = cudaMemcpy(mx, maxes, 8, cudaMemcpyDeviceToHost);
+    }
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e == cudaSuccess) {
+        cudaEventElapsedTime(&sim_ms, ev[1], ev[2]);
+        cudaEventElapsedTime(&total_ms, ev[0], ev[3]);
+    }
+    drop_events();
+    if (e != cudaSuccess) return cuda_fail(e, "group construction");
+    // the result keeps exact-size copies of group_ptr; group_tok and the degrees are handed over as they are
+    int32_t *gptr_out = nullptr;
+    e = buf.alloc((void **)&gptr_out, ((size_t)M + 1) * 4);
+    if (e == cudaSuccess) e = cudaMemcpy(gptr_out, gptr, ((size_t)M + 1) * 4, cudaMemcpyDeviceToDevice);
+    if (e != cudaSuccess) return cuda_fail(e, "copying group_ptr");
+    pcg_asg *r = new (std::nothrow) pcg_asg();
+    if (!r) {
+        set_error("out of host memory");
+        return PCG_ERR_INVALID_ARG;
+    }
+    r->V = V;
+    r->M = M;
+    r->nnz = nnz;
+    r->max_group_size = mx[0];
+    r->max_degree = mx[1];
+    r->similarity_ms = sim_ms;
+    r->total_ms = total_ms;
+    r->group_ptr = gptr_out;
+    r->group_tok = gtok;
+    r->tok_degree = deg;
+    buf.release(gptr_out);
+    buf.release(gtok);
+    buf.release(deg);
+    *out = r;
+    return PCG_OK;
+}
+
+extern "C" pcg_status pcg_asg_info(const pcg_asg *asg, pcg_asg_info_t *out) {
+    if (!asg || !out) {
+        set_error("pcg_asg_info: null argument");
+        return PCG_ERR_INVALID_ARG;
+    }
+    out->V = asg->V;
+    out->M = asg->M;
+    out->nnz = asg->nnz;
+    out->max_group_size = asg->max_group_size;
+    out->max_degree = asg->max_degree;
+    out->similarity_ms = asg->similarity_ms;
+    out->total_ms = asg->total_ms;
+    return PCG_OK;
+}
+
+extern "C" pcg_status pcg_asg_csr(const pcg_asg *asg, pcg_csr *out) {
+    if (!asg || !out) {
+        set_error("pcg_asg_csr: null argument");
+        return PCG_ERR_INVALID_ARG;
+    }
+    out->V = asg->V;
+    out->M = asg->M;
+    out->nnz = asg->nnz;
+    out->group_ptr = asg->group_ptr;
+    out->group_tok = asg->group_tok;
+    out->tok_degree = asg->tok_degree;
+    out->weights = nullptr;
+    return PCG_OK;
+}
+
+extern "C" void pcg_asg_destroy(pcg_asg *asg) {
+    if (!asg) return;
+    cudaFree(asg->group_ptr);
+    cudaFree(asg->group_tok);
+    cudaFree(asg->tok_degree);
+    delete asg;
+}
