@@ -215,13 +215,16 @@ pcg_status pcg_verify_host(const void *target_logits, const void *draft_logits, 
  *          nearest even, first: the similarity is defined on bfloat16 values, with products and sums in float32
  *          and cos = dot * (1/|a|) * (1/|b|))
  *   theta  threshold (strict >).  t is always a member of G(t); a zero embedding is similar to nothing else.
+ *   flags  0: the similarity tiles run on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
+ *          memory); PCG_ASG_MMA_SYNC: the same tiles with warp-level mma.sync (kept as a cross-check)
  * Groups are numbered by the smallest token whose neighbourhood equals the set; tokens inside a group ascend;
  * tok_degree counts the distinct groups containing a token.
  * The call allocates device memory (V*V/8 bytes of scratch, freed before it returns, plus the result),
  * synchronises the device, and returns an object that owns the result until pcg_asg_destroy.
  * pcg_asg_csr fills a pcg_csr whose arrays are DEVICE pointers owned by the object (valid until destroy); it can
  * be handed to pcg_groups_create as is.
- * Errors: INVALID_ARG (null, V < 1, d < 1, bad dtype, theta not finite), UNSUPPORTED (V > 2^20), CUDA.
+ * Errors: INVALID_ARG (null, V < 1, d < 1, bad dtype, theta not finite, unknown flags), UNSUPPORTED (V > 2^20),
+ * CUDA (also when the tensor-core kernel gave up a bounded wait; pcg_last_error says so).
  */
 typedef struct pcg_asg pcg_asg;
 typedef struct {
@@ -231,8 +234,11 @@ typedef struct {
     int32_t max_degree;
     float similarity_ms; /* device time of the similarity (tensor-core) kernel */
     float total_ms;      /* device time of the whole construction */
+    int32_t tensor_path; /* 1 = tcgen05, 0 = mma.sync */
 } pcg_asg_info_t;
-pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V, int32_t d, float theta, pcg_asg **out);
+#define PCG_ASG_MMA_SYNC 1u
+pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V, int32_t d, float theta, uint32_t flags,
+                          pcg_asg **out);
 pcg_status pcg_asg_info(const pcg_asg *asg, pcg_asg_info_t *out);
 pcg_status pcg_asg_csr(const pcg_asg *asg, pcg_csr *out);
 void pcg_asg_destroy(pcg_asg *asg);

@@ -50,7 +50,7 @@ class GroupsInfo(ctypes.Structure):
 class AsgInfo(ctypes.Structure):
     _fields_ = [("V", ctypes.c_int32), ("M", ctypes.c_int32), ("nnz", ctypes.c_int64),
                 ("max_group_size", ctypes.c_int32), ("max_degree", ctypes.c_int32),
-                ("similarity_ms", ctypes.c_float), ("total_ms", ctypes.c_float)]
+                ("similarity_ms", ctypes.c_float), ("total_ms", ctypes.c_float), ("tensor_path", ctypes.c_int32)]
 
 
 _lib = None
@@ -93,7 +93,7 @@ def load(build_if_missing: bool = True):
     lib.pcg_verify_host.restype = ctypes.c_int
     lib.pcg_verify_static.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, f32, vp, vp, vp, vp, vp]
     lib.pcg_verify_static.restype = ctypes.c_int
-    lib.pcg_asg_create.argtypes = [vp, ctypes.c_int, i32, i32, f32, ctypes.POINTER(vp)]
+    lib.pcg_asg_create.argtypes = [vp, ctypes.c_int, i32, i32, f32, u32, ctypes.POINTER(vp)]
     lib.pcg_asg_create.restype = ctypes.c_int
     lib.pcg_asg_info.argtypes, lib.pcg_asg_info.restype = [vp, ctypes.POINTER(AsgInfo)], ctypes.c_int
     lib.pcg_asg_csr.argtypes, lib.pcg_asg_csr.restype = [vp, ctypes.POINTER(_Csr)], ctypes.c_int
@@ -259,12 +259,12 @@ class Asg:
     ``emb`` is a contiguous CUDA tensor [V, d], bfloat16 or float32.  ``csr_arrays()`` downloads the result;
     ``groups()`` hands the device-resident CSR straight to ``pcg_groups_create``."""
 
-    def __init__(self, emb, theta: float):
+    def __init__(self, emb, theta: float, mma_sync: bool = False):
         if emb.dim() != 2 or not emb.is_cuda or not emb.is_contiguous():
             raise ValueError("emb must be a contiguous CUDA tensor [V, d]")
         self.handle = ctypes.c_void_p()
         _check(load().pcg_asg_create(_dev_ptr(emb), dtype_code(emb), emb.shape[0], emb.shape[1], float(theta),
-                                     ctypes.byref(self.handle)))
+                                     1 if mma_sync else 0, ctypes.byref(self.handle)))
         self.info = AsgInfo()
         _check(load().pcg_asg_info(self.handle, ctypes.byref(self.info)))
         self._csr = _Csr()

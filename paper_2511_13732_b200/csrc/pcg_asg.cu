@@ -26,6 +26,7 @@ struct pcg_asg {
     int32_t max_group_size, max_degree;
     float similarity_ms, total_ms;
     int32_t *group_ptr, *group_tok, *tok_degree;  // device
+    int32_t tensor_path;                          // 1 = tcgen05, 0 = mma.sync
 };
 
 namespace pcg {
@@ -182,6 +183,207 @@ __global__ void __launch_bounds__(kAsgThreads) asg_similarity_kernel(const __nv_
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------- similarity, tcgen05
+// 256 x 256 tiles on the 5th-generation tensor cores: one thread issues tcgen05.mma (M = 128, N = 256, K = 16 per
+// instruction, two instructions per K step for the two 128-row halves of the tile) on operands staged in shared
+// memory; the two 128 x 256 fp32 accumulators fill the SM's tensor memory (128 lanes x 512 columns) and are read
+// back with tcgen05.ld, one accumulator row per thread, which is exactly the row of 256 decisions (eight 32-bit
+// words) that thread then writes.  The large tile is what keeps the operand traffic from L2 (128 flop per byte)
+// below the tensor cores' appetite; a 128 x 128 tile (64 flop per byte) is L2-bound.
+//
+// Shared-memory operand layout (K-major, no swizzle): 8 rows x 16 bytes form a 128-byte core matrix; core
+// matrices that are neighbours along K sit 128 bytes apart (leading byte offset), groups of 8 rows 1024 bytes
+// apart (stride byte offset).  With 64 bf16 (8 chunks of 16 bytes) per row and stage, chunk (row, c) lands at
+// byte (row/8)*1024 + c*128 + (row%8)*16, which makes the cp.async destinations of consecutive threads contiguous.
+// Every wait on an mbarrier is bounded: on a time-out the block records an error code, drains its own copies,
+// frees its tensor memory and returns.
+constexpr int kTcBK = 64;       // bf16 per row and stage
+#ifndef PCG_TC_HALVES
+#define PCG_TC_HALVES 2  // 128-row accumulators per block: 2 = 256 x 256 tiles, one block per SM (measured best); 1 = 128 x 256
+#endif
+#ifndef PCG_TC_STAGES
+#define PCG_TC_STAGES 3
+#endif
+constexpr int kTcHalves = PCG_TC_HALVES;
+constexpr int kTcStages = PCG_TC_STAGES;  // operand stages in shared memory
+constexpr int kTcThreads = 128 * kTcHalves;
+constexpr int kTcTile = 256;              // columns of a tile (rows of the B operand); Vp is a multiple of it
+constexpr int kTcRows = 128 * kTcHalves;  // rows of a tile (rows of the A operand)
+constexpr int kTcABytes = kTcRows * kTcBK * 2, kTcBBytes = kTcTile * kTcBK * 2;
+constexpr int kTcStageBytes = kTcABytes + kTcBBytes;
+constexpr uint32_t kTcSpinLimit = 1u << 22;  // polls of about 50 ns each: gives up after a fraction of a second
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        __nanosleep(32);
+    }
+    return false;
+}
+__device__ __forceinline__ uint64_t umma_desc_kmajor_noswizzle(uint32_t smem_addr) {
+    // start address >> 4 | leading byte offset (128) >> 4 at bit 16 | stride byte offset (1024) >> 4 at bit 32 |
+    // descriptor version 1 at bit 46; layout type 0 (no swizzle), base offset 0
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           (1ull << 46);
+}
+// kind::f16 instruction descriptor: D = fp32 (1 << 4), A = B = bf16 (1 << 7, 1 << 10), both K-major,
+// N = 256 (256 >> 3 at bit 17), M = 128 (128 >> 4 at bit 24)
+constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+
+__global__ void __launch_bounds__(kTcThreads) asg_similarity_tc_kernel(const __nv_bfloat16 *E, const float *rnorm,
+                                                                      int V, int dp, float theta, int W,
+                                                                      uint32_t *bits, int *error) {
+    constexpr int T = kTcTile, BK = kTcBK, S = kTcStages;
+    extern __shared__ __align__(128) unsigned char tc_smem[];  // [S][A | B][256 rows x 128 bytes]
+    __shared__ __align__(8) uint64_t mbar[S + 1];              // stage s: its MMAs have finished; [S]: accumulator ready
+    __shared__ uint32_t tmem_slot;
+    __shared__ float rnj[T];
+    __shared__ int failed;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int i0 = blockIdx.y * kTcRows, j0 = blockIdx.x * T;
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(tc_smem);
+    const uint32_t bar_base = (uint32_t)__cvta_generic_to_shared(mbar);
+    if (tid == 0) {
+        for (int s = 0; s <= S; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_base + 8 * s));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        failed = 0;
+    }
+    for (int c = tid; c < T; c += kTcThreads) rnj[c] = rnorm[j0 + c];
+    if (warp == 0) {  // tensor memory: 256 columns per 128 x 256 accumulator, allocated and freed by warp 0
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         (uint32_t)__cvta_generic_to_shared(&tmem_slot)),
+                     "r"(256 * kTcHalves));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_slot;
+
+    auto load_stage = [&](int s, int k0) {
+        // per operand 256 rows x 8 chunks; thread handles chunks idx = tid + 256 i: row = (idx/64)*8 + idx%8,
+        // chunk = (idx/8)%8, destination byte idx*16 (see the layout above)
+        unsigned char *a = tc_smem + (size_t)s * kTcStageBytes, *b = a + kTcABytes;
+#pragma unroll
+        for (int i = 0; i < kTcRows * 8 / kTcThreads; ++i) {
+            const int idx = tid + i * kTcThreads, row = (idx >> 6) * 8 + (idx & 7), c = (idx >> 3) & 7;
+            asg_cp_async16(a + idx * 16, E + (size_t)(i0 + row) * dp + k0 + c * 8);
+        }
+#pragma unroll
+        for (int i = 0; i < T * 8 / kTcThreads; ++i) {
+            const int idx = tid + i * kTcThreads, row = (idx >> 6) * 8 + (idx & 7), c = (idx >> 3) & 7;
+            asg_cp_async16(b + idx * 16, E + (size_t)(j0 + row) * dp + k0 + c * 8);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    const int nk = dp / BK;
+    bool ok = true;
+    // tiles 0 .. S-2 in flight before the loop; inside, tile kt + S - 1 is fetched once the MMAs of tile kt - 1
+    // (same stage) have finished
+#pragma unroll
+    for (int p = 0; p < S - 1; ++p) {
+        if (p < nk) load_stage(p, p * BK);
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (int kt = 0; kt < nk; ++kt) {
+        const int nxt = kt + S - 1;
+        if (nxt < nk) {
+            if (kt >= 1) ok = ok && mbar_wait_bounded(bar_base + 8 * ((kt - 1) % S), ((kt - 1) / S) & 1);
+            if (ok) load_stage(nxt % S, nxt * BK);
+            else asm volatile("cp.async.commit_group;" ::: "memory");
+        } else {
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        asm volatile("cp.async.wait_group %0;" ::"n"(S - 1) : "memory");  // this thread's part of tile kt has landed
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // ... and is visible to the tensor core
+        if (!ok) failed = 1;
+        __syncthreads();
+        if (failed) break;
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a = smem_base + (uint32_t)((kt % S) * kTcStageBytes), b = a + kTcABytes;
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk) {
+                const uint64_t db = umma_desc_kmajor_noswizzle(b + kk * 256);
+                const uint32_t accumulate = (kt > 0 || kk > 0) ? 1u : 0u;
+#pragma unroll
+                for (int half = 0; half < kTcHalves; ++half) {  // rows 0-127 -> columns 0-255 of tensor memory, rows 128-255 -> 256-511
+                    const uint64_t da = umma_desc_kmajor_noswizzle(a + half * (128 * 128) + kk * 256);
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+                        :
+                        : "r"(tmem + half * 256), "l"(da), "l"(db), "r"(kTcIdesc), "r"(accumulate), "r"(0u), "r"(0u),
+                          "r"(0u), "r"(0u)
+                        : "memory");
+                }
+            }
+            // arrives on the stage's barrier when every MMA issued so far has finished reading shared memory
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                             bar_base + 8 * (kt % S))
+                         : "memory");
+            if (kt == nk - 1)
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                                 bar_base + 8 * S)
+                             : "memory");
+        }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (!failed) {
+        if (!mbar_wait_bounded(bar_base + 8 * S, 0)) failed = 2;
+    }
+    __syncthreads();
+    if (!failed) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // warps 0-3 read the first accumulator (tile rows 0-127), warps 4-7 the second; a warp may only touch the
+        // 32 lanes of tensor memory given by its index modulo 4.  Thread = one tile row: eight loads of 32 columns
+        // = eight words of decisions
+        const int half = warp >> 2, quarter = warp & 3;
+        const int r = half * 128 + quarter * 32 + lane;
+        const float rni = rnorm[i0 + r];
+        uint32_t words[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t v[32];
+            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256 + q * 32);
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
+                "%15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                  "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                  "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                  "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                : "r"(taddr));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            uint32_t word = 0;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                const int col = q * 32 + c;
+                const float cosv = __fmul_rn(__fmul_rn(__uint_as_float(v[c]), rni), rnj[col]);
+                const bool in = (j0 + col < V) && (cosv > theta || i0 + r == j0 + col);
+                word |= (in ? 1u : 0u) << c;
+            }
+            words[q] = word;
+        }
+        if (i0 + r < V) {
+            uint4 *dst = reinterpret_cast<uint4 *>(bits + (size_t)(i0 + r) * W + (j0 >> 5));
+            dst[0] = make_uint4(words[0], words[1], words[2], words[3]);
+            dst[1] = make_uint4(words[4], words[5], words[6], words[7]);
+        }
+    } else if (tid == 0) {
+        atomicMax(error, failed);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256 * kTcHalves));
+}
 
 // ---------------------------------------------------------------------------------------------- rows
 __device__ __forceinline__ uint64_t mix64(uint64_t x) {  // splitmix64 finaliser
@@ -357,10 +559,14 @@ struct DeviceBuffers {  // frees whatever was allocated when it goes out of scop
 }  // namespace
 
 extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V, int32_t d, float theta,
-                                     pcg_asg **out) {
+                                     uint32_t flags, pcg_asg **out) {
     if (out) *out = nullptr;
     if (!emb || !out || V < 1 || d < 1 || (dtype != PCG_F32 && dtype != PCG_BF16) || !std::isfinite(theta)) {
         set_error("pcg_asg_create: null pointer, V < 1, d < 1, bad dtype or a threshold that is not finite");
+        return PCG_ERR_INVALID_ARG;
+    }
+    if (flags & ~PCG_ASG_MMA_SYNC) {
+        set_error("pcg_asg_create: unknown flag bits 0x%x", flags);
         return PCG_ERR_INVALID_ARG;
     }
     if (V > (1 << 20)) {
@@ -368,7 +574,7 @@ extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V
                   (long long)((int64_t)V * V / 8 >> 30));
         return PCG_ERR_UNSUPPORTED;
     }
-    const int Vp = (V + kAsgTile - 1) / kAsgTile * kAsgTile, dp = (d + kAsgBK - 1) / kAsgBK * kAsgBK, W = Vp / 32;
+    const int Vp = (V + kTcTile - 1) / kTcTile * kTcTile, dp = (d + kTcBK - 1) / kTcBK * kTcBK, W = Vp / 32;
     DeviceBuffers buf;
     __nv_bfloat16 *E = nullptr;
     float *rnorm = nullptr;
@@ -387,7 +593,7 @@ extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V
     if (e == cudaSuccess) e = buf.alloc((void **)&sizes, (size_t)V * 4);
     if (e == cudaSuccess) e = buf.alloc((void **)&gptr, ((size_t)V + 1) * 4);
     if (e == cudaSuccess) e = buf.alloc((void **)&deg, (size_t)V * 4);
-    if (e == cudaSuccess) e = buf.alloc((void **)&maxes, 8);
+    if (e == cudaSuccess) e = buf.alloc((void **)&maxes, 16);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc (group construction)");
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     for (auto &x : ev)
@@ -406,9 +612,35 @@ extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V
         asg_prepare_kernel<uint16_t><<<(Vp + 7) / 8, 256>>>((const uint16_t *)emb, V, d, dp, Vp, E, rnorm);
     else
         asg_prepare_kernel<float><<<(Vp + 7) / 8, 256>>>((const float *)emb, V, d, dp, Vp, E, rnorm);
+    cudaMemsetAsync(maxes, 0, 16, 0);  // [0] largest group, [1] largest degree, [2] error code of the tensor-core kernel
     cudaEventRecord(ev[1], 0);
-    asg_similarity_kernel<<<dim3(Vp / kAsgTile, Vp / kAsgTile), kAsgThreads>>>(E, rnorm, V, dp, theta, W, bits);
+    const dim3 tiles(Vp / kAsgTile, Vp / kAsgTile);
+    if (flags & PCG_ASG_MMA_SYNC) {
+        asg_similarity_kernel<<<tiles, kAsgThreads>>>(E, rnorm, V, dp, theta, W, bits);
+    } else {
+        const int smem = kTcStages * kTcStageBytes;
+        e = cudaFuncSetAttribute(asg_similarity_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) {
+            drop_events();
+            return cuda_fail(e, "cudaFuncSetAttribute (asg_similarity_tc_kernel)");
+        }
+        asg_similarity_tc_kernel<<<dim3(Vp / kTcTile, Vp / kTcRows), kTcThreads, smem>>>(E, rnorm, V, dp, theta, W, bits,
+                                                                                        maxes + 2);
+    }
     cudaEventRecord(ev[2], 0);
+    {
+        int32_t tc_error = 0;
+        e = cudaMemcpy(&tc_error, maxes + 2, 4, cudaMemcpyDeviceToHost);
+        if (e == cudaSuccess && tc_error) {
+            drop_events();
+            set_error("pcg_asg_create: the tensor-core pipeline gave up waiting on a barrier (code %d)", tc_error);
+            return PCG_ERR_CUDA;
+        }
+        if (e != cudaSuccess) {
+            drop_events();
+            return cuda_fail(e, "similarity kernel");
+        }
+    }
     asg_row_kernel<<<row_blocks, 256>>>(bits, V, W, count, hash);
     asg_representative_kernel<<<row_blocks, 256>>>(bits, V, W, count, hash, rep);
     asg_flag_kernel<<<(V + 255) / 256, 256>>>(rep, V, flag);
@@ -423,7 +655,6 @@ extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V
     if (e == cudaSuccess) e = cudaMemcpy(&nnz, gptr + M, 4, cudaMemcpyDeviceToHost);
     if (e == cudaSuccess) e = buf.alloc((void **)&gtok, (size_t)nnz * 4);
     if (e == cudaSuccess) e = cudaMemsetAsync(deg, 0, (size_t)V * 4, 0);
-    if (e == cudaSuccess) e = cudaMemsetAsync(maxes, 0, 8, 0);
     int32_t mx[2] = {0, 0};
     float sim_ms = 0.f, total_ms = 0.f;
     if (e == cudaSuccess) {
@@ -458,6 +689,7 @@ extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V
     r->max_degree = mx[1];
     r->similarity_ms = sim_ms;
     r->total_ms = total_ms;
+    r->tensor_path = (flags & PCG_ASG_MMA_SYNC) ? 0 : 1;
     r->group_ptr = gptr_out;
     r->group_tok = gtok;
     r->tok_degree = deg;
@@ -480,6 +712,7 @@ extern "C" pcg_status pcg_asg_info(const pcg_asg *asg, pcg_asg_info_t *out) {
     out->max_degree = asg->max_degree;
     out->similarity_ms = asg->similarity_ms;
     out->total_ms = asg->total_ms;
+    out->tensor_path = asg->tensor_path;
     return PCG_OK;
 }
 

@@ -34,17 +34,21 @@ def _clear_threshold(emb, theta0, width=0.02):
 
 
 def _check(emb, theta):
+    """Both tensor-core paths (tcgen05 and mma.sync) against the oracle."""
     from oracle import asg_oracle as A
     from paper_2511_13732_b200 import binding
 
     want = A.build_groups(emb, theta)
     assert want.min_margin > BAND, "test table has a pair too close to the threshold"
-    asg = binding.Asg(_to_device(emb), theta)
-    gp, gt, dg = asg.csr_arrays()
-    assert asg.info.M == want.M and asg.info.nnz == want.group_tok.size
-    assert np.array_equal(gp, want.group_ptr) and np.array_equal(gt, want.group_tok) and np.array_equal(dg, want.tok_degree)
-    sizes = np.diff(want.group_ptr)
-    assert asg.info.max_group_size == sizes.max() and asg.info.max_degree == want.tok_degree.max()
+    for mma_sync in (False, True):
+        asg = binding.Asg(_to_device(emb), theta, mma_sync=mma_sync)
+        assert asg.info.tensor_path == (0 if mma_sync else 1)
+        gp, gt, dg = asg.csr_arrays()
+        assert asg.info.M == want.M and asg.info.nnz == want.group_tok.size
+        assert np.array_equal(gp, want.group_ptr) and np.array_equal(gt, want.group_tok)
+        assert np.array_equal(dg, want.tok_degree)
+        sizes = np.diff(want.group_ptr)
+        assert asg.info.max_group_size == sizes.max() and asg.info.max_degree == want.tok_degree.max()
     return asg, want
 
 
