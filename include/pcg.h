@@ -37,8 +37,9 @@ typedef enum {
 } pcg_status;
 
 typedef enum {
-    PCG_F32 = 0, /* IEEE float32 logits */
-    PCG_BF16 = 1 /* bfloat16 logits (upper 16 bits of a float32) */
+    PCG_F32 = 0,  /* IEEE float32 logits */
+    PCG_BF16 = 1, /* bfloat16 logits (upper 16 bits of a float32) */
+    PCG_F16 = 2   /* IEEE binary16 logits */
 } pcg_dtype;
 
 /* CUDA stream handle (a cudaStream_t / CUstream); NULL is the default stream. */
@@ -133,6 +134,14 @@ pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg_groups **o
 void pcg_groups_destroy(pcg_groups *groups);
 
 pcg_status pcg_groups_info(const pcg_groups *groups, pcg_groups_info_t *out);
+
+/*
+ * Constant added to the acceptance ratio of every later pcg_verify call with this handle: accept iff
+ * u < min(1, P/Q) + bias.  0 (the default) is PCG; a positive value gives the lossy relaxation the paper compares
+ * against (Sec. 3.2: speculative decoding with a constant bias of 0.3 on the acceptance probability).  The
+ * residual and the token draws are unchanged.  Errors: INVALID_ARG (null, bias < 0 or not finite).
+ */
+pcg_status pcg_groups_set_accept_bias(pcg_groups *groups, float bias);
 
 /*
  * Coarse-grained group distribution of every row (the coarse-grained

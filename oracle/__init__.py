@@ -6,6 +6,7 @@ this package.  It shares nothing with the CUDA library and never imports it.
 from .pcg_oracle import (  # noqa: F401
     F32,
     BF16,
+    F16,
     FLAG_ZERO_RESIDUAL,
     build,
     max_threads,

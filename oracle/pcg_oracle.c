@@ -38,14 +38,30 @@
 
 #define ORACLE_F32 0
 #define ORACLE_BF16 1
+#define ORACLE_F16 2
 
 /* flag bits written per sequence */
 #define ORACLE_FLAG_ZERO_RESIDUAL 2 /* reject taken but sum of (P-Q)_+ was <= 0 */
+
+/* IEEE binary16 bit pattern to double, from the format's definition: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static double half_bits_to_double(uint16_t h) {
+    int sign = h >> 15, ex = (h >> 10) & 0x1f, frac = h & 0x3ff;
+    double v;
+    if (ex == 0)
+        v = ldexp((double)frac, -24); /* zero and subnormals: frac * 2^-10 * 2^-14 */
+    else if (ex == 31)
+        v = frac ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + (double)frac / 1024.0, ex - 15);
+    return sign ? -v : v;
+}
 
 /* Widen one stored logit to double exactly (bf16 = upper 16 bits of a float). */
 static double load_logit(const void *base, int dtype, int64_t idx) {
     if (dtype == ORACLE_F32) {
         return (double)((const float *)base)[idx];
+    } else if (dtype == ORACLE_F16) {
+        return half_bits_to_double(((const uint16_t *)base)[idx]);
     } else {
         uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
         float f;

@@ -2,7 +2,7 @@
 
 The arithmetic lives in ``pcg_oracle.c`` beside this file; this module only
 compiles it with gcc, marshals numpy arrays and returns numpy arrays.  Logits
-are passed as float32 arrays, or as uint16 arrays holding bf16 bit patterns.
+are passed as float32 or float16 arrays, or as uint16 arrays holding bf16 bit patterns.
 """
 from __future__ import annotations
 
@@ -15,6 +15,7 @@ import numpy as np
 
 F32 = 0
 BF16 = 1
+F16 = 2
 FLAG_ZERO_RESIDUAL = 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -61,7 +62,9 @@ def _logits(a):
         return a, F32
     if a.dtype == np.uint16:
         return a, BF16
-    raise TypeError("logits must be float32 or uint16 (bf16 bit patterns)")
+    if a.dtype == np.float16:
+        return a, F16
+    raise TypeError("logits must be float32, float16 or uint16 (bf16 bit patterns)")
 
 
 def _i32(a):

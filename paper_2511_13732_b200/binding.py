@@ -16,7 +16,7 @@ import numpy as np
 
 from . import build as _build
 
-PCG_F32, PCG_BF16 = 0, 1
+PCG_F32, PCG_BF16, PCG_F16 = 0, 1, 2
 FLAG_BAD_DRAFT_TOKEN, FLAG_ZERO_RESIDUAL, FLAG_NONFINITE = 1, 2, 4
 VERIFY_DEFAULT, VERIFY_DENSE, VERIFY_CLUSTER_TERMINAL, VERIFY_BATCHED_TERMINAL = 0, 1, 2, 4
 STATUS_NAMES = {0: "PCG_OK", 1: "PCG_ERR_INVALID_ARG", 2: "PCG_ERR_INVALID_GROUPS", 3: "PCG_ERR_UNSUPPORTED",
@@ -24,6 +24,7 @@ STATUS_NAMES = {0: "PCG_OK", 1: "PCG_ERR_INVALID_ARG", 2: "PCG_ERR_INVALID_GROUP
 
 EXPORTS = [
     "pcg_status_string", "pcg_last_error", "pcg_groups_create", "pcg_groups_destroy", "pcg_groups_info",
+    "pcg_groups_set_accept_bias",
     "pcg_group_probs", "pcg_verify_workspace_bytes", "pcg_verify", "pcg_verify_host_arena_bytes", "pcg_verify_host",
     "pcg_verify_static", "pcg_asg_create", "pcg_asg_info", "pcg_asg_csr", "pcg_asg_destroy",
 ]
@@ -81,6 +82,7 @@ def load(build_if_missing: bool = True):
     lib.pcg_groups_create.restype = ctypes.c_int
     lib.pcg_groups_destroy.argtypes, lib.pcg_groups_destroy.restype = [vp], None
     lib.pcg_groups_info.argtypes, lib.pcg_groups_info.restype = [vp, ctypes.POINTER(GroupsInfo)], ctypes.c_int
+    lib.pcg_groups_set_accept_bias.argtypes, lib.pcg_groups_set_accept_bias.restype = [vp, f32], ctypes.c_int
     lib.pcg_group_probs.argtypes = [vp, ctypes.c_int, i64, f32, vp, vp, vp]
     lib.pcg_group_probs.restype = ctypes.c_int
     lib.pcg_verify_workspace_bytes.argtypes = [i32, i32, i32, i32, ctypes.c_int, u32]
@@ -130,7 +132,9 @@ def dtype_code(t) -> int:
         return PCG_F32
     if t.dtype == torch.bfloat16 or t.dtype == torch.uint16 or t.dtype == torch.int16:
         return PCG_BF16
-    raise TypeError(f"logits must be float32 or bfloat16 (or 16-bit integer bit patterns), got {t.dtype}")
+    if t.dtype == torch.float16:
+        return PCG_F16
+    raise TypeError(f"logits must be float32, float16 or bfloat16 (or 16-bit integer bf16 bit patterns), got {t.dtype}")
 
 
 class Groups:
@@ -149,6 +153,10 @@ class Groups:
         _check(lib.pcg_groups_info(self.handle, ctypes.byref(info)))
         self.info = info
         self.V, self.M = info.V, info.M
+
+    def set_accept_bias(self, bias: float):
+        """``pcg_groups_set_accept_bias``: constant added to the acceptance ratio of later ``pcg_verify`` calls."""
+        _check(load().pcg_groups_set_accept_bias(self.handle, float(bias)))
 
     def close(self):
         if getattr(self, "handle", None):

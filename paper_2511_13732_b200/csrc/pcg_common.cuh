@@ -1,6 +1,7 @@
 // Shared device helpers and the group handle of libpcg (sm_100a only).
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -52,12 +53,31 @@ struct pcg_groups {
     int64_t device_bytes;
     void *allocation;  // single device allocation holding every array
     size_t agg_smem_bytes;  // dynamic shared memory of the aggregation kernels
+    float accept_bias;      // constant added to the acceptance ratio (0 = PCG)
 };
 
 namespace pcg {
 
 void set_error(const char *fmt, ...);
 pcg_status cuda_fail(cudaError_t e, const char *what);
+
+inline bool valid_dtype(pcg_dtype d) { return d == PCG_F32 || d == PCG_BF16 || d == PCG_F16; }
+inline size_t dtype_bytes(pcg_dtype d) { return d == PCG_F32 ? 4 : 2; }
+
+// Runs `...` with LogitT bound to the element type of `dtype` (float, uint16_t for bfloat16 bit patterns, f16_t).
+#define PCG_DISPATCH_DTYPE(dtype, ...)        \
+    do {                                      \
+        if ((dtype) == PCG_F32) {             \
+            using LogitT = float;             \
+            __VA_ARGS__;                      \
+        } else if ((dtype) == PCG_BF16) {     \
+            using LogitT = uint16_t;          \
+            __VA_ARGS__;                      \
+        } else {                              \
+            using LogitT = pcg::f16_t;        \
+            __VA_ARGS__;                      \
+        }                                     \
+    } while (0)
 
 #ifdef __CUDACC__
 
@@ -88,6 +108,24 @@ struct Elem<uint16_t> {  // bfloat16 bit patterns: the upper half of a float
         v[5] = __uint_as_float(r.z & 0xffff0000u);
         v[6] = __uint_as_float(r.w << 16);
         v[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+};
+
+struct f16_t {  // IEEE binary16 bit pattern (a tag type: bfloat16 patterns travel as plain uint16_t)
+    uint16_t bits;
+};
+template <>
+struct Elem<f16_t> {
+    static constexpr int kPerVec = 8;
+    static __device__ __forceinline__ float widen(f16_t x) { return __half2float(__ushort_as_half(x.bits)); }
+    static __device__ __forceinline__ void unpack(const uint4 &r, float (&v)[8]) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+            v[2 * i] = f.x;
+            v[2 * i + 1] = f.y;
+        }
     }
 };
 

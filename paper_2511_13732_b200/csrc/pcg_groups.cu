@@ -323,6 +323,7 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     h->device_bytes = (int64_t)total;
     h->allocation = mem;
     h->agg_smem_bytes = agg_smem_bytes(SL, M, C);
+    h->accept_bias = 0.f;
     *out = h;
     return PCG_OK;
 }
@@ -348,5 +349,14 @@ extern "C" pcg_status pcg_groups_info(const pcg_groups *groups, pcg_groups_info_
     out->device = groups->device;
     out->has_weights = groups->dev.pair_w != nullptr;
     out->device_bytes = groups->device_bytes;
+    return PCG_OK;
+}
+
+extern "C" pcg_status pcg_groups_set_accept_bias(pcg_groups *groups, float bias) {
+    if (!groups || !std::isfinite(bias) || bias < 0.f) {
+        pcg::set_error("pcg_groups_set_accept_bias: null handle, or a bias that is negative or not finite");
+        return PCG_ERR_INVALID_ARG;
+    }
+    groups->accept_bias = bias;
     return PCG_OK;
 }

@@ -16,7 +16,7 @@ Arena layout(int32_t B, int32_t K, int32_t V, int32_t M, pcg_dtype dtype, uint32
         off = (off + bytes + 255) & ~(size_t)255;
         return at;
     };
-    const size_t esz = dtype == PCG_F32 ? 4 : 2;
+    const size_t esz = pcg::dtype_bytes(dtype);
     const size_t b = B > 0 ? B : 0, k = K > 0 ? K : 0, v = V > 0 ? V : 0;
     a.target_bytes = b * (k + 1) * v * esz;
     a.draft_bytes = b * k * v * esz;
@@ -56,8 +56,8 @@ extern "C" pcg_status pcg_verify_host(const void *target_logits, const void *dra
         set_error("pcg_verify_host: null group handle");
         return PCG_ERR_INVALID_ARG;
     }
-    if (dtype != PCG_F32 && dtype != PCG_BF16) {
-        set_error("pcg_verify_host: dtype must be PCG_F32 or PCG_BF16");
+    if (!valid_dtype(dtype)) {
+        set_error("pcg_verify_host: dtype must be PCG_F32, PCG_BF16 or PCG_F16");
         return PCG_ERR_INVALID_ARG;
     }
     if (B < 0 || K < 1) {

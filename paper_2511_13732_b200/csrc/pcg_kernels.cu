@@ -101,6 +101,7 @@ struct PositionArgs {
     const float *uniforms;   // [B, K+1, 2]
     int K;
     float s;                 // log2(e) / temperature
+    float bias;              // constant added to the acceptance ratio (0 for PCG)
     int32_t *accept;         // [B*K] 1 = accepted
     int32_t *labels;         // [B*K] group label of the draft token
     int32_t *posflags;       // [B*K]
@@ -267,7 +268,7 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
         }
         // acceptance u < min(1, P/Q) without a division: P = Sp/Zp, Q = Sq/Zq
         const float lhs = Sp * Zq, rhs = Sq * Zp;
-        const int acc = (lhs >= rhs) || (c_u1 * rhs < lhs);
+        const int acc = (lhs >= rhs) || (c_u1 * rhs < __fmaf_rn(a.bias, rhs, lhs));
         int flag = c_flag;
         if (!(Zp > 0.f) || !(Zq > 0.f) || isinf(Zp) || isinf(Zq) || isinf(rs_p) || isinf(rs_q))
             flag |= PCG_FLAG_NONFINITE;
@@ -1267,6 +1268,7 @@ struct DenseAcceptArgs {
     int B, K;
     const float *Pws;  // [B*(K+1), M]
     const float *Qws;  // [B*K, M]
+    float bias;        // constant added to the acceptance ratio (0 for PCG)
     int32_t *accept, *labels, *posflags;
 };
 
@@ -1285,7 +1287,7 @@ __global__ void dense_accept_kernel(DenseAcceptArgs a, GroupsDev G) {
     const int g = draw_label(G, r0, G.rev_ptr[x + 1] - r0, u[0]);
     const float P = a.Pws[((size_t)b * (a.K + 1) + i) * G.M + g], Q = a.Qws[(size_t)pos * G.M + g];
     if (isnan(P) || isnan(Q)) flag |= PCG_FLAG_NONFINITE;
-    a.accept[pos] = (P >= Q) || (u[1] * Q < P);
+    a.accept[pos] = (P >= Q) || (u[1] * Q < __fmaf_rn(a.bias, Q, P));
     a.labels[pos] = g;
     a.posflags[pos] = flag;
 }
@@ -1297,8 +1299,8 @@ static pcg_status check_common(const pcg_groups *groups, pcg_dtype dtype, float 
         set_error("%s: null group handle", who);
         return PCG_ERR_INVALID_ARG;
     }
-    if (dtype != PCG_F32 && dtype != PCG_BF16) {
-        set_error("%s: dtype must be PCG_F32 or PCG_BF16", who);
+    if (!valid_dtype(dtype)) {
+        set_error("%s: dtype must be PCG_F32, PCG_BF16 or PCG_F16", who);
         return PCG_ERR_INVALID_ARG;
     }
     if (!(temperature >= 1e-6f) || !std::isfinite(temperature)) {
@@ -1408,12 +1410,8 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
     }
     ProbsArgs a{logits, out, (float)((double)kLog2e / (double)temperature)};
     cudaError_t e;
-    if (dtype == PCG_F32)
-        e = launch_cluster(group_probs_kernel<float>, (int)(rows * G.slices), G.slices, groups->agg_smem_bytes,
-                           (cudaStream_t)stream, a, G);
-    else
-        e = launch_cluster(group_probs_kernel<uint16_t>, (int)(rows * G.slices), G.slices, groups->agg_smem_bytes,
-                           (cudaStream_t)stream, a, G);
+    PCG_DISPATCH_DTYPE(dtype, e = launch_cluster(group_probs_kernel<LogitT>, (int)(rows * G.slices), G.slices,
+                                                 groups->agg_smem_bytes, (cudaStream_t)stream, a, G));
     if (e != cudaSuccess) return cuda_fail(e, "launching group_probs_kernel");
     return PCG_OK;
 }
@@ -1452,7 +1450,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         return PCG_ERR_INVALID_ARG;
     }
     const GroupsDev &G = groups->dev;
-    const size_t esz = dtype == PCG_F32 ? 4 : 2;
+    const size_t esz = dtype_bytes(dtype);
     if (((uintptr_t)target_logits % esz) || ((uintptr_t)draft_logits % esz)) {
         set_error("pcg_verify: logits pointers must be aligned to their element size");
         return PCG_ERR_INVALID_ARG;
@@ -1491,16 +1489,14 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         pcg_status st2 = pcg_group_probs(target_logits, dtype, (int64_t)B * (K + 1), temperature, groups, w.Pws, stream);
         if (st2 == PCG_OK) st2 = pcg_group_probs(draft_logits, dtype, (int64_t)B * K, temperature, groups, w.Qws, stream);
         if (st2 != PCG_OK) return st2;
-        DenseAcceptArgs da{draft_tokens, uniforms, B, K, w.Pws, w.Qws, w.accept, w.labels, w.posflags};
+        DenseAcceptArgs da{draft_tokens, uniforms, B, K, w.Pws, w.Qws, groups->accept_bias, w.accept, w.labels, w.posflags};
         dense_accept_kernel<<<(B * K + 127) / 128, 128, 0, cs>>>(da, G);
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching dense_accept_kernel");
     } else {
-        PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, w.accept, w.labels, w.posflags, w.stats};
-        if (dtype == PCG_F32)
-            position_kernel<float><<<B * K, kPosThreads, 0, cs>>>(pa, G);
-        else
-            position_kernel<uint16_t><<<B * K, kPosThreads, 0, cs>>>(pa, G);
+        PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
+                        w.accept,      w.labels,     w.posflags,   w.stats};
+        PCG_DISPATCH_DTYPE(dtype, position_kernel<LogitT><<<B * K, kPosThreads, 0, cs>>>(pa, G));
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
     }
@@ -1513,22 +1509,17 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
     if (cluster_terminal) {
         TerminalArgs ta{target_logits, draft_logits, draft_tokens, uniforms,       K,          s,         w.accept,
                         w.labels,      w.posflags,   w.stats,      out_accept_len, out_tokens, out_groups, out_flags};
-        if (dtype == PCG_F32)
-            e = launch_cluster(terminal_kernel<float>, B * G.slices, G.slices, groups->agg_smem_bytes, cs, ta, G);
-        else
-            e = launch_cluster(terminal_kernel<uint16_t>, B * G.slices, G.slices, groups->agg_smem_bytes, cs, ta, G);
+        PCG_DISPATCH_DTYPE(dtype, e = launch_cluster(terminal_kernel<LogitT>, B * G.slices, G.slices,
+                                                     groups->agg_smem_bytes, cs, ta, G));
         if (e != cudaSuccess) return cuda_fail(e, "launching terminal_kernel");
     } else {
         PrepareArgs pr{target_logits, K, s, dense ? 0 : 1, w.accept, w.posflags, w.stats, w.term_n, w.term_flags, w.term_stats};
-        if (dtype == PCG_F32)
-            terminal_prepare_kernel<float><<<B, kPrepThreads, 0, cs>>>(pr, G);
-        else
-            terminal_prepare_kernel<uint16_t><<<B, kPrepThreads, 0, cs>>>(pr, G);
+        PCG_DISPATCH_DTYPE(dtype, terminal_prepare_kernel<LogitT><<<B, kPrepThreads, 0, cs>>>(pr, G));
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching terminal_prepare_kernel");
         if (!dense) {
             const int chunk = terminal_chunk(B, G.V);
-            const int tt = 32 * (dtype == PCG_F32 ? 4 : 8);
+            const int tt = 32 * (int)(16 / dtype_bytes(dtype));
             const bool wide = B >= 32 * kSpmmWide;  // several sequences per lane in the sparse product
             for (int b0 = 0; b0 < B; b0 += chunk) {
                 // blocks of 32 sequences in this chunk, rounded up to what one block of the sparse product reads
@@ -1536,10 +1527,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
                 const int nb = (std::min(B - b0, chunk) + unit - 1) / unit * (unit / 32);
                 TransposeArgs tr{target_logits, draft_logits, B, K, b0, chunk, s, w.term_n, w.term_stats, w.Dt};
                 const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
-                if (dtype == PCG_F32)
-                    residual_transpose_kernel<float><<<tgrid, kTrThreads, 0, cs>>>(tr, G);
-                else
-                    residual_transpose_kernel<uint16_t><<<tgrid, kTrThreads, 0, cs>>>(tr, G);
+                PCG_DISPATCH_DTYPE(dtype, residual_transpose_kernel<LogitT><<<tgrid, kTrThreads, 0, cs>>>(tr, G));
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
                 SpmmArgs sp{w.Dt, B, b0, chunk, w.R};
@@ -1573,11 +1561,8 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
             kern<<<B, kDrawThreads, draw_smem, cs>>>(dr, G);
             return cudaGetLastError();
         };
-        if (dtype == PCG_F32)
-            e = dense ? launch_draw(terminal_draw_kernel<float, true>) : launch_draw(terminal_draw_kernel<float, false>);
-        else
-            e = dense ? launch_draw(terminal_draw_kernel<uint16_t, true>)
-                      : launch_draw(terminal_draw_kernel<uint16_t, false>);
+        PCG_DISPATCH_DTYPE(dtype, e = dense ? launch_draw(terminal_draw_kernel<LogitT, true>)
+                                            : launch_draw(terminal_draw_kernel<LogitT, false>));
         if (e != cudaSuccess) return cuda_fail(e, "launching terminal_draw_kernel");
     }
     if (stage_events) {

@@ -11,7 +11,7 @@ is not available offline; these generators stand in for it with the same shapes
 
 Everything is a pure function of (config name, sequence index): sequence ``b``
 of a config can be regenerated alone, which is what the full-size parity checks
-do.  bf16 logits are returned as uint16 bit patterns.
+do.  bf16 logits are returned as uint16 bit patterns, fp16 logits as numpy float16.
 """
 from __future__ import annotations
 
@@ -33,7 +33,7 @@ class Config:
     K: int
     V: int
     M: int
-    dtype: str  # "f32" | "bf16"
+    dtype: str  # "f32" | "bf16" | "f16"
     temperature: float
     logits: str  # recipe name
     groups: str  # recipe name
@@ -274,6 +274,9 @@ def make_sequence(cfg: Config, b: int):
     if cfg.dtype == "bf16":
         tgt_s, drf_s = f32_to_bf16_bits(tgt), f32_to_bf16_bits(drf)
         drf_val = bf16_bits_to_f32(drf_s)
+    elif cfg.dtype == "f16":
+        tgt_s, drf_s = tgt.astype(np.float16), drf.astype(np.float16)
+        drf_val = drf_s.astype(np.float32)
     else:
         tgt_s, drf_s, drf_val = tgt, drf, drf
     # drafted tokens follow the draft distribution at the call's temperature; drawn with
@@ -289,7 +292,7 @@ def make_batch(cfg: Config, B: Optional[int] = None, seqs: Optional[Sequence[int
     if seqs is None:
         seqs = range(cfg.B if B is None else B)
     seqs = list(seqs)
-    dt = np.uint16 if cfg.dtype == "bf16" else np.float32
+    dt = {"bf16": np.uint16, "f16": np.float16}.get(cfg.dtype, np.float32)
     n = len(seqs)
     tl = np.empty((n, cfg.K + 1, cfg.V), dt)
     dl = np.empty((n, cfg.K, cfg.V), dt)

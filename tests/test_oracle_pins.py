@@ -46,6 +46,22 @@ def test_softmax_bf16_bits_are_widened_exactly(oracle):
     np.testing.assert_allclose(oracle.softmax(bits, 1.0), want, rtol=1e-13)
 
 
+def test_softmax_fp16_values_are_widened_exactly(oracle):
+    rng = np.random.default_rng(21)
+    x = (4.0 * rng.standard_normal((3, 80))).astype(np.float16)
+    x[0, :4] = np.array([6.0e-8, -6.0e-5, 65504.0, -np.inf], np.float16)  # subnormal, small normal, largest, mask
+    x[0, 2] = np.float16(11.0)
+    want = scipy_softmax(x.astype(np.float64), axis=1)
+    np.testing.assert_allclose(oracle.softmax(x, 1.0), want, rtol=1e-13)
+    # every finite binary16 pattern widens to the value numpy assigns to it (checked through a two-token softmax)
+    bits = np.arange(0, 0x7C00, 37, dtype=np.uint16)
+    vals = bits.view(np.float16)
+    pair = np.stack([vals / np.float16(1.0), np.zeros_like(vals)], axis=1).astype(np.float16)
+    got = oracle.softmax(pair[pair[:, 0] < 30], 1.0)
+    v64 = pair[pair[:, 0] < 30][:, 0].astype(np.float64)
+    np.testing.assert_allclose(got[:, 0], 1.0 / (1.0 + np.exp(-v64)), rtol=1e-13)
+
+
 def test_softmax_handles_masked_tokens(oracle):
     x = np.array([[0.0, -np.inf, 1.0, -np.inf]], np.float32)
     p = oracle.softmax(x, 1.0)

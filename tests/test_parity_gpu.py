@@ -139,6 +139,42 @@ def test_verify_extreme_k(oracle, K, mode):
 
 
 @pytest.mark.parametrize("mode", MODES)
+def test_verify_with_constant_acceptance_bias(oracle, mode):
+    """The lossy relaxation the paper compares against (a constant added to the acceptance ratio, Sec. 3.2)."""
+    cfg = W.scaled(W.CONFIGS["C3"], B=48, K=6, V=5000, M=1200)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    plain = run_oracle(oracle, bt, groups)
+    biased = oracle.verify(bt.target_logits, bt.draft_logits, bt.draft_tokens, groups.group_ptr, groups.group_tok,
+                           groups.tok_degree, bt.uniforms, bt.temperature, accept_bias=float(np.float32(0.3)), threads=0)
+    assert biased.accept_len.sum() > plain.accept_len.sum()  # the bias does accept more
+    h = make_handle(groups)
+    h.set_accept_bias(0.3)
+    _assert_parity(run_verify(bt, h, mode=mode), biased)
+    h.set_accept_bias(0.0)
+    _assert_parity(run_verify(bt, h, mode=mode), plain)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_verify_fp16_logits(oracle, mode):
+    """IEEE binary16 logits (the third element type) through every mode, plus pcg_group_probs."""
+    cfg = W.scaled(W.CONFIGS["C3"], B=40, K=5, V=6000, M=1500, dtype="f16")
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    assert bt.target_logits.dtype == np.float16
+    ref = run_oracle(oracle, bt, groups)
+    h = make_handle(groups)
+    _assert_parity(run_verify(bt, h, mode=mode), ref)
+    if mode == 0:
+        from paper_2511_13732_b200 import binding
+
+        x = bt.draft_logits.reshape(-1, cfg.V)[:9]
+        want = oracle.group_probs(x, groups.group_ptr, groups.group_tok, groups.tok_degree, cfg.temperature)
+        got = binding.pcg_group_probs(logits_to_device(x), h, cfg.temperature).cpu().numpy()
+        np.testing.assert_allclose(got, want, rtol=1e-5, atol=1e-37)
+
+
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_verify_general_split_weights(oracle, dtype, mode):
     """General weights w_{k,t} (non-negative, summing to one over the groups of each token) in place of the equal
