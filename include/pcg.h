@@ -186,9 +186,9 @@ size_t pcg_verify_workspace_bytes(int32_t B, int32_t K, int32_t V, int32_t M, pc
  *              calls that share a workspace must not overlap on the device
  *   stage_events: NULL, or 3 events recorded on `stream` before the position kernel, between it and the
  *              terminal kernel, and after the terminal kernel (for timing the stages)
- * Results are bit-identical from run to run.  1 <= K <= 32, B >= 0 (B == 0 is a no-op).
+ * Results are bit-identical from run to run.  1 <= K <= 1024, B >= 0 (B == 0 is a no-op).
  * Masses below the float32 normal range flush to zero.
- * Errors: INVALID_ARG, UNSUPPORTED (K > 32), WORKSPACE, CUDA.
+ * Errors: INVALID_ARG, UNSUPPORTED (K > 1024), WORKSPACE, CUDA.
  */
 pcg_status pcg_verify(const void *target_logits, const void *draft_logits, pcg_dtype dtype, int32_t B, int32_t K,
                       const int32_t *draft_tokens, const pcg_groups *groups, const float *uniforms, float temperature,

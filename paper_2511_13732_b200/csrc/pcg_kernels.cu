@@ -466,13 +466,21 @@ __global__ void __launch_bounds__(kAggThreads, 2) terminal_kernel(TerminalArgs a
     const int b = blockIdx.x / C;
     const int tid = threadIdx.x;
 
-    // ---- first rejected position: one ballot over the K <= 32 accept bits ----
+    // ---- first rejected position: warp ballots over the accept bits, 32 positions at a time ----
     if (tid < 32) {
-        const int rej = (tid < K) && (a.accept[b * K + tid] == 0);
-        const unsigned mask = __ballot_sync(0xffffffffu, rej);
-        const int n = mask ? (__ffs(mask) - 1) : K;
-        const int f = (tid < K && tid <= n) ? a.posflags[b * K + tid] : 0;
-        const int flags = __reduce_or_sync(0xffffffffu, f);
+        // 32 accept bits per ballot; the first word with a rejection ends the search
+        int n = K, flags = 0;
+        for (int base = 0; base < K && n == K; base += 32) {
+            const int i = base + tid;
+            const int rej = (i < K) && (a.accept[b * K + i] == 0);
+            const unsigned mask = __ballot_sync(0xffffffffu, rej);
+            if (mask) n = base + __ffs(mask) - 1;
+        }
+        for (int base = 0; base < K && base <= n; base += 32) {
+            const int i = base + tid;
+            const int f = (i < K && i <= n) ? a.posflags[b * K + i] : 0;
+            flags |= __reduce_or_sync(0xffffffffu, f);
+        }
         if (tid == 0) {
             sm.ibox[0] = n;
             sm.ibox[1] = flags;
@@ -668,18 +676,18 @@ __global__ void __launch_bounds__(kAggThreads, 2) terminal_kernel(TerminalArgs a
             }
         }
         // ---- emit: accepted draft tokens, the drawn token, then filler ----
-        if (tid <= K) {
+        for (int i = tid; i <= K; i += NT) {
             int tok = -1, grp = -1;
-            if (tid < n) {
-                tok = a.draft_tokens[b * K + tid];
+            if (i < n) {
+                tok = a.draft_tokens[b * K + i];
                 if (tok < 0 || tok >= V) tok = 0;  // verified as token 0 (and flagged), so emitted as token 0
-                grp = a.labels[b * K + tid];
-            } else if (tid == n) {
+                grp = a.labels[b * K + i];
+            } else if (i == n) {
                 tok = z;
                 grp = gsel;
             }
-            a.out_tokens[(int64_t)b * (K + 1) + tid] = tok;
-            if (a.out_groups) a.out_groups[(int64_t)b * (K + 1) + tid] = grp;
+            a.out_tokens[(int64_t)b * (K + 1) + i] = tok;
+            if (a.out_groups) a.out_groups[(int64_t)b * (K + 1) + i] = grp;
         }
         if (tid == 0) {
             a.out_accept_len[b] = n;
@@ -743,13 +751,21 @@ __global__ void __launch_bounds__(kPrepThreads) terminal_prepare_kernel(PrepareA
     __shared__ int s_n, s_flags;
     __shared__ float red[2 * NW];
     const int b = blockIdx.x, tid = threadIdx.x, K = a.K, V = G.V;
-    // ---- first rejected position: one ballot over the K <= 32 accept bits ----
+    // ---- first rejected position: warp ballots over the accept bits, 32 positions at a time ----
     if (tid < 32) {
-        const int rej = (tid < K) && (a.accept[b * K + tid] == 0);
-        const unsigned mask = __ballot_sync(0xffffffffu, rej);
-        const int n = mask ? (__ffs(mask) - 1) : K;
-        const int f = (tid < K && tid <= n) ? a.posflags[b * K + tid] : 0;
-        const int flags = __reduce_or_sync(0xffffffffu, f);
+        // 32 accept bits per ballot; the first word with a rejection ends the search
+        int n = K, flags = 0;
+        for (int base = 0; base < K && n == K; base += 32) {
+            const int i = base + tid;
+            const int rej = (i < K) && (a.accept[b * K + i] == 0);
+            const unsigned mask = __ballot_sync(0xffffffffu, rej);
+            if (mask) n = base + __ffs(mask) - 1;
+        }
+        for (int base = 0; base < K && base <= n; base += 32) {
+            const int i = base + tid;
+            const int f = (i < K && i <= n) ? a.posflags[b * K + i] : 0;
+            flags |= __reduce_or_sync(0xffffffffu, f);
+        }
         if (tid == 0) {
             s_n = n;
             s_flags = flags;
@@ -1242,18 +1258,18 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
         }
     }
     // ---- emit: accepted draft tokens, the drawn token, then filler ----
-    if (tid <= K) {
+    for (int i = tid; i <= K; i += NT) {
         int tok = -1, grp = -1;
-        if (tid < n) {
-            tok = a.draft_tokens[b * K + tid];
+        if (i < n) {
+            tok = a.draft_tokens[b * K + i];
             if (tok < 0 || tok >= V) tok = 0;  // verified as token 0 (and flagged), so emitted as token 0
-            grp = a.labels[b * K + tid];
-        } else if (tid == n) {
+            grp = a.labels[b * K + i];
+        } else if (i == n) {
             tok = z;
             grp = gsel;
         }
-        a.out_tokens[(int64_t)b * (K + 1) + tid] = tok;
-        if (a.out_groups) a.out_groups[(int64_t)b * (K + 1) + tid] = grp;
+        a.out_tokens[(int64_t)b * (K + 1) + i] = tok;
+        if (a.out_groups) a.out_groups[(int64_t)b * (K + 1) + i] = grp;
     }
     if (tid == 0) {
         a.out_accept_len[b] = n;
@@ -1435,8 +1451,8 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         set_error("pcg_verify: need B >= 0 and K >= 1 (B=%d K=%d)", B, K);
         return PCG_ERR_INVALID_ARG;
     }
-    if (K > 32) {
-        set_error("pcg_verify: K=%d exceeds the 32 positions one ballot covers", K);
+    if (K > 1024) {
+        set_error("pcg_verify: K=%d exceeds the supported 1024 drafted positions per sequence", K);
         return PCG_ERR_UNSUPPORTED;
     }
     if (mode != PCG_VERIFY_DEFAULT && mode != PCG_VERIFY_DENSE && mode != PCG_VERIFY_CLUSTER_TERMINAL &&
