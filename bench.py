@@ -331,6 +331,39 @@ def main():
             other_modes[name] = {"ms_per_step": m0.elapsed_time(m1) / reps, "steps": reps,
                                  "outputs_equal_to_timed_mode": bool(same)}
             del ws_m
+
+    # the other two entry points of the boundary, briefly: pcg_group_probs on a slice of the target rows, and the
+    # one-time group construction on a seeded clustered table of the workload's vocabulary size
+    extras = {}
+    if world == 1 and not args.no_other_modes:
+        rows = min(B * (K + 1), 1024)
+        x_rows = tl.reshape(-1, V)[:rows]
+        P = binding.pcg_group_probs(x_rows, handle, cfg.temperature)
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(5):
+            binding.pcg_group_probs(x_rows, handle, cfg.temperature, out=P)
+        g1.record()
+        torch.cuda.synchronize()
+        gp_ms = g0.elapsed_time(g1) / 5
+        extras["group_probs"] = {"rows": rows, "ms": gp_ms, "rows_per_s": rows / (gp_ms * 1e-3),
+                                 "counted_gbs": rows * (V * esz + M * 4) / (gp_ms * 1e-3) / 1e9,
+                                 "row_sum_max_error": float((P.sum(dim=1) - 1).abs().max())}
+        d_emb = 512 if V >= 32768 else 128
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(2511)
+        centres = torch.randn((max(1, V // 24), d_emb), device="cuda", generator=gen)
+        which = torch.randint(0, max(1, V // 24), (V,), device="cuda", generator=gen)
+        table = (centres[which] + 0.35 * torch.randn((V, d_emb), device="cuda", generator=gen)).to(torch.bfloat16)
+        for flag, key in ((False, "tcgen05"), (True, "mma_sync")):
+            asg = binding.Asg(table, 0.42, mma_sync=flag)
+            asg.close()
+            asg = binding.Asg(table, 0.42, mma_sync=flag)
+            extras.setdefault("group_construction", {"V": V, "d": d_emb, "theta": 0.42})[key] = {
+                "similarity_ms": asg.info.similarity_ms, "total_ms": asg.info.total_ms, "groups": asg.info.M,
+                "tflops": 2.0 * V * V * d_emb / (asg.info.similarity_ms * 1e-3) / 1e12}
+            asg.close()
+        del table, centres, which
     if rank == 0:
         peak, peak_src = hbm_peak()
         alg_bytes = B * K * 2 * V * esz  # per drafted position: one target and one draft row, read once
@@ -352,6 +385,7 @@ def main():
             "mode": args.mode + (" (per-sequence stage: " + ("cluster" if default_is_cluster else "batched") + ")"
                                  if args.mode == "default" else ""),
             "other_modes": other_modes,
+            "other_entry_points": extras,
             "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
                     "api": "pcg_verify_host (pinned host tensors)"},
