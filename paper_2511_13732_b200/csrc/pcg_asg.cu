@@ -12,8 +12,10 @@
 //                           a full comparison of the two bit rows
 //   scans, asg_fill_kernel  group numbers by ascending representative, group_ptr, token lists from the bit rows,
 //                           token degrees by counting
+#include <cuda.h>  // CUtensorMap and its enums only; the encoder is fetched through the runtime, not linked
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <cmath>
 #include <new>
 #include <vector>
@@ -185,36 +187,43 @@ __global__ void __launch_bounds__(kAsgThreads) asg_similarity_kernel(const __nv_
 
 
 // ---------------------------------------------------------------------------------------------- similarity, tcgen05
-// 256 x 256 tiles on the 5th-generation tensor cores: one thread issues tcgen05.mma (M = 128, N = 256, K = 16 per
-// instruction, two instructions per K step for the two 128-row halves of the tile) on operands staged in shared
-// memory; the two 128 x 256 fp32 accumulators fill the SM's tensor memory (128 lanes x 512 columns) and are read
-// back with tcgen05.ld, one accumulator row per thread, which is exactly the row of 256 decisions (eight 32-bit
-// words) that thread then writes.  The large tile is what keeps the operand traffic from L2 (128 flop per byte)
-// below the tensor cores' appetite; a 128 x 128 tile (64 flop per byte) is L2-bound.
+// Persistent, warp-specialised tiles on the 5th-generation tensor cores.  One block per SM walks the 128 x 256
+// tiles of E * E^T; its warps have fixed roles that meet only through mbarriers:
+//   warps 0-7  epilogue: read a finished 128 x 256 fp32 accumulator from tensor memory (tcgen05.ld, a warp may
+//              touch the 32 lanes given by its index modulo 4; thread = accumulator row), turn it into 256
+//              decisions cos > theta and write them as eight 32-bit words
+//   warp 8     producer: one thread fetches the operands of the next K step (64 bf16 per row: a 128-row box of A and
+//              two 128-row boxes of B) with TMA (cp.async.bulk.tensor, 128-byte swizzle) into a ring of stages; the
+//              copies complete the stage's "full" barrier by byte count (expect_tx / complete_tx)
+//   warp 9     one thread issues tcgen05.mma (M = 128, N = 256, K = 16, four per stage), hands each stage back to
+//              the producers with tcgen05.commit on its "empty" barrier, and commits the tile's last K step on the
+//              accumulator's "full" barrier
+// The two 128 x 256 accumulators fill the SM's 512 columns of tensor memory, so the epilogue of one tile runs
+// under the MMAs of the next.
 //
-// Shared-memory operand layout (K-major, no swizzle): 8 rows x 16 bytes form a 128-byte core matrix; core
-// matrices that are neighbours along K sit 128 bytes apart (leading byte offset), groups of 8 rows 1024 bytes
-// apart (stride byte offset).  With 64 bf16 (8 chunks of 16 bytes) per row and stage, chunk (row, c) lands at
-// byte (row/8)*1024 + c*128 + (row%8)*16, which makes the cp.async destinations of consecutive threads contiguous.
-// Every wait on an mbarrier is bounded: on a time-out the block records an error code, drains its own copies,
-// frees its tensor memory and returns.
-constexpr int kTcBK = 64;       // bf16 per row and stage
-#ifndef PCG_TC_HALVES
-#define PCG_TC_HALVES 2  // 128-row accumulators per block: 2 = 256 x 256 tiles, one block per SM (measured best); 1 = 128 x 256
-#endif
+// Shared-memory operand layout: the canonical K-major 128-byte-swizzle layout that TMA writes -- row r of a box at
+// byte r * 128, its eight 16-byte chunks XOR-permuted by r % 8; groups of 8 rows are 1024 bytes apart (the
+// descriptor's stride byte offset), every stage starts on a 1024-byte boundary, and a K step of 16 bf16 advances
+// the descriptor's start address by 32 bytes inside the swizzled row.
+// Every wait on an mbarrier is a bounded poll that also watches a block-wide failure flag: on a time-out the
+// waiting role raises the flag, every role leaves its loop, the block drains its copies, frees its tensor memory,
+// records an error code and returns.
+constexpr int kTcBK = 64;        // bf16 per row and stage
+constexpr int kTcTile = 256;     // columns of a tile (rows of the B operand); Vp is a multiple of it
+constexpr int kTcRows = 128;     // rows of a tile (rows of the A operand) = lanes of tensor memory
 #ifndef PCG_TC_STAGES
-#define PCG_TC_STAGES 3
+#define PCG_TC_STAGES 4
 #endif
-constexpr int kTcHalves = PCG_TC_HALVES;
-constexpr int kTcStages = PCG_TC_STAGES;  // operand stages in shared memory
-constexpr int kTcThreads = 128 * kTcHalves;
-constexpr int kTcTile = 256;              // columns of a tile (rows of the B operand); Vp is a multiple of it
-constexpr int kTcRows = 128 * kTcHalves;  // rows of a tile (rows of the A operand)
+constexpr int kTcStages = PCG_TC_STAGES;
+constexpr int kTcEpilogueWarps = 8, kTcProducerWarps = 1;
+constexpr int kTcRasterRows = 16, kTcRasterCols = 8;  // tiles are visited in blocks of 16 x 8 (see tile_origin)
+constexpr int kTcThreads = 32 * (kTcEpilogueWarps + kTcProducerWarps + 1);
 constexpr int kTcABytes = kTcRows * kTcBK * 2, kTcBBytes = kTcTile * kTcBK * 2;
 constexpr int kTcStageBytes = kTcABytes + kTcBBytes;
 constexpr uint32_t kTcSpinLimit = 1u << 22;  // polls of about 50 ns each: gives up after a fraction of a second
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+// false = gave up (time-out, or another role raised the failure flag)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *failed) {
     for (uint32_t i = 0; i < kTcSpinLimit; ++i) {
         uint32_t done;
         asm volatile(
@@ -223,166 +232,209 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
             : "r"(bar), "r"(parity)
             : "memory");
         if (done) return true;
-        __nanosleep(32);
+        if (*failed) return false;
+        __nanosleep(20);
     }
+    *failed = 1;
     return false;
 }
-__device__ __forceinline__ uint64_t umma_desc_kmajor_noswizzle(uint32_t smem_addr) {
-    // start address >> 4 | leading byte offset (128) >> 4 at bit 16 | stride byte offset (1024) >> 4 at bit 32 |
-    // descriptor version 1 at bit 46; layout type 0 (no swizzle), base offset 0
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           (1ull << 46);
+__device__ __forceinline__ uint64_t umma_desc_kmajor_sw128(uint32_t smem_addr) {
+    // start address >> 4 | leading byte offset field 1 (not used by swizzled K-major layouts) at bit 16 |
+    // stride byte offset (1024: one group of 8 rows) >> 4 at bit 32 | descriptor version 1 at bit 46 |
+    // layout type 2 (128-byte swizzle) at bit 61
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
 }
 // kind::f16 instruction descriptor: D = fp32 (1 << 4), A = B = bf16 (1 << 7, 1 << 10), both K-major,
 // N = 256 (256 >> 3 at bit 17), M = 128 (128 >> 4 at bit 24)
 constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
 
-__global__ void __launch_bounds__(kTcThreads) asg_similarity_tc_kernel(const __nv_bfloat16 *E, const float *rnorm,
-                                                                      int V, int dp, float theta, int W,
-                                                                      uint32_t *bits, int *error) {
-    constexpr int T = kTcTile, BK = kTcBK, S = kTcStages;
-    extern __shared__ __align__(128) unsigned char tc_smem[];  // [S][A | B][256 rows x 128 bytes]
-    __shared__ __align__(8) uint64_t mbar[S + 1];              // stage s: its MMAs have finished; [S]: accumulator ready
+__global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const __grid_constant__ CUtensorMap tmap,
+                                                                         const float *rnorm, int V, int Vp, int dp,
+                                                                         float theta, int W, uint32_t *bits,
+                                                                         int *error) {
+    constexpr int S = kTcStages, BK = kTcBK;
+    extern __shared__ unsigned char tc_smem_raw[];  // [S][A 128 rows | B 256 rows][128 bytes per row], 1024-aligned below
+    __shared__ __align__(8) uint64_t bars[2 * S + 4];          // full[S], empty[S], acc_full[2], acc_empty[2]
     __shared__ uint32_t tmem_slot;
-    __shared__ float rnj[T];
-    __shared__ int failed;
+    __shared__ int failed_flag;
+    volatile int *failed = &failed_flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int i0 = blockIdx.y * kTcRows, j0 = blockIdx.x * T;
-    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(tc_smem);
-    const uint32_t bar_base = (uint32_t)__cvta_generic_to_shared(mbar);
+    const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(tc_smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar0 = (uint32_t)__cvta_generic_to_shared(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
+    auto acc_full_bar = [&](int b) { return bar0 + 8u * (2 * S + b); };
+    auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * S + 2 + b); };
     if (tid == 0) {
-        for (int s = 0; s <= S; ++s) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_base + 8 * s));
+        for (int s = 0; s < S; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_bar(s)));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(empty_bar(s)));
+        }
+        for (int b = 0; b < 2; ++b) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(acc_full_bar(b)));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(acc_empty_bar(b)), "r"(32 * kTcEpilogueWarps));
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        failed = 0;
+        failed_flag = 0;
     }
-    for (int c = tid; c < T; c += kTcThreads) rnj[c] = rnorm[j0 + c];
-    if (warp == 0) {  // tensor memory: 256 columns per 128 x 256 accumulator, allocated and freed by warp 0
+    if (warp == 0) {  // tensor memory: all 512 columns (two 128 x 256 accumulators), allocated and freed by warp 0
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                          (uint32_t)__cvta_generic_to_shared(&tmem_slot)),
-                     "r"(256 * kTcHalves));
+                     "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = tmem_slot;
-
-    auto load_stage = [&](int s, int k0) {
-        // per operand 256 rows x 8 chunks; thread handles chunks idx = tid + 256 i: row = (idx/64)*8 + idx%8,
-        // chunk = (idx/8)%8, destination byte idx*16 (see the layout above)
-        unsigned char *a = tc_smem + (size_t)s * kTcStageBytes, *b = a + kTcABytes;
-#pragma unroll
-        for (int i = 0; i < kTcRows * 8 / kTcThreads; ++i) {
-            const int idx = tid + i * kTcThreads, row = (idx >> 6) * 8 + (idx & 7), c = (idx >> 3) & 7;
-            asg_cp_async16(a + idx * 16, E + (size_t)(i0 + row) * dp + k0 + c * 8);
-        }
-#pragma unroll
-        for (int i = 0; i < T * 8 / kTcThreads; ++i) {
-            const int idx = tid + i * kTcThreads, row = (idx >> 6) * 8 + (idx & 7), c = (idx >> 3) & 7;
-            asg_cp_async16(b + idx * 16, E + (size_t)(j0 + row) * dp + k0 + c * 8);
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
+    const int nI = Vp / kTcRows, nJ = Vp / kTcTile, nk = dp / BK;
+    // Tile numbers run through blocks of 16 row blocks x 8 column blocks (128 tiles, about one wave of the
+    // persistent grid), so the tiles in flight at any time share 4096 rows of E (4 MB at d = 512) and the operands
+    // come out of L2 rather than HBM; numbers that fall outside the matrix are skipped by every role alike.
+    const int sbI = (nI + kTcRasterRows - 1) / kTcRasterRows, sbJ = (nJ + kTcRasterCols - 1) / kTcRasterCols;
+    const int ntiles = sbI * sbJ * kTcRasterRows * kTcRasterCols;
+    auto tile_origin = [&](int tile, int &i0, int &j0) -> bool {
+        const int sb = tile / (kTcRasterRows * kTcRasterCols), local = tile % (kTcRasterRows * kTcRasterCols);
+        const int ti = (sb / sbJ) * kTcRasterRows + local % kTcRasterRows;
+        const int tj = (sb % sbJ) * kTcRasterCols + local / kTcRasterRows;
+        i0 = ti * kTcRows;
+        j0 = tj * kTcTile;
+        return ti < nI && tj < nJ;
     };
-    const int nk = dp / BK;
-    bool ok = true;
-    // tiles 0 .. S-2 in flight before the loop; inside, tile kt + S - 1 is fetched once the MMAs of tile kt - 1
-    // (same stage) have finished
+
+    if (warp < kTcEpilogueWarps) {
+        // ------------------------------------------------------------------ epilogue warps
+        // warps 0-3 take columns 0-127 of the accumulator, warps 4-7 columns 128-255; a warp may only touch the 32
+        // lanes of tensor memory given by its index modulo 4.  Thread = accumulator row, 128 decisions = 4 words.
+        const int quarter = warp & 3, chalf = warp >> 2;
+        int tcount = 0;
+        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+            int i0, j0;
+            if (!tile_origin(tile, i0, j0)) continue;
+            const int buf = tcount & 1;
+            const int r = quarter * 32 + lane, c0 = chalf * 128;
+            const float rni = rnorm[i0 + r];
+            float rnq[4];  // 1/|column| of columns c0 + 32 q + lane, handed round by shuffle below
 #pragma unroll
-    for (int p = 0; p < S - 1; ++p) {
-        if (p < nk) load_stage(p, p * BK);
-        else asm volatile("cp.async.commit_group;" ::: "memory");
-    }
-    for (int kt = 0; kt < nk; ++kt) {
-        const int nxt = kt + S - 1;
-        if (nxt < nk) {
-            if (kt >= 1) ok = ok && mbar_wait_bounded(bar_base + 8 * ((kt - 1) % S), ((kt - 1) / S) & 1);
-            if (ok) load_stage(nxt % S, nxt * BK);
-            else asm volatile("cp.async.commit_group;" ::: "memory");
-        } else {
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        }
-        asm volatile("cp.async.wait_group %0;" ::"n"(S - 1) : "memory");  // this thread's part of tile kt has landed
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // ... and is visible to the tensor core
-        if (!ok) failed = 1;
-        __syncthreads();
-        if (failed) break;
-        if (tid == 0) {
+            for (int q = 0; q < 4; ++q) rnq[q] = rnorm[j0 + c0 + q * 32 + lane];
+            const bool ready = mbar_wait_bounded(acc_full_bar(buf), (tcount >> 1) & 1, failed);
+            if (!__all_sync(0xffffffffu, ready)) break;  // warp-uniform: tcgen05.ld below needs the whole warp
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a = smem_base + (uint32_t)((kt % S) * kTcStageBytes), b = a + kTcABytes;
+            uint32_t words[4];
 #pragma unroll
-            for (int kk = 0; kk < BK / 16; ++kk) {
-                const uint64_t db = umma_desc_kmajor_noswizzle(b + kk * 256);
-                const uint32_t accumulate = (kt > 0 || kk > 0) ? 1u : 0u;
+            for (int q = 0; q < 4; ++q) {
+                uint32_t v[32];
+                const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 256 + c0 + q * 32);
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, "
+                    "%14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                      "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),
+                      "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),
+                      "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),
+                      "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                    : "r"(taddr));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                uint32_t word = 0;
 #pragma unroll
-                for (int half = 0; half < kTcHalves; ++half) {  // rows 0-127 -> columns 0-255 of tensor memory, rows 128-255 -> 256-511
-                    const uint64_t da = umma_desc_kmajor_noswizzle(a + half * (128 * 128) + kk * 256);
+                for (int c = 0; c < 32; ++c) {
+                    const float rnc = __shfl_sync(0xffffffffu, rnq[q], c);
+                    const float cosv = __fmul_rn(__fmul_rn(__uint_as_float(v[c]), rni), rnc);
+                    word |= (cosv > theta ? 1u : 0u) << c;
+                }
+                // t is always a member of G(t); columns past the end of the vocabulary are never members
+                const int first = j0 + c0 + q * 32, diag = i0 + r - first;
+                if (diag >= 0 && diag < 32) word |= 1u << diag;
+                const int valid = V - first;
+                if (valid < 32) word = valid <= 0 ? 0u : (word & ((1u << valid) - 1u));
+                words[q] = word;
+            }
+            // the accumulator may be overwritten: hand it back to the MMA warp before the stores
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty_bar(buf)) : "memory");
+            if (i0 + r < V)
+                *reinterpret_cast<uint4 *>(bits + (size_t)(i0 + r) * W + ((j0 + c0) >> 5)) =
+                    make_uint4(words[0], words[1], words[2], words[3]);
+            ++tcount;
+        }
+    } else if (warp < kTcEpilogueWarps + kTcProducerWarps) {
+        // ------------------------------------------------------------------ producer (one thread)
+        if (lane == 0) {
+            const uint64_t map = reinterpret_cast<uint64_t>(&tmap);
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                int i0, j0;
+                if (!tile_origin(tile, i0, j0)) continue;
+                for (int kt = 0; kt < nk; ++kt, ++it) {
+                    const int s = it % S;
+                    if (it >= S && !mbar_wait_bounded(empty_bar(s), ((it / S) - 1) & 1, failed)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t a = smem_base + (uint32_t)(s * kTcStageBytes), b = a + kTcABytes, bar = full_bar(s);
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTcStageBytes)
+                                 : "memory");
+                    const int k0 = kt * BK;  // inner coordinate: a multiple of 64 elements = 128 bytes
+                    auto tma_box = [&](uint32_t dst, int row) {  // 128 rows x 64 bf16 of E starting at (row, k0)
+                        asm volatile(
+                            "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, "
+                            "%3}], [%4];" ::"r"(dst),
+                            "l"(map), "r"(k0), "r"(row), "r"(bar)
+                            : "memory");
+                    };
+                    tma_box(a, i0);
+                    tma_box(b, j0);
+                    tma_box(b + kTcABytes, j0 + 128);
+                }
+            }
+        }
+    } else if (warp == kTcEpilogueWarps + kTcProducerWarps && lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (one thread)
+        int it = 0, tcount = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+            int i0, j0;
+            if (!tile_origin(tile, i0, j0)) continue;
+            const int buf = tcount & 1;
+            if (tcount >= 2 && !mbar_wait_bounded(acc_empty_bar(buf), ((tcount >> 1) - 1) & 1, failed)) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            for (int kt = 0; kt < nk; ++kt, ++it) {
+                const int s = it % S;
+                if (!mbar_wait_bounded(full_bar(s), (it / S) & 1, failed)) {
+                    ok = false;
+                    break;
+                }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a = smem_base + (uint32_t)(s * kTcStageBytes), b = a + kTcABytes;
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; ++kk) {
+                    const uint64_t da = umma_desc_kmajor_sw128(a + kk * 32), db = umma_desc_kmajor_sw128(b + kk * 32);
+                    const uint32_t accumulate = (kt > 0 || kk > 0) ? 1u : 0u;
                     asm volatile(
                         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
                         :
-                        : "r"(tmem + half * 256), "l"(da), "l"(db), "r"(kTcIdesc), "r"(accumulate), "r"(0u), "r"(0u),
-                          "r"(0u), "r"(0u)
+                        : "r"(tmem + buf * 256), "l"(da), "l"(db), "r"(kTcIdesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u),
+                          "r"(0u)
                         : "memory");
                 }
-            }
-            // arrives on the stage's barrier when every MMA issued so far has finished reading shared memory
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                             bar_base + 8 * (kt % S))
-                         : "memory");
-            if (kt == nk - 1)
-                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                                 bar_base + 8 * S)
+                // arrives when every MMA issued so far has finished reading the stage: the producers may refill it
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(empty_bar(s))
                              : "memory");
-        }
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (!failed) {
-        if (!mbar_wait_bounded(bar_base + 8 * S, 0)) failed = 2;
-    }
-    __syncthreads();
-    if (!failed) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        // warps 0-3 read the first accumulator (tile rows 0-127), warps 4-7 the second; a warp may only touch the
-        // 32 lanes of tensor memory given by its index modulo 4.  Thread = one tile row: eight loads of 32 columns
-        // = eight words of decisions
-        const int half = warp >> 2, quarter = warp & 3;
-        const int r = half * 128 + quarter * 32 + lane;
-        const float rni = rnorm[i0 + r];
-        uint32_t words[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            uint32_t v[32];
-            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * 256 + q * 32);
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
-                "%15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                  "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-                  "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-                  "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                : "r"(taddr));
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            uint32_t word = 0;
-#pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                const int col = q * 32 + c;
-                const float cosv = __fmul_rn(__fmul_rn(__uint_as_float(v[c]), rni), rnj[col]);
-                const bool in = (j0 + col < V) && (cosv > theta || i0 + r == j0 + col);
-                word |= (in ? 1u : 0u) << c;
             }
-            words[q] = word;
+            if (ok)  // ... and when the tile's accumulator is complete
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                                 acc_full_bar(buf))
+                             : "memory");
+            ++tcount;
         }
-        if (i0 + r < V) {
-            uint4 *dst = reinterpret_cast<uint4 *>(bits + (size_t)(i0 + r) * W + (j0 >> 5));
-            dst[0] = make_uint4(words[0], words[1], words[2], words[3]);
-            dst[1] = make_uint4(words[4], words[5], words[6], words[7]);
-        }
-    } else if (tid == 0) {
-        atomicMax(error, failed);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256 * kTcHalves));
+    if (tid == 0 && failed_flag) atomicMax(error, 1);
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
 }
 
 // ---------------------------------------------------------------------------------------------- rows
@@ -618,14 +670,41 @@ extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V
     if (flags & PCG_ASG_MMA_SYNC) {
         asg_similarity_kernel<<<tiles, kAsgThreads>>>(E, rnorm, V, dp, theta, W, bits);
     } else {
-        const int smem = kTcStages * kTcStageBytes;
+        // TMA descriptor of E as a [Vp rows, dp columns] bf16 matrix, boxes of 128 rows x 64 columns, 128-byte swizzle
+        typedef CUresult (*EncodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                        const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                        CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres = cudaDriverEntryPointSymbolNotFound;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+            drop_events();
+            set_error("pcg_asg_create: the driver does not provide cuTensorMapEncodeTiled");
+            return PCG_ERR_CUDA;
+        }
+        alignas(64) CUtensorMap tmap;
+        const cuuint64_t gdim[2] = {(cuuint64_t)dp, (cuuint64_t)Vp}, gstride[1] = {(cuuint64_t)dp * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)kTcBK, 128u}, estride[2] = {1u, 1u};
+        const CUresult cr = ((EncodeTiled)fn)(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, E, gdim, gstride, box, estride,
+                                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (cr != CUDA_SUCCESS) {
+            drop_events();
+            set_error("pcg_asg_create: cuTensorMapEncodeTiled failed (%d)", (int)cr);
+            return PCG_ERR_CUDA;
+        }
+        const int smem = kTcStages * kTcStageBytes + 1024;  // room to start the stages on a 1024-byte boundary
         e = cudaFuncSetAttribute(asg_similarity_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) {
             drop_events();
             return cuda_fail(e, "cudaFuncSetAttribute (asg_similarity_tc_kernel)");
         }
-        asg_similarity_tc_kernel<<<dim3(Vp / kTcTile, Vp / kTcRows), kTcThreads, smem>>>(E, rnorm, V, dp, theta, W, bits,
-                                                                                        maxes + 2);
+        int dev = 0, sms = 1;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int ntiles = (Vp / kTcRows) * (Vp / kTcTile);
+        asg_similarity_tc_kernel<<<std::min(sms, std::max(1, ntiles)), kTcThreads, smem>>>(tmap, rnorm, V, Vp, dp, theta, W,
+                                                                                          bits, maxes + 2);
     }
     cudaEventRecord(ev[2], 0);
     {
