@@ -3,9 +3,9 @@
 //
 // Stages (all on the device):
 //   asg_prepare_kernel      rows to bfloat16 (zero-padded to a multiple of 32 columns and 128 rows), 1/|row| in fp32
-//   asg_similarity_kernel   E * E^T on the tensor cores, 128 x 128 tiles; the epilogue turns each dot product
-//                           into cos = dot * rn_i * rn_j, compares with theta and packs the decisions into a
-//                           V x V BIT matrix (the V x V similarities are never stored)
+//   asg_similarity_tc_kernel  E * E^T on the tensor cores (tcgen05, TMA; asg_similarity_kernel is the mma.sync form);
+//                           the epilogue turns each dot product into cos = dot * rn_i * rn_j, compares with theta
+//                           and packs the decisions into a V x V BIT matrix (the similarities are never stored)
 //   asg_row_kernel          per row: population count and a position-aware 64-bit hash of its bit row
 //   asg_representative_kernel  rep(t) = smallest t' with G(t') == G(t).  Such a t' is itself a member of G(t)
 //                           (t' is in G(t') = G(t)), so only the set bits below t are candidates: hash, then
