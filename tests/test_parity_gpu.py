@@ -88,6 +88,19 @@ def test_verify_c5_shape_small_batch(oracle, mode):
     _assert_parity(run_verify(bt, h, mode=mode), ref)
 
 
+@pytest.mark.parametrize("mode", MODES)
+def test_verify_c5_disjoint_groups_variant(oracle, mode):
+    """The disjoint-groups variant of the largest configuration (every token in exactly one of 16384 groups): PCG
+    then is standard speculative sampling on the lumped distributions (the oracle is pinned to a textbook
+    verifier for exactly this case on the CPU)."""
+    cfg = W.CONFIGS["C5d"]
+    groups = W.make_groups(cfg)
+    assert np.all(groups.tok_degree == 1) and groups.nnz == cfg.V
+    bt = W.make_batch(cfg, B=10)
+    ref = run_oracle(oracle, bt, groups)
+    _assert_parity(run_verify(bt, make_handle(groups), mode=mode), ref)
+
+
 def test_verify_batch_spanning_several_sequence_blocks(oracle):
     """The batched per-sequence stage handles 32 sequences per line: 70 sequences = two full blocks and a ragged one,
     with a group count that is not a multiple of the 32 groups a block of the sparse product owns."""
