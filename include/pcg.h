@@ -118,7 +118,8 @@ const char *pcg_last_error(void);
  * validates the CSR on the host, builds the reverse membership S(t) (ascending
  * group id -- the "optional reverse indices" of the same paragraph), the 1/N(t)
  * table and a token-sliced copy of the CSR with 16-bit in-slice token offsets,
- * uploads them and synchronises the device.
+ * uploads them and synchronises the device.  The handle also holds the scratch of pcg_group_probs
+ * (4 * V * min(256, ...) bytes: 64 MB at V = 65536).
  *
  *   slices_hint: 0 = choose automatically; 1, 2, 4 or 8 = force that many token
  *                slices (= cluster size).  Rounded up if a slice would not fit
@@ -153,6 +154,9 @@ pcg_status pcg_groups_set_accept_bias(pcg_groups *groups, float bias);
  *   logits  [rows, V] of `dtype`; base 16-byte aligned for the vector path
  *           (other alignments, or V*elemsize not a multiple of 16, use a slower scalar path)
  *   out     [rows, M] float32, fully overwritten
+ * From 64 rows on the rows go, up to 256 at a time, through scratch memory that belongs to the handle (a
+ * transposed copy of the rows' probabilities): two such calls with the SAME handle must not overlap on the device
+ * (different streams); pcg_verify in PCG_VERIFY_DENSE mode makes such calls too.
  * rows == 0 is a no-op.  Errors: INVALID_ARG (null, rows < 0, temperature <= 0 or not finite, bad dtype,
  * wrong device), CUDA (launch failure).
  */

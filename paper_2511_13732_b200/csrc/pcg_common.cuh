@@ -54,6 +54,12 @@ struct pcg_groups {
     void *allocation;  // single device allocation holding every array
     size_t agg_smem_bytes;  // dynamic shared memory of the aggregation kernels
     float accept_bias;      // constant added to the acceptance ratio (0 = PCG)
+    // scratch of the batched route of pcg_group_probs (inside `allocation`): rows are processed in chunks of
+    // probs_chunk; the transposed operand Dt[V, probs_chunk], per-row statistics and a row of zeros
+    int probs_chunk;
+    float *probs_dt;
+    float4 *probs_stats;
+    int32_t *probs_zero;
 };
 
 namespace pcg {

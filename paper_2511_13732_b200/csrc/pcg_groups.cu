@@ -269,6 +269,10 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     const size_t o_rptr = cv.take(rptr.size() * 4), o_rgrp = cv.take(rgrp.size() * 4);
     const size_t o_eoff = cv.take(eoff.size() * 4), o_ent = cv.take(ent.size() * 4);
     const size_t o_w = cv.take(w.size() * 4), o_entw = cv.take(entw.size() * 4), o_rw = cv.take(rw.size() * 4);
+    // scratch of the batched route of pcg_group_probs: 128 rows per chunk, more while Dt stays within 64 MB
+    int probs_chunk = (int)std::min<int64_t>(256, std::max<int64_t>(128, ((int64_t)64 << 20) / ((int64_t)V * 4) / 128 * 128));
+    const size_t o_pdt = cv.take((size_t)V * probs_chunk * 4), o_pst = cv.take((size_t)probs_chunk * 16);
+    const size_t o_pz = cv.take((size_t)probs_chunk * 4);
     const size_t total = cv.off ? cv.off : 256;
     void *mem = nullptr;
     if (!have_device) {
@@ -288,6 +292,7 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     if (e == cudaSuccess) e = upload(base, o_w, w);
     if (e == cudaSuccess) e = upload(base, o_entw, entw);
     if (e == cudaSuccess) e = upload(base, o_rw, rw);
+    if (e == cudaSuccess) e = cudaMemset(base + o_pz, 0, (size_t)probs_chunk * 4);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         cudaFree(mem);
@@ -324,6 +329,10 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     h->allocation = mem;
     h->agg_smem_bytes = agg_smem_bytes(SL, M, C);
     h->accept_bias = 0.f;
+    h->probs_chunk = probs_chunk;
+    h->probs_dt = (float *)(base + o_pdt);
+    h->probs_stats = (float4 *)(base + o_pst);
+    h->probs_zero = (int32_t *)(base + o_pz);
     *out = h;
     return PCG_OK;
 }

@@ -712,7 +712,8 @@ __global__ void __launch_bounds__(kAggThreads, 2) terminal_kernel(TerminalArgs a
 //                              within-group token draw, outputs
 // Sequences are processed in chunks whose Dt fits in L2.
 
-constexpr int kPrepThreads = 256;  // terminal_prepare_kernel
+constexpr int kPrepThreads = 256;  // terminal_prepare_kernel, row_stats_kernel
+constexpr int kProbsBatchedRows = 64;  // pcg_group_probs: from this many rows on, the batched kernels
 constexpr int kTrThreads = 256;    // residual_transpose_kernel
 #ifndef PCG_SPMM_THREADS
 #define PCG_SPMM_THREADS 128
@@ -827,6 +828,54 @@ __global__ void __launch_bounds__(kPrepThreads) terminal_prepare_kernel(PrepareA
     }
 }
 
+// Softmax statistics (scaled reference, 1/Z) of plain rows: one block per row.  Used by the batched route of
+// pcg_group_probs.
+template <typename T>
+__global__ void __launch_bounds__(kPrepThreads) row_stats_kernel(const void *logits, float s, float4 *stats, GroupsDev G) {
+    constexpr int NT = kPrepThreads, NW = NT / 32, NV = Elem<T>::kPerVec;
+    __shared__ float red[2 * NW];
+    const int tid = threadIdx.x, V = G.V;
+    const T *row = reinterpret_cast<const T *>(logits) + (int64_t)blockIdx.x * V;
+    RefSum st{kRefInit * s, 0.f};
+    int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
+    if (head > V) head = V;
+    const int nvec = (V - head) / NV;
+    const uint4 *vp = reinterpret_cast<const uint4 *>(row + head);
+    int idx = tid;
+    for (; idx + 3 * NT < nvec; idx += 4 * NT) {
+        uint4 r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) r[j] = ld_stream(vp + idx + j * NT);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float v[NV];
+            Elem<T>::unpack(r[j], v);
+            absorb<NV>(st, v, s);
+        }
+    }
+    for (; idx < nvec; idx += NT) {
+        float v[NV];
+        Elem<T>::unpack(ld_stream(vp + idx), v);
+        absorb<NV>(st, v, s);
+    }
+    for (int t = tid; t < head; t += NT) absorb1(st, Elem<T>::widen(row[t]), s);
+    for (int t = head + nvec * NV + tid; t < V; t += NT) absorb1(st, Elem<T>::widen(row[t]), s);
+    float rs = st.rs, Z = st.acc;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) merge(rs, Z, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, Z, o));
+    if ((tid & 31) == 0) {
+        red[2 * (tid >> 5)] = rs;
+        red[2 * (tid >> 5) + 1] = Z;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        rs = red[0];
+        Z = red[1];
+        for (int w = 1; w < NW; ++w) merge(rs, Z, red[2 * w], red[2 * w + 1]);
+        stats[blockIdx.x] = make_float4(rs, 1.0f / Z, 0.f, 0.f);
+    }
+}
+
 // Loads of Dt: cached in L2 only (.cg).  Every line of Dt is read once per group its token belongs to, at
 // unrelated times, so it has to survive in L2 between those reads; the streaming form used for the logits
 // (ld.global.nc.L1::no_allocate) is retained in L2 for too short a time for that.
@@ -898,7 +947,7 @@ __global__ void __launch_bounds__(kTrThreads, PCG_TR_MINBLOCKS) residual_transpo
     for (int q = 0; q < 4; ++q) {
         const int b = bbase + warp + 8 * q;
         const T *tp = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + max(n[q], 0)) * V + t;
-        const T *qp = reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(max(n[q], 0), K - 1)) * V + t;
+        const T *qp = K > 0 ? reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(max(n[q], 0), K - 1)) * V + t : tp;
         fast[q] = n[q] >= 0 && t + NV <= V && (((uintptr_t)tp | (uintptr_t)qp) & 15u) == 0;
         rp[q] = rq[q] = make_uint4(0u, 0u, 0u, 0u);
         if (fast[q]) {
@@ -921,7 +970,7 @@ __global__ void __launch_bounds__(kTrThreads, PCG_TR_MINBLOCKS) residual_transpo
                 Elem<T>::unpack(rq[q], lq);
             } else {  // ragged end of the row or rows that are not 16-byte aligned
                 const T *tp = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n[q]) * V + t;
-                const T *qp = reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(n[q], K - 1)) * V + t;
+                const T *qp = K > 0 ? reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(n[q], K - 1)) * V + t : tp;
 #pragma unroll
                 for (int e = 0; e < NV; ++e) {
                     const bool in = t + e < V;
@@ -1406,6 +1455,26 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
     return w;
 }
 
+// The sparse product over nb blocks of 32 sequences (nb a multiple of kSpmmWide when `wide`).
+static void launch_spmm(const SpmmArgs &sp, int nb, bool wide, const GroupsDev &G, cudaStream_t cs) {
+    const int gpb = kSpmmGroupsPerWarp * (kSpmmThreads / 32);  // groups per block
+    const unsigned gx = (unsigned)((G.M + gpb - 1) / gpb);
+    const bool has_w = G.pair_w != nullptr;
+    if (wide) {
+        const dim3 grid(gx, (unsigned)(nb / kSpmmWide));
+        if (has_w)
+            group_spmm_kernel<kSpmmWide, kSpmmDepth, true><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
+        else
+            group_spmm_kernel<kSpmmWide, kSpmmDepth, false><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
+    } else {
+        const dim3 grid(gx, (unsigned)nb);
+        if (has_w)
+            group_spmm_kernel<1, 16, true><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
+        else
+            group_spmm_kernel<1, 16, false><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
+    }
+}
+
 }  // namespace pcg
 
 using namespace pcg;
@@ -1424,10 +1493,32 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
         set_error("pcg_group_probs: too many rows for one launch");
         return PCG_ERR_UNSUPPORTED;
     }
-    ProbsArgs a{logits, out, (float)((double)kLog2e / (double)temperature)};
+    const float s = (float)((double)kLog2e / (double)temperature);
+    cudaStream_t cs = (cudaStream_t)stream;
     cudaError_t e;
+    if (rows >= kProbsBatchedRows) {
+        // many rows: the same transposed-operand / sparse-product kernels as the per-sequence stage of pcg_verify,
+        // a chunk of rows at a time through the handle's scratch (row statistics, then p(t) w in place of p - q)
+        const int chunk = groups->probs_chunk;  // a multiple of 128
+        const int tt = 32 * (int)(16 / dtype_bytes(dtype));
+        for (int64_t r0 = 0; r0 < rows; r0 += chunk) {
+            const int nr = (int)std::min<int64_t>(chunk, rows - r0);
+            const char *base = (const char *)logits + (size_t)r0 * G.V * dtype_bytes(dtype);
+            PCG_DISPATCH_DTYPE(dtype, row_stats_kernel<LogitT><<<nr, kPrepThreads, 0, cs>>>(base, s, groups->probs_stats, G));
+            const int nb = (nr + 127) / 128 * 4;  // blocks of 32 rows, whole warps of the sparse product
+            // every row is "a sequence whose only row is accepted": K = 0 makes the kernel form p alone
+            TransposeArgs tr{base, base, nr, 0, 0, chunk, s, groups->probs_zero, groups->probs_stats, groups->probs_dt};
+            const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
+            PCG_DISPATCH_DTYPE(dtype, residual_transpose_kernel<LogitT><<<tgrid, kTrThreads, 0, cs>>>(tr, G));
+            launch_spmm(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M}, nb, true, G, cs);
+        }
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e, "launching the batched group-probability kernels");
+        return PCG_OK;
+    }
+    ProbsArgs a{logits, out, s};
     PCG_DISPATCH_DTYPE(dtype, e = launch_cluster(group_probs_kernel<LogitT>, (int)(rows * G.slices), G.slices,
-                                                 groups->agg_smem_bytes, (cudaStream_t)stream, a, G));
+                                                 groups->agg_smem_bytes, cs, a, G));
     if (e != cudaSuccess) return cuda_fail(e, "launching group_probs_kernel");
     return PCG_OK;
 }
@@ -1546,23 +1637,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
                 PCG_DISPATCH_DTYPE(dtype, residual_transpose_kernel<LogitT><<<tgrid, kTrThreads, 0, cs>>>(tr, G));
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
-                SpmmArgs sp{w.Dt, B, b0, chunk, w.R};
-                const int gpb = kSpmmGroupsPerWarp * (kSpmmThreads / 32);  // groups per block
-                const unsigned gx = (unsigned)((G.M + gpb - 1) / gpb);
-                const bool has_w = G.pair_w != nullptr;
-                if (wide) {
-                    const dim3 grid(gx, (unsigned)(nb / kSpmmWide));
-                    if (has_w)
-                        group_spmm_kernel<kSpmmWide, kSpmmDepth, true><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
-                    else
-                        group_spmm_kernel<kSpmmWide, kSpmmDepth, false><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
-                } else {
-                    const dim3 grid(gx, (unsigned)nb);
-                    if (has_w)
-                        group_spmm_kernel<1, 16, true><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
-                    else
-                        group_spmm_kernel<1, 16, false><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
-                }
+                launch_spmm(SpmmArgs{w.Dt, B, b0, chunk, w.R}, nb, wide, G, cs);
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
             }

@@ -49,6 +49,35 @@ def test_group_probs_matches_oracle(oracle, name, rows):
     assert np.max(np.abs(got - want) / np.maximum(want, 1e-37)) < 1e-5
 
 
+@pytest.mark.parametrize("name,rows", [("C2", 150), ("C3", 300), ("C4", 64)])
+def test_group_probs_batched_route(oracle, name, rows):
+    """From 64 rows on pcg_group_probs runs the row-statistics / transposed-operand / sparse-product kernels, a chunk
+    of rows at a time (150 and 300 are ragged: not multiples of the 128 rows a warp of the product covers)."""
+    from paper_2511_13732_b200 import binding
+
+    cfg = W.CONFIGS[name]
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg, B=rows // cfg.K + 1)
+    x = np.ascontiguousarray(bt.draft_logits.reshape(-1, cfg.V)[:rows])
+    want = oracle.group_probs(x, groups.group_ptr, groups.group_tok, groups.tok_degree, cfg.temperature)
+    h = make_handle(groups)
+    got = binding.pcg_group_probs(logits_to_device(x), h, cfg.temperature).cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(got, want, rtol=1e-5, atol=1e-37)
+    np.testing.assert_allclose(got.sum(axis=1), 1.0, rtol=4e-6)
+    again = binding.pcg_group_probs(logits_to_device(x), h, cfg.temperature).cpu().numpy()
+    assert np.array_equal(again.astype(np.float64), got)  # bit-reproducible
+    # with general weights
+    rng = np.random.default_rng(3)
+    raw = rng.random(groups.nnz) + 0.05
+    tot = np.zeros(cfg.V)
+    np.add.at(tot, groups.group_tok, raw)
+    w = (raw / tot[groups.group_tok]).astype(np.float32)
+    want_w = oracle.group_probs(x, groups.group_ptr, groups.group_tok, groups.tok_degree, cfg.temperature,
+                                weights=w.astype(np.float64))
+    got_w = binding.pcg_group_probs(logits_to_device(x), make_handle(groups, weights=w), cfg.temperature).cpu().numpy()
+    np.testing.assert_allclose(got_w, want_w, rtol=1e-5, atol=1e-37)
+
+
 @pytest.mark.parametrize("hint", [1, 2, 4, 8])
 def test_group_probs_any_slicing(oracle, hint):
     from paper_2511_13732_b200 import binding
