@@ -124,9 +124,11 @@ const char *pcg_last_error(void);
  *   slices_hint: 0 = choose automatically; 1, 2, 4 or 8 = force that many token
  *                slices (= cluster size).  Rounded up if a slice would not fit
  *                in shared memory.
- * Limits (PCG_ERR_UNSUPPORTED beyond them): per thread block, slice_len*4 +
- * M*4 + (M/slices)*4 bytes plus 2 KB must fit in 227 KB of shared memory with
- * slices <= 8 and slice_len <= 65536; e.g. V <= 262144 with M <= 32768.
+ * The token-sliced copy needs M <= 65534 (16-bit group ids) and, per thread block, slice_len*4 + M*4 +
+ * (M/slices)*4 bytes plus 2 KB within 227 KB of shared memory with slices <= 8.  Where that is impossible the
+ * handle is built WITHOUT it (pcg_groups_info reports slices = 0): everything runs on the batched kernels,
+ * PCG_VERIFY_CLUSTER_TERMINAL and pcg_verify_static then return PCG_ERR_UNSUPPORTED, and a slices_hint other than 0
+ * is refused.
  * Errors: INVALID_ARG (null, V/M < 1), INVALID_GROUPS, UNSUPPORTED, CUDA.
  */
 pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg_groups **out);

@@ -54,6 +54,7 @@ struct pcg_groups {
     void *allocation;  // single device allocation holding every array
     size_t agg_smem_bytes;  // dynamic shared memory of the aggregation kernels
     float accept_bias;      // constant added to the acceptance ratio (0 = PCG)
+    bool has_sweep;         // the token-sliced sweep layout exists (M <= 65534 and it fits in shared memory)
     // scratch of the batched route of pcg_group_probs (inside `allocation`): rows are processed in chunks of
     // probs_chunk; the transposed operand Dt[V, probs_chunk], per-row statistics and a row of zeros
     int probs_chunk;

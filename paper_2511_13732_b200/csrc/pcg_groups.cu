@@ -181,18 +181,24 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     int C = slices_hint ? slices_hint : 1;
     if (!slices_hint)
         while (C < 8 && (V + C - 1) / C > 8192) C *= 2;
-    if (M >= (int)kNoGroup) {
-        set_error("M=%d: the sweep layout holds group ids in 16 bits (M <= 65534)", M);
-        return PCG_ERR_UNSUPPORTED;
-    }
+    // Beyond 65534 groups (the sweep entries hold group ids in 16 bits) or when a token slice plus the per-group
+    // partial sums cannot fit in shared memory, the handle carries no sweep layout: the kernels that need it (the
+    // per-row cluster kernel of pcg_group_probs, PCG_VERIFY_CLUSTER_TERMINAL) are then unavailable and the batched
+    // kernels are used throughout.
+    bool has_sweep = M < (int)kNoGroup;
     int SL = 0;
-    for (;; C *= 2) {
+    for (; has_sweep; C *= 2) {
         SL = (((V + C - 1) / C) + 63) / 64 * 64;
         if (SL <= 65472 && agg_smem_bytes(SL, M, C) <= kMaxSmem) break;
-        if (C >= 8) {
-            set_error("V=%d, M=%d do not fit the aggregation kernels' shared memory even with 8 slices", V, M);
+        if (C >= 8) has_sweep = false;
+    }
+    if (!has_sweep) {
+        if (slices_hint) {
+            set_error("V=%d, M=%d: no sweep layout is possible, so slices_hint must be 0", V, M);
             return PCG_ERR_UNSUPPORTED;
         }
+        C = 1;
+        SL = ((V + 63) / 64) * 64;
     }
 
     // ---- token-sliced sweep layout (see GroupsDev::ent) ----
@@ -206,7 +212,7 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
         std::vector<int32_t> cursor(gptr.begin(), gptr.end() - 1);  // tokens ascend, so each slice is a sub-range
         std::vector<int32_t> sub_lo((size_t)M), sub_hi((size_t)M), order((size_t)M);
         std::vector<std::vector<int32_t>> owned(NT);
-        for (int c = 0; c < C; ++c) {
+        for (int c = 0; c < C && has_sweep; ++c) {
             const int32_t t_end = (int32_t)std::min<int64_t>((int64_t)(c + 1) * SL, V);
             for (int g = 0; g < M; ++g) {
                 int32_t k = cursor[g];
@@ -327,7 +333,8 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     h->max_degree = max_deg;
     h->device_bytes = (int64_t)total;
     h->allocation = mem;
-    h->agg_smem_bytes = agg_smem_bytes(SL, M, C);
+    h->agg_smem_bytes = has_sweep ? agg_smem_bytes(SL, M, C) : 0;
+    h->has_sweep = has_sweep;
     h->accept_bias = 0.f;
     h->probs_chunk = probs_chunk;
     h->probs_dt = (float *)(base + o_pdt);
@@ -351,7 +358,7 @@ extern "C" pcg_status pcg_groups_info(const pcg_groups *groups, pcg_groups_info_
     out->V = groups->dev.V;
     out->M = groups->dev.M;
     out->nnz = groups->nnz;
-    out->slices = groups->dev.slices;
+    out->slices = groups->has_sweep ? groups->dev.slices : 0;
     out->slice_len = groups->dev.slice_len;
     out->max_group_size = groups->max_group_size;
     out->max_degree = groups->max_degree;

@@ -1143,7 +1143,9 @@ struct DrawArgs {
     const int32_t *term_n;
     const int32_t *term_flags;
     const float4 *term_stats;
-    const float *R;    // default mode: [B, M] residual sums
+    float *R;          // default mode: [B, M] residual sums (clamped in place when the masses are staged in global memory)
+    float *own_rows;   // dense mode with M too large for shared memory: [B, M] staging rows, else null
+    int own_in_smem;   // 1: the M clamped masses of a sequence are staged in shared memory, 0: in global memory
     const float *Pws;  // dense mode: [B*(K+1), M] target group masses
     const float *Qws;  // dense mode: [B*K, M] draft group masses
     int32_t *out_accept_len;
@@ -1162,12 +1164,16 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
     constexpr int NT = kDrawThreads;
     extern __shared__ __align__(16) unsigned char raw[];
     const int M = G.M, V = G.V, K = a.K;
-    float *own = reinterpret_cast<float *>(raw);
-    unsigned char *tail = raw + (((size_t)own_slot(M) + 1) * 4 + 15) / 16 * 16;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    // The M clamped masses of the sequence: in (padded) shared memory when they fit, else in a row of global memory
+    // (the sequence's own row of R, or a staging row in dense mode); `slot` maps a group to its place.
+    const bool in_smem = a.own_in_smem;
+    float *own = in_smem ? reinterpret_cast<float *>(raw) : (DENSE ? a.own_rows : a.R) + (size_t)b * M;
+    auto slot = [&](int j) { return in_smem ? own_slot(j) : j; };
+    unsigned char *tail = raw + (in_smem ? (((size_t)own_slot(M) + 1) * 4 + 15) / 16 * 16 : 0);
     double *dscratch = reinterpret_cast<double *>(tail);      // 32 doubles
     float *scratch = reinterpret_cast<float *>(dscratch + 32);  // 64 floats
     int *ibox = reinterpret_cast<int *>(scratch + 64);          // 8 ints
-    const int b = blockIdx.x, tid = threadIdx.x;
     // The transposed operand has been consumed (workspace contents are of no interest after the call):
     // dropping its dirty lines from L2 spares the write-back that would otherwise compete with the next call's
     // streaming reads (measured: the next position kernel runs 4 % faster).
@@ -1189,11 +1195,11 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
     for (int attempt = 0; attempt < 2; ++attempt) {
         if (DENSE) {
             for (int g = tid; g < M; g += NT)
-                own[own_slot(g)] = fmaxf(residual ? Pn[g] - Qn[g] : Pn[g], 0.f);  // (P - Q)_+ ; NaN becomes 0
+                own[slot(g)] = fmaxf(residual ? Pn[g] - Qn[g] : Pn[g], 0.f);  // (P - Q)_+ ; NaN becomes 0
         } else if (attempt == 0) {
             // R holds sum_t (p - q)/N for a rejection and sum_t p/N for the bonus row
-            const float *Rb = a.R + (size_t)b * M;
-            for (int g = tid; g < M; g += NT) own[own_slot(g)] = fmaxf(Rb[g], 0.f);
+            const float *Rb = a.R + (size_t)b * M;  // (with global staging this is `own` itself: clamped in place)
+            for (int g = tid; g < M; g += NT) own[slot(g)] = fmaxf(Rb[g], 0.f);
         } else {
             // slow path of the zero-residual fallback: the target masses straight from the row
             const float rs = a.term_stats[b].x;
@@ -1204,13 +1210,13 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
                     const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
                     acc += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs)), w);
                 }
-                own[own_slot(g)] = fmaxf(acc, 0.f);
+                own[slot(g)] = fmaxf(acc, 0.f);
             }
         }
         __syncthreads();
         // ---- prefix sums over the groups (double): a contiguous chunk per thread, then a block scan ----
         my_sum = 0.0;
-        for (int j = i0; j < i1; ++j) my_sum += (double)own[own_slot(j)];
+        for (int j = i0; j < i1; ++j) my_sum += (double)own[slot(j)];
         block_scan<NT>(my_sum, dscratch, &my_excl, &my_incl, &Ztot);
         if (Ztot > 0.0 || !residual) break;
         // a rejection whose residual vanished (P == Q to rounding): draw from P instead
@@ -1229,7 +1235,7 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
     __syncthreads();
     int my_last = -1;
     for (int j = i0; j < i1; ++j)
-        if (own[own_slot(j)] > 0.f) my_last = j;
+        if (own[slot(j)] > 0.f) my_last = j;
     if (my_last >= 0) atomicMax(&ibox[3], my_last);
     if (my_sum > 0.0 && my_incl > target) atomicMin(&ibox[2], tid);
     __syncthreads();
@@ -1237,7 +1243,7 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
         double loc = 0.0;
         int pick = my_last;
         for (int j = i0; j < i1; ++j) {
-            loc += (double)own[own_slot(j)];
+            loc += (double)own[slot(j)];
             if (my_excl + loc > target) {
                 pick = j;
                 break;
@@ -1424,6 +1430,7 @@ struct VerifyWorkspace {
     float4 *stats, *term_stats;
     float *Dt, *R;     // default mode
     float *Pws, *Qws;  // dense mode
+    float *own_rows;   // dense mode, M beyond the draw kernel's shared memory
     size_t bytes;
 };
 
@@ -1447,6 +1454,7 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
     if (mode == PCG_VERIFY_DENSE) {
         w.Pws = (float *)(p + take((size_t)(B * (K + 1) * M) * 4));
         w.Qws = (float *)(p + take((size_t)(B * K * M) * 4));
+        if (draw_smem_bytes((int)M) > kMaxDynSmem) w.own_rows = (float *)(p + take((size_t)(B * M) * 4));
     } else if (mode != PCG_VERIFY_CLUSTER_TERMINAL) {
         w.Dt = (float *)(p + take((size_t)V * (size_t)terminal_chunk((int)B, (int)V) * 4));
         w.R = (float *)(p + take((size_t)(B * M) * 4));
@@ -1496,7 +1504,7 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
     const float s = (float)((double)kLog2e / (double)temperature);
     cudaStream_t cs = (cudaStream_t)stream;
     cudaError_t e;
-    if (rows >= kProbsBatchedRows) {
+    if (rows >= kProbsBatchedRows || !groups->has_sweep) {
         // many rows: the same transposed-operand / sparse-product kernels as the per-sequence stage of pcg_verify,
         // a chunk of rows at a time through the handle's scratch (row statistics, then p(t) w in place of p - q)
         const int chunk = groups->probs_chunk;  // a multiple of 128
@@ -1576,13 +1584,15 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
     // Default: one cluster per sequence while all clusters are resident in about one wave (a handful of
     // sequences: fewer launches, lower latency), the batched kernels beyond that.
     const bool cluster_terminal = mode == PCG_VERIFY_CLUSTER_TERMINAL ||
-                                  (mode == PCG_VERIFY_DEFAULT && (int64_t)B * G.slices <= 2 * (int64_t)groups->sm_count);
-    const size_t draw_smem = draw_smem_bytes(G.M);
-    if (!cluster_terminal && draw_smem > kMaxDynSmem) {
-        set_error("pcg_verify: M=%d needs %zu bytes of shared memory in the terminal draw (limit %zu)", G.M, draw_smem,
-                  kMaxDynSmem);
+                                  (mode == PCG_VERIFY_DEFAULT && groups->has_sweep &&
+                                   (int64_t)B * G.slices <= 2 * (int64_t)groups->sm_count);
+    if (cluster_terminal && !groups->has_sweep) {
+        set_error("pcg_verify: this handle has no sweep layout (M=%d, V=%d), so the cluster terminal is unavailable", G.M,
+                  G.V);
         return PCG_ERR_UNSUPPORTED;
     }
+    const bool own_in_smem = draw_smem_bytes(G.M) <= kMaxDynSmem;
+    const size_t draw_smem = own_in_smem ? draw_smem_bytes(G.M) : 1024;
     cudaStream_t cs = (cudaStream_t)stream;
     const VerifyWorkspace w = carve_workspace(workspace, B, K, G.V, G.M, mode);
     const float s = (float)((double)kLog2e / (double)temperature);
@@ -1643,7 +1653,8 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
             }
         }
         DrawArgs dr{target_logits, draft_tokens, uniforms, K,     s,     w.labels,       w.term_n,   w.term_flags,
-                    w.term_stats,  w.R,          w.Pws,    w.Qws, out_accept_len, out_tokens, out_groups, out_flags,
+                    w.term_stats,  w.R,          w.own_rows, own_in_smem ? 1 : 0, w.Pws, w.Qws, out_accept_len, out_tokens,
+                    out_groups,    out_flags,
                     dense ? nullptr : w.Dt,
                     dense ? 0 : (size_t)G.V * (size_t)terminal_chunk(B, G.V) * 4 / 128};
         auto launch_draw = [&](auto kern) -> cudaError_t {
@@ -1688,6 +1699,11 @@ extern "C" pcg_status pcg_verify_static(const void *target_logits, const void *d
     if (B < 0 || K < 1) {
         set_error("pcg_verify_static: need B >= 0 and K >= 1 (B=%d K=%d)", B, K);
         return PCG_ERR_INVALID_ARG;
+    }
+    if (!groups->has_sweep) {
+        set_error("pcg_verify_static: this handle has no sweep layout (M=%d), which the scratch-free mode needs",
+                  groups->dev.M);
+        return PCG_ERR_UNSUPPORTED;
     }
     const uint32_t mode = PCG_VERIFY_CLUSTER_TERMINAL;  // the mode whose scratch is a few bytes per position
     const size_t need = pcg_verify_workspace_bytes(B, K, groups->dev.V, groups->dev.M, dtype, mode);

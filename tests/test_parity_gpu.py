@@ -130,6 +130,33 @@ def test_verify_c5_disjoint_groups_variant(oracle, mode):
     _assert_parity(run_verify(bt, make_handle(groups), mode=mode), ref)
 
 
+@pytest.mark.parametrize("mode", [pytest.param(0, id="default"), pytest.param(1, id="dense"), pytest.param(4, id="batched")])
+def test_verify_singleton_groups_at_full_vocabulary(oracle, mode):
+    """65,536 singleton groups (token-level speculative sampling at the paper's vocabulary size): more groups than
+    the 16-bit sweep layout and the draw kernel's shared memory hold, so the handle has no sweep layout, the
+    masses are staged in global memory, and the cluster terminal is refused."""
+    from paper_2511_13732_b200 import binding
+
+    cfg = W.CONFIGS["C5s"]
+    groups = W.make_groups(cfg)
+    assert groups.M == 65536
+    bt = W.make_batch(cfg, B=6)
+    ref = run_oracle(oracle, bt, groups)
+    h = make_handle(groups)
+    assert h.info.slices == 0
+    got = run_verify(bt, h, mode=mode)
+    _assert_parity(got, ref)
+    assert np.array_equal(got[2][got[2] >= 0], got[1][got[1] >= 0])  # singleton groups: group id = token id
+    if mode == 0:
+        with pytest.raises(binding.PcgError) as err:
+            run_verify(bt, h, mode=2)
+        assert err.value.status == 3
+        x = bt.target_logits.reshape(-1, cfg.V)[:3]
+        want = oracle.softmax(x, cfg.temperature)  # with singleton groups P is the token distribution itself
+        P = binding.pcg_group_probs(logits_to_device(x), h, cfg.temperature).cpu().numpy()
+        np.testing.assert_allclose(P, want, rtol=1e-5, atol=1e-37)
+
+
 def test_verify_batch_spanning_several_sequence_blocks(oracle):
     """The batched per-sequence stage handles 32 sequences per line: 70 sequences = two full blocks and a ragged one,
     with a group count that is not a multiple of the 32 groups a block of the sparse product owns."""
