@@ -157,6 +157,19 @@ def test_verify_singleton_groups_at_full_vocabulary(oracle, mode):
         np.testing.assert_allclose(P, want, rtol=1e-5, atol=1e-37)
 
 
+def test_verify_batch_larger_than_one_chunk_of_the_batched_stage(oracle):
+    """At V = 65536 the transposed operand of 256 sequences fills the L2 budget, so 288 sequences run the batched
+    per-sequence stage in two chunks (256 + 32)."""
+    cfg = W.scaled(W.CONFIGS["C5"], B=288, K=2)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    ref = run_oracle(oracle, bt, groups)
+    h = make_handle(groups)
+    got = run_verify(bt, h, mode=4)
+    _assert_parity(got, ref)
+    assert len(set(ref.accept_len[256:].tolist())) > 1  # the second chunk holds different outcomes
+
+
 def test_verify_batch_spanning_several_sequence_blocks(oracle):
     """The batched per-sequence stage handles 32 sequences per line: 70 sequences = two full blocks and a ragged one,
     with a group count that is not a multiple of the 32 groups a block of the sparse product owns."""
