@@ -332,6 +332,28 @@ def main():
                                  "outputs_equal_to_timed_mode": bool(same)}
             del ws_m
 
+    # the timed mode once more, captured in a CUDA graph and replayed (launch overhead off the host)
+    if world == 1 and not args.no_other_modes:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        reps = 200
+        for _ in range(3):
+            graph.replay()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        for _ in range(reps):
+            graph.replay()
+        c1.record()
+        torch.cuda.synchronize()
+        other_modes["cuda_graph_replay_of_timed_mode"] = {"ms_per_step": c0.elapsed_time(c1) / reps, "steps": reps}
+
     # the other two entry points of the boundary, briefly: pcg_group_probs on a slice of the target rows, and the
     # one-time group construction on a seeded clustered table of the workload's vocabulary size
     extras = {}
