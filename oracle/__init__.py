@@ -8,6 +8,7 @@ from .pcg_oracle import (  # noqa: F401
     BF16,
     F16,
     FLAG_ZERO_RESIDUAL,
+    FLAG_THINNING_EXHAUSTED,
     build,
     max_threads,
     softmax,

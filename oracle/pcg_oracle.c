@@ -22,11 +22,16 @@
  * Parity status.  Every function below is pinned by the CPU test-suite to
  * facts that do not come from this file (a library softmax, dense-matrix brute
  * force in exact rationals, the exactness proposition checked by enumeration,
- * a separately written token-level speculative-sampling verifier).  What can
+ * a separately written token-level speculative-sampling verifier).  The
+ * thinning sampler of pcg_oracle_verify_thinning is pinned by the laws the
+ * paper states for it, measured over many seeded uniforms (kept group ~
+ * normalised residual, emitted group ~ target coarse distribution, mean
+ * number of trials = 1/TV, token ~ target-conditional), by its singleton-group
+ * special case and by its fallback equalling the enumerated draw.  What can
  * NOT be pinned: draw-by-draw agreement with the authors' own program (none is
- * published, and its residual sampler uses thinning with different
- * randomness) -- for that comparison alone: "parity unpinned"; agreement in
- * distribution is what is pinned.
+ * published, and how it maps random numbers to draws is not stated) -- for
+ * that comparison alone: "parity unpinned"; agreement in distribution is what
+ * is pinned.
  */
 #include <math.h>
 #include <stdint.h>
@@ -42,6 +47,7 @@
 
 /* flag bits written per sequence */
 #define ORACLE_FLAG_ZERO_RESIDUAL 2 /* reject taken but sum of (P-Q)_+ was <= 0 */
+#define ORACLE_FLAG_THINNING_EXHAUSTED 8 /* every supplied thinning trial was turned down; enumerated draw used */
 
 /* IEEE binary16 bit pattern to double, from the format's definition: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
 static double half_bits_to_double(uint16_t h) {
@@ -169,12 +175,54 @@ static int inverse_cdf(const double *w, int n, double u, double *total_out, doub
 }
 
 /*
+ * Group-label coupling (Sec. 2.2): the label of token x is drawn from w_{.,x} over S(x), the groups containing
+ * x in ascending group id.  Equal split: j = min(floor(u N), N-1); general weights: inverse CDF over them.
+ * Returns the group id; *margin receives the distance from u to the nearest point where the label changes.
+ */
+static int32_t draw_label(int32_t x, double u, const double *weights, const int32_t *rev_ptr, const int32_t *rev_grp,
+                          const int32_t *rev_nz, double *margin) {
+    int32_t N = rev_ptr[x + 1] - rev_ptr[x];
+    int j;
+    if (!weights) {
+        double uj = u * (double)N;
+        j = (int)floor(uj);
+        if (j > N - 1) j = N - 1;
+        if (margin) {
+            double d = INFINITY;
+            for (int e = 1; e < N; ++e) {
+                double dd = fabs(u - (double)e / (double)N);
+                if (dd < d) d = dd;
+            }
+            *margin = d;
+        }
+    } else {
+        /* inverse CDF over the weights of x's groups, ascending group id */
+        double *wx = (double *)malloc(sizeof(double) * (size_t)N);
+        for (int e = 0; e < N; ++e) wx[e] = weights[rev_nz[rev_ptr[x] + e]];
+        j = inverse_cdf(wx, N, u, NULL, margin);
+        free(wx);
+    }
+    return rev_grp[rev_ptr[x] + j];
+}
+
+/*
  * One sequence of Algorithm 1 with the randomness supplied from outside.
  *
  * uniforms[i][0], i < K : group-label draw for drafted position i
  * uniforms[i][1], i < K : accept draw for drafted position i
  * uniforms[K][0]        : terminal group draw (residual or bonus)
  * uniforms[K][1]        : terminal within-group token draw
+ *
+ * Terminal group, two ways.  thin == NULL: enumerate the residual over all groups and invert its CDF with
+ * uniforms[K][0].  thin != NULL ([B, n_trials, 3]): the paper's own sampler, "Residual sampling via thinning"
+ * (Sec. 2.2), which never enumerates the groups.  Trial r uses thin[r][0] to draw a token y from the target
+ * row by inverse CDF in token order, thin[r][1] to draw y's label k ~ w_{.,y} (so that k ~ the target's coarse
+ * distribution), and keeps k if thin[r][2] < [1 - draft mass(k) / target mass(k)]_+; otherwise the next trial
+ * draws a new (y, k).  After all accepted positions (no rejection) there is no draft mass: the first candidate
+ * is kept, which draws the bonus group from the target's coarse distribution.  The paper's sampler is not
+ * bounded; here the trials are: if all n_trials candidates are turned down the group is drawn by the enumerated
+ * inverse CDF with uniforms[K][0] instead (same law) and the sequence is flagged.  The token inside the kept
+ * group is then drawn from the target-conditional with uniforms[K][1], as the thinning paragraph prescribes.
  *
  * rev_ptr/rev_grp is the reverse membership S(t) (groups containing t, in
  * ascending group id) built by the caller of verify_sequence from the CSR.
@@ -183,9 +231,9 @@ static void verify_sequence(const void *target_logits, const void *draft_logits,
                             double T, const int32_t *draft_tokens, int M, const int32_t *group_ptr,
                             const int32_t *group_tok, const int32_t *tok_degree, const double *weights,
                             const int32_t *rev_ptr, const int32_t *rev_grp, const int32_t *rev_nz,
-                            const float *uniforms, double accept_bias, int32_t *accept_len, int32_t *tokens,
-                            int32_t *groups, int32_t *flags, double *margins, double *p, double *q, double *P,
-                            double *Q, double *R) {
+                            const float *uniforms, const float *thin, int n_trials, double accept_bias,
+                            int32_t *accept_len, int32_t *tokens, int32_t *groups, int32_t *flags, int32_t *trials,
+                            double *margins, double *p, double *q, double *P, double *Q, double *R) {
     const float *u = uniforms + b * (int64_t)(K + 1) * 2;
     int32_t *tok_out = tokens + b * (int64_t)(K + 1);
     int32_t *grp_out = groups + b * (int64_t)(K + 1);
@@ -205,28 +253,7 @@ static void verify_sequence(const void *target_logits, const void *draft_logits,
         coarse_grain(q, M, group_ptr, group_tok, tok_degree, weights, Q);
         /* group-label coupling (Sec. 2.2): K_i ~ w_{.,x} over S(x) */
         int32_t x = draft_tokens[b * (int64_t)K + i];
-        int32_t N = rev_ptr[x + 1] - rev_ptr[x];
-        int j;
-        if (!weights) {
-            double uj = (double)u[2 * i] * (double)N;
-            j = (int)floor(uj);
-            if (j > N - 1) j = N - 1;
-            if (mg) {
-                double d = INFINITY;
-                for (int e = 1; e < N; ++e) {
-                    double dd = fabs((double)u[2 * i] - (double)e / (double)N);
-                    if (dd < d) d = dd;
-                }
-                mg[2 * i] = d;
-            }
-        } else {
-            /* inverse CDF over the weights of x's groups, ascending group id */
-            double *wx = (double *)malloc(sizeof(double) * (size_t)N);
-            for (int e = 0; e < N; ++e) wx[e] = weights[rev_nz[rev_ptr[x] + e]];
-            j = inverse_cdf(wx, N, (double)u[2 * i], NULL, mg ? &mg[2 * i] : NULL);
-            free(wx);
-        }
-        int32_t g = rev_grp[rev_ptr[x] + j];
+        int32_t g = draw_label(x, (double)u[2 * i], weights, rev_ptr, rev_grp, rev_nz, mg ? &mg[2 * i] : NULL);
         grp_out[i] = g;
         /* acceptance (Sec. 2.2): u < min(1, target mass / draft mass); a constant
            bias on the ratio (the SSD comparison system of Sec. 3.2) is 0 for PCG */
@@ -245,17 +272,49 @@ static void verify_sequence(const void *target_logits, const void *draft_logits,
     if (!have_Q) {
         softmax_row(target_logits, dtype, b * (int64_t)(K + 1) + K, V, T, p);
         coarse_grain(p, M, group_ptr, group_tok, tok_degree, weights, P);
-        for (int g = 0; g < M; ++g) R[g] = P[g];
-    } else {
-        for (int g = 0; g < M; ++g) R[g] = P[g] > Q[g] ? P[g] - Q[g] : 0.0;
     }
-    double Z = 0.0;
-    for (int g = 0; g < M; ++g) Z += R[g];
-    if (!(Z > 0.0)) { /* cannot happen in exact arithmetic after a rejection */
-        for (int g = 0; g < M; ++g) R[g] = P[g];
-        fl |= ORACLE_FLAG_ZERO_RESIDUAL;
+    int gs = -1;
+    double m_group = INFINITY; /* smallest margin over the decisions that led to the terminal group */
+    if (thin) {
+        const float *tu = thin + b * (int64_t)n_trials * 3;
+        int used = 0;
+        for (int r = 0; r < n_trials && gs < 0; ++r) {
+            double m_tok = INFINITY, m_lab = INFINITY, m_keep = INFINITY;
+            int y = inverse_cdf(p, V, (double)tu[3 * r], NULL, &m_tok);            /* y ~ target */
+            int32_t k = draw_label(y, (double)tu[3 * r + 1], weights, rev_ptr, rev_grp, rev_nz, &m_lab); /* k ~ w_{.,y} */
+            int keep = 1;
+            if (have_Q) { /* thinning probability a(k) = [1 - draft mass / target mass]_+ */
+                double a = P[k] > 0.0 ? 1.0 - Q[k] / P[k] : 0.0;
+                if (a < 0.0) a = 0.0;
+                keep = (double)tu[3 * r + 2] < a;
+                m_keep = fabs((double)tu[3 * r + 2] - a);
+            }
+            if (m_tok < m_group) m_group = m_tok;
+            if (m_lab < m_group) m_group = m_lab;
+            if (m_keep < m_group) m_group = m_keep;
+            used = r + 1;
+            if (keep) gs = k;
+        }
+        if (trials) trials[b] = used;
+        if (gs < 0) fl |= ORACLE_FLAG_THINNING_EXHAUSTED;
     }
-    int gs = inverse_cdf(R, M, (double)u[2 * K], NULL, mg ? &mg[2 * K] : NULL);
+    if (gs < 0) { /* enumerated residual over all groups, inverse CDF in group order */
+        if (!have_Q) {
+            for (int g = 0; g < M; ++g) R[g] = P[g];
+        } else {
+            for (int g = 0; g < M; ++g) R[g] = P[g] > Q[g] ? P[g] - Q[g] : 0.0;
+        }
+        double Z = 0.0;
+        for (int g = 0; g < M; ++g) Z += R[g];
+        if (!(Z > 0.0)) { /* cannot happen in exact arithmetic after a rejection */
+            for (int g = 0; g < M; ++g) R[g] = P[g];
+            fl |= ORACLE_FLAG_ZERO_RESIDUAL;
+        }
+        double m_enum = INFINITY;
+        gs = inverse_cdf(R, M, (double)u[2 * K], NULL, &m_enum);
+        if (m_enum < m_group) m_group = m_enum;
+    }
+    if (mg) mg[2 * K] = m_group;
     /* within-group conditional (Sec. 2.2): Pr(z = t | g*) = p(t) w_{g*,t} / P[g*] */
     int32_t lo = group_ptr[gs], hi = group_ptr[gs + 1];
     int len = hi - lo;
@@ -282,11 +341,11 @@ static void verify_sequence(const void *target_logits, const void *draft_logits,
  *   flags [B] (may be NULL), margins [B, K+1, 2] doubles (may be NULL).
  * threads <= 0 means "all cores".  Returns 0, or non-zero on bad arguments.
  */
-int pcg_oracle_verify(const void *target_logits, const void *draft_logits, int dtype, int B, int K, int V,
-                      const int32_t *draft_tokens, int M, const int32_t *group_ptr, const int32_t *group_tok,
-                      const int32_t *tok_degree, const double *weights, const float *uniforms, float temperature,
-                      double accept_bias, int32_t *accept_len, int32_t *tokens, int32_t *groups, int32_t *flags,
-                      double *margins, int threads) {
+static int verify_batch(const void *target_logits, const void *draft_logits, int dtype, int B, int K, int V,
+                        const int32_t *draft_tokens, int M, const int32_t *group_ptr, const int32_t *group_tok,
+                        const int32_t *tok_degree, const double *weights, const float *uniforms, const float *thin,
+                        int n_trials, float temperature, double accept_bias, int32_t *accept_len, int32_t *tokens,
+                        int32_t *groups, int32_t *flags, int32_t *trials, double *margins, int threads) {
     if (!target_logits || !draft_logits || !draft_tokens || !group_ptr || !group_tok || !tok_degree || !uniforms ||
         !accept_len || !tokens || !groups)
         return 1;
@@ -337,7 +396,8 @@ int pcg_oracle_verify(const void *target_logits, const void *draft_logits, int d
             for (int b = 0; b < B; ++b)
                 verify_sequence(target_logits, draft_logits, dtype, b, K, V, (double)temperature, draft_tokens, M,
                                 group_ptr, group_tok, tok_degree, weights, rev_ptr, rev_grp, rev_nz, uniforms,
-                                accept_bias, accept_len, tokens, groups, flags, margins, p, q, P, Q, R);
+                                thin, n_trials, accept_bias, accept_len, tokens, groups, flags, trials, margins,
+                                p, q, P, Q, R);
         }
         free(p);
         free(q);
@@ -350,6 +410,34 @@ int pcg_oracle_verify(const void *target_logits, const void *draft_logits, int d
     free(rev_nz);
     free(fill);
     return failed ? 2 : 0;
+}
+
+int pcg_oracle_verify(const void *target_logits, const void *draft_logits, int dtype, int B, int K, int V,
+                      const int32_t *draft_tokens, int M, const int32_t *group_ptr, const int32_t *group_tok,
+                      const int32_t *tok_degree, const double *weights, const float *uniforms, float temperature,
+                      double accept_bias, int32_t *accept_len, int32_t *tokens, int32_t *groups, int32_t *flags,
+                      double *margins, int threads) {
+    return verify_batch(target_logits, draft_logits, dtype, B, K, V, draft_tokens, M, group_ptr, group_tok,
+                        tok_degree, weights, uniforms, NULL, 0, temperature, accept_bias, accept_len, tokens, groups,
+                        flags, NULL, margins, threads);
+}
+
+/*
+ * Batched verification with the thinning sampler for the terminal group (see verify_sequence).
+ * thin_uniforms [B, n_trials, 3] floats in [0,1), n_trials >= 1; trials [B] (may be NULL) receives the number
+ * of candidates drawn (1 after an all-accepted sequence).  margins[b][K][0] is the smallest margin over every
+ * decision that led to the terminal group.  Everything else as pcg_oracle_verify.
+ */
+int pcg_oracle_verify_thinning(const void *target_logits, const void *draft_logits, int dtype, int B, int K, int V,
+                               const int32_t *draft_tokens, int M, const int32_t *group_ptr,
+                               const int32_t *group_tok, const int32_t *tok_degree, const double *weights,
+                               const float *uniforms, const float *thin_uniforms, int n_trials, float temperature,
+                               double accept_bias, int32_t *accept_len, int32_t *tokens, int32_t *groups,
+                               int32_t *flags, int32_t *trials, double *margins, int threads) {
+    if (!thin_uniforms || n_trials < 1) return 1;
+    return verify_batch(target_logits, draft_logits, dtype, B, K, V, draft_tokens, M, group_ptr, group_tok,
+                        tok_degree, weights, uniforms, thin_uniforms, n_trials, temperature, accept_bias, accept_len,
+                        tokens, groups, flags, trials, margins, threads);
 }
 
 /* Number of threads pcg_oracle_verify uses for threads <= 0. */

@@ -17,6 +17,7 @@ F32 = 0
 BF16 = 1
 F16 = 2
 FLAG_ZERO_RESIDUAL = 2
+FLAG_THINNING_EXHAUSTED = 8
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "pcg_oracle.c")
@@ -46,6 +47,9 @@ def _load():
         lib.pcg_oracle_verify.argtypes = [c_vp, c_vp, c_i, c_i, c_i, c_i, c_vp, c_i, c_vp, c_vp, c_vp, c_vp, c_vp,
                                           c_f, c_d, c_vp, c_vp, c_vp, c_vp, c_vp, c_i]
         lib.pcg_oracle_verify.restype = c_i
+        lib.pcg_oracle_verify_thinning.argtypes = [c_vp, c_vp, c_i, c_i, c_i, c_i, c_vp, c_i, c_vp, c_vp, c_vp, c_vp,
+                                                   c_vp, c_vp, c_i, c_f, c_d, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_i]
+        lib.pcg_oracle_verify_thinning.restype = c_i
         lib.pcg_oracle_max_threads.argtypes = []
         lib.pcg_oracle_max_threads.restype = c_i
         _lib = lib
@@ -108,11 +112,17 @@ class OracleResult:
     groups: np.ndarray  # [B, K+1] int32, unused slots -1
     flags: np.ndarray  # [B] int32
     margins: np.ndarray  # [B, K+1, 2] float64: [i<K] = (label, accept); [K] = (terminal group, terminal token)
+    trials: np.ndarray = None  # [B] int32, thinning only: candidates drawn for the terminal group
 
 
 def verify(target_logits, draft_logits, draft_tokens, group_ptr, group_tok, tok_degree, uniforms,
-           temperature: float = 1.0, weights=None, accept_bias: float = 0.0, threads: int = 1) -> OracleResult:
-    """Run Algorithm 1's verification for a batch; see pcg_oracle.c for the layouts."""
+           temperature: float = 1.0, weights=None, accept_bias: float = 0.0, threads: int = 1,
+           thin_uniforms=None) -> OracleResult:
+    """Run Algorithm 1's verification for a batch; see pcg_oracle.c for the layouts.
+
+    With ``thin_uniforms`` ([B, n_trials, 3]) the terminal group comes from the thinning sampler of Sec. 2.2
+    instead of the enumerated inverse CDF, and ``trials`` is filled in.
+    """
     tl, dt = _logits(target_logits)
     dl, dt2 = _logits(draft_logits)
     if dt != dt2:
@@ -135,6 +145,18 @@ def verify(target_logits, draft_logits, draft_tokens, group_ptr, group_tok, tok_
         flags=np.zeros(B, np.int32),
         margins=np.empty((B, K + 1, 2), np.float64),
     )
+    if thin_uniforms is not None:
+        tu = np.ascontiguousarray(thin_uniforms, dtype=np.float32)
+        if tu.ndim != 3 or tu.shape[0] != B or tu.shape[1] < 1 or tu.shape[2] != 3:
+            raise ValueError("thin_uniforms must be [B, n_trials >= 1, 3]")
+        res.trials = np.zeros(B, np.int32)
+        rc = _load().pcg_oracle_verify_thinning(_ptr(tl), _ptr(dl), dt, B, K, V, _ptr(x), M, _ptr(gp), _ptr(gt), _ptr(dg),
+                                                _ptr(w), _ptr(u), _ptr(tu), tu.shape[1], temperature, accept_bias,
+                                                _ptr(res.accept_len), _ptr(res.tokens), _ptr(res.groups),
+                                                _ptr(res.flags), _ptr(res.trials), _ptr(res.margins), threads)
+        if rc:
+            raise ValueError(f"pcg_oracle_verify_thinning failed ({rc})")
+        return res
     rc = _load().pcg_oracle_verify(_ptr(tl), _ptr(dl), dt, B, K, V, _ptr(x), M, _ptr(gp), _ptr(gt), _ptr(dg), _ptr(w),
                                    _ptr(u), temperature, accept_bias, _ptr(res.accept_len), _ptr(res.tokens),
                                    _ptr(res.groups), _ptr(res.flags), _ptr(res.margins), threads)

@@ -10,6 +10,7 @@ import shutil
 import pytest
 
 import test_oracle_pins as pins
+import test_thinning_oracle_pins as thin_pins
 
 ORACLE_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle")
 
@@ -30,8 +31,8 @@ MUTATIONS = [
     ("temperature_ignored", "p[t] = load_logit(logits, dtype, off + t) / T;", "p[t] = load_logit(logits, dtype, off + t);", 0),
     ("bonus_token_from_last_drafted_row", "softmax_row(target_logits, dtype, b * (int64_t)(K + 1) + K, V, T, p);",
      "softmax_row(target_logits, dtype, b * (int64_t)(K + 1) + K - 1, V, T, p);", 0),
-    ("terminal_group_uses_token_uniform", "int gs = inverse_cdf(R, M, (double)u[2 * K], NULL,",
-     "int gs = inverse_cdf(R, M, (double)u[2 * K + 1], NULL,", 0),
+    ("terminal_group_uses_token_uniform", "gs = inverse_cdf(R, M, (double)u[2 * K], NULL,",
+     "gs = inverse_cdf(R, M, (double)u[2 * K + 1], NULL,", 0),
     ("residual_not_clamped", "R[g] = P[g] > Q[g] ? P[g] - Q[g] : 0.0;", "R[g] = fabs(P[g] - Q[g]);", 0),
     ("accepted_position_emits_group_representative", "tok_out[i] = x; /*", "tok_out[i] = group_tok[group_ptr[g]]; /*", 0),
     ("first_rejection_does_not_stop_the_loop", "            n = i;\n            have_Q = 1;\n            break;",
@@ -48,6 +49,29 @@ PIN_CALLS = (
     + [lambda o, s=s: pins.test_residual_group_law_and_emitted_group_is_target_coarse(o, s) for s in (11, 13)]
     + [lambda o, s=s: pins.test_within_group_and_bonus_token_law(o, s) for s in (11, 14)]
     + [lambda o, n=n: pins.test_emission_structure_on_workloads(o, n) for n in ("C1",)]
+)
+
+
+# planted mistakes in the thinning sampler, checked against the thinning pins
+THIN_MUTATIONS = [
+    ("thinning_ratio_inverted", "double a = P[k] > 0.0 ? 1.0 - Q[k] / P[k] : 0.0;",
+     "double a = Q[k] > 0.0 ? 1.0 - P[k] / Q[k] : 0.0;", 0),
+    ("thinning_candidate_from_draft", "int y = inverse_cdf(p, V, (double)tu[3 * r], NULL, &m_tok);",
+     "int y = inverse_cdf(have_Q ? q : p, V, (double)tu[3 * r], NULL, &m_tok);", 0),
+    ("thinning_keep_uses_label_uniform", "keep = (double)tu[3 * r + 2] < a;", "keep = (double)tu[3 * r + 1] < a;", 0),
+    ("thinning_label_uses_token_uniform", "draw_label(y, (double)tu[3 * r + 1], weights,", "draw_label(y, (double)tu[3 * r], weights,", 0),
+    ("thinning_bonus_is_thinned_too", "if (have_Q) { /* thinning probability", "if (1) { /* thinning probability", 0),
+    ("thinning_keeps_with_complement", "keep = (double)tu[3 * r + 2] < a;", "keep = (double)tu[3 * r + 2] >= a;", 0),
+    ("thinning_token_from_draft_conditional", "w[k] = weights ? p[t] * weights[lo + k] : p[t] / (double)tok_degree[t];",
+     "w[k] = weights ? q[t] * weights[lo + k] : q[t] / (double)tok_degree[t];", 0),
+]
+
+THIN_PIN_CALLS = (
+    [lambda o, s=s: thin_pins.test_thinning_group_law_trials_and_token_law(o, s) for s in (11, 13)]
+    + [lambda o, s=s: thin_pins.test_thinning_bonus_is_one_candidate_from_the_target(o, s) for s in (11,)]
+    + [lambda o: thin_pins.test_thinning_with_singleton_groups_is_token_level_residual_sampling(o),
+       lambda o: thin_pins.test_thinning_exhaustion_falls_back_to_the_enumerated_draw(o),
+       lambda o: thin_pins.test_thinning_never_reads_trials_it_does_not_reach(o)]
 )
 
 
@@ -78,8 +102,20 @@ def test_every_planted_mistake_is_caught_by_a_pin(tmp_path, name, old, new, occu
     assert caught, f"no pin noticed the planted mistake '{name}'"
 
 
+@pytest.mark.parametrize("name,old,new,occurrence", THIN_MUTATIONS, ids=[m[0] for m in THIN_MUTATIONS])
+def test_every_planted_thinning_mistake_is_caught_by_a_pin(tmp_path, name, old, new, occurrence):
+    mutant = _mutant(tmp_path, name, old, new, occurrence)
+    caught = []
+    for i, call in enumerate(THIN_PIN_CALLS):
+        try:
+            call(mutant)
+        except AssertionError:
+            caught.append(i)
+    assert caught, f"no pin noticed the planted mistake '{name}'"
+
+
 def test_the_unmodified_copy_passes_every_pin(tmp_path):
     """Control: the same machinery with no mistake planted must pass, so a failure above means the mistake."""
     clean = _mutant(tmp_path, "clean", "double ratio", "double ratio", 0)
-    for call in PIN_CALLS:
+    for call in PIN_CALLS + THIN_PIN_CALLS:
         call(clean)
