@@ -51,6 +51,8 @@ typedef struct CUevent_st *pcg_event;
 #define PCG_FLAG_BAD_DRAFT_TOKEN 1 /* a draft token id outside [0,V) was seen and treated as token 0 */
 #define PCG_FLAG_ZERO_RESIDUAL 2   /* a rejection whose residual mass summed to <= 0; drew from P instead */
 #define PCG_FLAG_NONFINITE 4       /* a row's maximum or normaliser was not finite (NaN/+inf logits, or all -inf) */
+#define PCG_FLAG_THINNING_EXHAUSTED 8 /* pcg_verify_thinning: every supplied trial was turned down; the group was
+                                         drawn from the enumerated residual instead (same law) */
 
 /* Bits of the `mode` argument of pcg_verify. */
 #define PCG_VERIFY_DEFAULT 0u /* per position only the label group's P and Q are formed (what the accept test
@@ -285,6 +287,39 @@ pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits
                              const int32_t *draft_tokens, const pcg_groups *groups, const float *uniforms,
                              float temperature, int32_t *out_accept_len, int32_t *out_tokens, int32_t *out_groups,
                              int32_t *out_flags, pcg_stream stream);
+
+/*
+ * pcg_verify with the paper's own sampler for the terminal group: "Residual sampling via thinning" (Sec. 2.2).
+ *
+ * Everything up to the first rejection is pcg_verify's per-position stage (label, acceptance, first-reject scan).
+ * The group at the rejected position is then drawn WITHOUT enumerating the groups.  Trial r = 0, 1, ... draws a
+ * token y from the target row by inverse CDF in token order with thin_uniforms[b, r, 0], a label k ~ w_{.,y} over
+ * the groups containing y with thin_uniforms[b, r, 1] (so k follows the target's coarse distribution), and keeps
+ * k if thin_uniforms[b, r, 2] < [1 - Q(k)/P(k)]_+ (draft mass over target mass of group k alone); otherwise the
+ * next trial draws a new candidate.  The kept group's law is the normalised residual (P - Q)_+ exactly; the
+ * expected number of trials is 1 / TV(P, Q).  After a sequence whose K positions were all accepted there is no
+ * draft mass: the first candidate is kept (the bonus group, from the target's coarse distribution).  The token
+ * inside the kept group is drawn from the target-conditional p(t) w / P(k) with uniforms[b, K, 1], as in
+ * pcg_verify.  The paper's loop is unbounded; this call runs at most n_trials trials per sequence and, if all
+ * are turned down, draws the group from the enumerated residual with uniforms[b, K, 0] (what pcg_verify does;
+ * same law) and sets PCG_FLAG_THINNING_EXHAUSTED for that sequence.  Results are a deterministic function of
+ * the inputs; they equal pcg_verify's in distribution, not draw by draw (the two consume different uniforms).
+ *
+ *   thin_uniforms [B, n_trials, 3] float in [0,1), device, read-only; 1 <= n_trials <= 65536
+ *   out_trials    [B] int32 or NULL: candidates drawn (1 after an all-accepted sequence; n_trials when exhausted)
+ *   workspace     device, 256-byte aligned, at least pcg_verify_thinning_workspace_bytes(...) bytes (28 bytes per
+ *                 drafted position plus B*M*4 for sequences whose trials run out); contents need no initialisation
+ *   the remaining arguments, ownership, asynchrony (no allocation, no synchronisation, the caller's stream only)
+ *   and errors are pcg_verify's; V is limited by the shared memory the tile prefix needs (8 bytes per 16-byte
+ *   vector of a row: V <= 3.6 million for 16-bit logits), beyond that PCG_ERR_UNSUPPORTED.
+ */
+size_t pcg_verify_thinning_workspace_bytes(int32_t B, int32_t K, int32_t V, int32_t M, pcg_dtype dtype);
+pcg_status pcg_verify_thinning(const void *target_logits, const void *draft_logits, pcg_dtype dtype, int32_t B, int32_t K,
+                               const int32_t *draft_tokens, const pcg_groups *groups, const float *uniforms,
+                               const float *thin_uniforms, int32_t n_trials, float temperature,
+                               int32_t *out_accept_len, int32_t *out_tokens, int32_t *out_groups, int32_t *out_flags,
+                               int32_t *out_trials, void *workspace, size_t workspace_bytes, pcg_stream stream,
+                               const pcg_event *stage_events);
 
 #ifdef __cplusplus
 }

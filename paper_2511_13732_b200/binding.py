@@ -17,7 +17,7 @@ import numpy as np
 from . import build as _build
 
 PCG_F32, PCG_BF16, PCG_F16 = 0, 1, 2
-FLAG_BAD_DRAFT_TOKEN, FLAG_ZERO_RESIDUAL, FLAG_NONFINITE = 1, 2, 4
+FLAG_BAD_DRAFT_TOKEN, FLAG_ZERO_RESIDUAL, FLAG_NONFINITE, FLAG_THINNING_EXHAUSTED = 1, 2, 4, 8
 VERIFY_DEFAULT, VERIFY_DENSE, VERIFY_CLUSTER_TERMINAL, VERIFY_BATCHED_TERMINAL = 0, 1, 2, 4
 STATUS_NAMES = {0: "PCG_OK", 1: "PCG_ERR_INVALID_ARG", 2: "PCG_ERR_INVALID_GROUPS", 3: "PCG_ERR_UNSUPPORTED",
                 4: "PCG_ERR_WORKSPACE", 5: "PCG_ERR_CUDA"}
@@ -95,6 +95,11 @@ def load(build_if_missing: bool = True):
     lib.pcg_verify_host.restype = ctypes.c_int
     lib.pcg_verify_static.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, f32, vp, vp, vp, vp, vp]
     lib.pcg_verify_static.restype = ctypes.c_int
+    lib.pcg_verify_thinning_workspace_bytes.argtypes = [i32, i32, i32, i32, ctypes.c_int]
+    lib.pcg_verify_thinning_workspace_bytes.restype = sz
+    lib.pcg_verify_thinning.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp, vp,
+                                        sz, vp, vp]
+    lib.pcg_verify_thinning.restype = ctypes.c_int
     lib.pcg_asg_create.argtypes = [vp, ctypes.c_int, i32, i32, f32, u32, ctypes.POINTER(vp)]
     lib.pcg_asg_create.restype = ctypes.c_int
     lib.pcg_asg_info.argtypes, lib.pcg_asg_info.restype = [vp, ctypes.POINTER(AsgInfo)], ctypes.c_int
@@ -258,6 +263,52 @@ def pcg_verify_static(target_logits, draft_logits, draft_tokens, groups: Groups,
                                     K1 - 1, _dev_ptr(draft_tokens), groups.handle, _dev_ptr(uniforms),
                                     float(temperature), _dev_ptr(accept_len), _dev_ptr(tokens), _dev_ptr(grp),
                                     _dev_ptr(flags), _stream_ptr(stream)))
+    return out
+
+
+def pcg_verify_thinning_workspace_bytes(B: int, K: int, V: int, M: int, dtype: int) -> int:
+    return int(load().pcg_verify_thinning_workspace_bytes(B, K, V, M, dtype))
+
+
+def pcg_verify_thinning(target_logits, draft_logits, draft_tokens, groups: Groups, uniforms, thin_uniforms,
+                        temperature: float = 1.0, workspace=None, stream=None, out=None, stage_events=None):
+    """``pcg_verify_thinning`` on CUDA tensors: the terminal group by the paper's thinning sampler.
+
+    ``thin_uniforms`` is [B, n_trials, 3] float32.  Returns (accept_len, tokens, groups, flags, trials); ``out``
+    optionally supplies those five tensors (groups, flags and trials may be None).
+    """
+    import torch
+
+    B, K1, V = target_logits.shape
+    K = K1 - 1
+    dev = target_logits.device
+    if thin_uniforms.dim() != 3 or thin_uniforms.shape[0] != B or thin_uniforms.shape[2] != 3:
+        raise ValueError("thin_uniforms must be [B, n_trials, 3]")
+    n_trials = int(thin_uniforms.shape[1])
+    for t, shape in ((draft_logits, (B, K, V)), (draft_tokens, (B, K)), (uniforms, (B, K + 1, 2)),
+                     (thin_uniforms, (B, n_trials, 3))):
+        if tuple(t.shape) != shape or not t.is_contiguous() or t.device != dev:
+            raise ValueError(f"expected a contiguous tensor of shape {shape} on {dev}")
+    if not target_logits.is_contiguous() or draft_logits.dtype != target_logits.dtype:
+        raise ValueError("target and draft logits must be contiguous and share a dtype")
+    if draft_tokens.dtype != torch.int32 or uniforms.dtype != torch.float32 or thin_uniforms.dtype != torch.float32:
+        raise TypeError("draft_tokens must be int32 and the uniforms float32")
+    dt = dtype_code(target_logits)
+    if workspace is None:
+        workspace = torch.empty(pcg_verify_thinning_workspace_bytes(B, K, V, groups.M, dt), dtype=torch.uint8, device=dev)
+    if out is None:
+        out = (torch.empty(B, dtype=torch.int32, device=dev), torch.empty((B, K + 1), dtype=torch.int32, device=dev),
+               torch.empty((B, K + 1), dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev),
+               torch.empty(B, dtype=torch.int32, device=dev))
+    accept_len, tokens, grp, flags, trials = out
+    ev = None
+    if stage_events is not None:
+        ev = (ctypes.c_void_p * 3)(*[ctypes.c_void_p(e.cuda_event) for e in stage_events])
+    _check(load().pcg_verify_thinning(_dev_ptr(target_logits), _dev_ptr(draft_logits), dt, B, K, _dev_ptr(draft_tokens),
+                                      groups.handle, _dev_ptr(uniforms), _dev_ptr(thin_uniforms), n_trials,
+                                      float(temperature), _dev_ptr(accept_len), _dev_ptr(tokens), _dev_ptr(grp),
+                                      _dev_ptr(flags), _dev_ptr(trials), _dev_ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream_ptr(stream), ev))
     return out
 
 

@@ -1158,6 +1158,89 @@ struct DrawArgs {
 
 __device__ __forceinline__ int own_slot(int j) { return j + (j >> 5); }  // one pad word per 32: chunked reads spread over banks
 
+// Token inside the drawn group `gsel`: target-conditional p(t) w / P[g] over the group's CSR order, by inverse
+// CDF with `u_token` (whole block; dscratch: 32 doubles, scratch: 64 floats, ibox: 8 ints of shared memory).
+// Only ratios inside the group matter, so the terms are taken relative to the group's largest logit.
+template <typename T, int NT>
+__device__ __forceinline__ int draw_token_in_group(const GroupsDev &G, const T *trow, int gsel, float s, float u_token,
+                                                   double *dscratch, float *scratch, int *ibox, int &flags) {
+    const int tid = threadIdx.x;
+    const int lo = G.group_ptr[gsel], hi = G.group_ptr[gsel + 1], len = hi - lo;
+    const int per2 = (len + NT - 1) / NT;
+    const int k0 = min(len, tid * per2), k1 = min(len, k0 + per2);
+    float mloc = kNegInf;
+    for (int k = k0; k < k1; ++k) mloc = fmaxf(mloc, Elem<T>::widen(trow[G.group_tok[lo + k]]));
+    const float mg = block_max<NT>(mloc, scratch);
+    const float rs = mg > kNegInf ? mg * s : 0.f;
+    auto omega = [&](int k) -> float {
+        const int t = G.group_tok[lo + k];
+        const float w = G.pair_w ? G.pair_w[lo + k] : G.inv_deg[t];
+        return __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs)), w);
+    };
+    double wsum = 0.0;
+    int wlast = -1;
+    for (int k = k0; k < k1; ++k) {
+        const float w = omega(k);
+        wsum += (double)w;
+        if (w > 0.f) wlast = k;
+    }
+    double excl, incl, wtot;
+    block_scan<NT>(wsum, dscratch, &excl, &incl, &wtot);
+    if (tid == 0) {
+        ibox[2] = NT;
+        ibox[3] = -1;
+        ibox[4] = -1;
+    }
+    __syncthreads();
+    const double target2 = (double)u_token * wtot;
+    if (wlast >= 0) atomicMax(&ibox[3], wlast);
+    if (wsum > 0.0 && incl > target2) atomicMin(&ibox[2], tid);
+    __syncthreads();
+    if (ibox[2] == tid) {
+        double loc = 0.0;
+        int pick = wlast;
+        for (int k = k0; k < k1; ++k) {
+            loc += (double)omega(k);
+            if (excl + loc > target2) {
+                pick = k;
+                break;
+            }
+        }
+        ibox[4] = pick;
+    }
+    __syncthreads();
+    const int ksel = ibox[4] >= 0 ? ibox[4] : ibox[3];
+    if (ksel >= 0) return G.group_tok[lo + ksel];
+    flags |= PCG_FLAG_NONFINITE;  // the drawn group has no token with target mass (non-finite inputs)
+    return len > 0 ? G.group_tok[lo] : 0;
+}
+
+// Outputs of sequence b: accepted draft tokens, the drawn token z of group gsel at position n, then filler.
+template <int NT>
+__device__ __forceinline__ void emit_sequence(const GroupsDev &G, int b, int K, int n, int z, int gsel, int flags,
+                                              const int32_t *draft_tokens, const int32_t *labels,
+                                              int32_t *out_accept_len, int32_t *out_tokens, int32_t *out_groups,
+                                              int32_t *out_flags) {
+    const int tid = threadIdx.x;
+    for (int i = tid; i <= K; i += NT) {
+        int tok = -1, grp = -1;
+        if (i < n) {
+            tok = draft_tokens[b * K + i];
+            if (tok < 0 || tok >= G.V) tok = 0;  // verified as token 0 (and flagged), so emitted as token 0
+            grp = labels[b * K + i];
+        } else if (i == n) {
+            tok = z;
+            grp = gsel;
+        }
+        out_tokens[(int64_t)b * (K + 1) + i] = tok;
+        if (out_groups) out_groups[(int64_t)b * (K + 1) + i] = grp;
+    }
+    if (tid == 0) {
+        out_accept_len[b] = n;
+        if (out_flags) out_flags[b] = flags;
+    }
+}
+
 // One block per sequence.  Shared memory: the M clamped residual masses (padded), then scratch.
 template <typename T, bool DENSE>
 __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a, GroupsDev G) {
@@ -1258,78 +1341,10 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
         gsel = 0;
         flags |= PCG_FLAG_NONFINITE;
     } else {
-        // ---- token inside the drawn group: target-conditional p(t) w / P[g] over the group's CSR order.
-        // Only ratios inside the group matter, so the terms are taken relative to the group's largest logit.
-        const int lo = G.group_ptr[gsel], hi = G.group_ptr[gsel + 1], len = hi - lo;
-        const int per2 = (len + NT - 1) / NT;
-        const int k0 = min(len, tid * per2), k1 = min(len, k0 + per2);
-        float mloc = kNegInf;
-        for (int k = k0; k < k1; ++k) mloc = fmaxf(mloc, Elem<T>::widen(trow[G.group_tok[lo + k]]));
-        const float mg = block_max<NT>(mloc, scratch);
-        const float rs = mg > kNegInf ? mg * a.s : 0.f;
-        auto omega = [&](int k) -> float {
-            const int t = G.group_tok[lo + k];
-            const float w = G.pair_w ? G.pair_w[lo + k] : G.inv_deg[t];
-            return __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs)), w);
-        };
-        double wsum = 0.0;
-        int wlast = -1;
-        for (int k = k0; k < k1; ++k) {
-            const float w = omega(k);
-            wsum += (double)w;
-            if (w > 0.f) wlast = k;
-        }
-        double excl, incl, wtot;
-        block_scan<NT>(wsum, dscratch, &excl, &incl, &wtot);
-        if (tid == 0) {
-            ibox[2] = NT;
-            ibox[3] = -1;
-            ibox[4] = -1;
-        }
-        __syncthreads();
-        const double target2 = (double)u_token * wtot;
-        if (wlast >= 0) atomicMax(&ibox[3], wlast);
-        if (wsum > 0.0 && incl > target2) atomicMin(&ibox[2], tid);
-        __syncthreads();
-        if (ibox[2] == tid) {
-            double loc = 0.0;
-            int pick = wlast;
-            for (int k = k0; k < k1; ++k) {
-                loc += (double)omega(k);
-                if (excl + loc > target2) {
-                    pick = k;
-                    break;
-                }
-            }
-            ibox[4] = pick;
-        }
-        __syncthreads();
-        const int ksel = ibox[4] >= 0 ? ibox[4] : ibox[3];
-        if (ksel >= 0) {
-            z = G.group_tok[lo + ksel];
-        } else {  // the drawn group has no token with target mass (non-finite inputs)
-            z = len > 0 ? G.group_tok[lo] : 0;
-            flags |= PCG_FLAG_NONFINITE;
-        }
+        z = draw_token_in_group<T, NT>(G, trow, gsel, a.s, u_token, dscratch, scratch, ibox, flags);
     }
-    // ---- emit: accepted draft tokens, the drawn token, then filler ----
-    for (int i = tid; i <= K; i += NT) {
-        int tok = -1, grp = -1;
-        if (i < n) {
-            tok = a.draft_tokens[b * K + i];
-            if (tok < 0 || tok >= V) tok = 0;  // verified as token 0 (and flagged), so emitted as token 0
-            grp = a.labels[b * K + i];
-        } else if (i == n) {
-            tok = z;
-            grp = gsel;
-        }
-        a.out_tokens[(int64_t)b * (K + 1) + i] = tok;
-        if (a.out_groups) a.out_groups[(int64_t)b * (K + 1) + i] = grp;
-    }
-    if (tid == 0) {
-        a.out_accept_len[b] = n;
-        if (a.out_flags) a.out_flags[b] = flags;
-    }
+    emit_sequence<NT>(G, b, K, n, z, gsel, flags, a.draft_tokens, a.labels, a.out_accept_len, a.out_tokens, a.out_groups,
+                      a.out_flags);
 }
 
 // ---------------------------------------------------------------- dense mode: accept test from full P, Q -----
@@ -1482,6 +1497,8 @@ static void launch_spmm(const SpmmArgs &sp, int nb, bool wide, const GroupsDev &
             group_spmm_kernel<1, 16, false><<<grid, kSpmmThreads, 0, cs>>>(sp, G);
     }
 }
+
+#include "pcg_thinning.cuh"
 
 }  // namespace pcg
 
@@ -1667,6 +1684,116 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
                                             : launch_draw(terminal_draw_kernel<LogitT, false>));
         if (e != cudaSuccess) return cuda_fail(e, "launching terminal_draw_kernel");
     }
+    if (stage_events) {
+        e = cudaEventRecord((cudaEvent_t)stage_events[2], cs);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    }
+    return PCG_OK;
+}
+
+// ================================================================ verification with the thinning sampler ====
+
+namespace pcg {
+struct ThinWorkspace {
+    int32_t *accept, *labels, *posflags;
+    float4 *stats;
+    float *fallback_rows;
+    size_t bytes;
+};
+static ThinWorkspace carve_thin_workspace(void *base, int64_t B, int64_t K, int64_t M) {
+    ThinWorkspace w = {};
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = off;
+        off = (off + bytes + 255) & ~(size_t)255;
+        return at;
+    };
+    char *p = (char *)base;
+    w.stats = (float4 *)(p + take((size_t)(B * K) * 16));
+    w.accept = (int32_t *)(p + take((size_t)(B * K) * 4));
+    w.labels = (int32_t *)(p + take((size_t)(B * K) * 4));
+    w.posflags = (int32_t *)(p + take((size_t)(B * K) * 4));
+    w.fallback_rows = (float *)(p + take((size_t)(B * M) * 4));
+    w.bytes = off ? off : 256;
+    return w;
+}
+}  // namespace pcg
+
+extern "C" size_t pcg_verify_thinning_workspace_bytes(int32_t B, int32_t K, int32_t V, int32_t M, pcg_dtype dtype) {
+    (void)dtype;
+    if (B < 0 || K < 0 || V < 1 || M < 1) return 256;
+    return carve_thin_workspace(nullptr, B, K, M).bytes;
+}
+
+extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void *draft_logits, pcg_dtype dtype, int32_t B,
+                                          int32_t K, const int32_t *draft_tokens, const pcg_groups *groups,
+                                          const float *uniforms, const float *thin_uniforms, int32_t n_trials,
+                                          float temperature, int32_t *out_accept_len, int32_t *out_tokens,
+                                          int32_t *out_groups, int32_t *out_flags, int32_t *out_trials, void *workspace,
+                                          size_t workspace_bytes, pcg_stream stream, const pcg_event *stage_events) {
+    pcg_status st = check_common(groups, dtype, temperature, "pcg_verify_thinning");
+    if (st != PCG_OK) return st;
+    if (B < 0 || K < 1 || n_trials < 1) {
+        set_error("pcg_verify_thinning: need B >= 0, K >= 1 and n_trials >= 1 (B=%d K=%d n_trials=%d)", B, K, n_trials);
+        return PCG_ERR_INVALID_ARG;
+    }
+    if (K > 1024 || n_trials > 65536) {
+        set_error("pcg_verify_thinning: K=%d or n_trials=%d exceeds the supported 1024 positions / 65536 trials", K, n_trials);
+        return PCG_ERR_UNSUPPORTED;
+    }
+    if (B == 0) return PCG_OK;
+    if (!target_logits || !draft_logits || !draft_tokens || !uniforms || !thin_uniforms || !out_accept_len || !out_tokens) {
+        set_error("pcg_verify_thinning: null pointer");
+        return PCG_ERR_INVALID_ARG;
+    }
+    const GroupsDev &G = groups->dev;
+    const size_t esz = dtype_bytes(dtype);
+    if (((uintptr_t)target_logits % esz) || ((uintptr_t)draft_logits % esz)) {
+        set_error("pcg_verify_thinning: logits pointers must be aligned to their element size");
+        return PCG_ERR_INVALID_ARG;
+    }
+    if ((int64_t)B * (K + 1) > INT32_MAX / 8) {
+        set_error("pcg_verify_thinning: B*K too large for one launch");
+        return PCG_ERR_UNSUPPORTED;
+    }
+    const size_t smem = thin_smem_bytes(G.V, esz);
+    if (smem > kMaxDynSmem) {
+        set_error("pcg_verify_thinning: V=%d needs %zu bytes of shared memory for the tile prefix (limit %zu)", G.V, smem,
+                  kMaxDynSmem);
+        return PCG_ERR_UNSUPPORTED;
+    }
+    const size_t need = pcg_verify_thinning_workspace_bytes(B, K, G.V, G.M, dtype);
+    if (!workspace || ((uintptr_t)workspace & 255u) || workspace_bytes < need) {
+        set_error("pcg_verify_thinning: workspace must be 256-byte aligned and hold %zu bytes (got %zu)", need,
+                  workspace_bytes);
+        return PCG_ERR_WORKSPACE;
+    }
+    cudaStream_t cs = (cudaStream_t)stream;
+    const ThinWorkspace w = carve_thin_workspace(workspace, B, K, G.M);
+    const float s = (float)((double)kLog2e / (double)temperature);
+    cudaError_t e = cudaSuccess;
+    if (stage_events) e = cudaEventRecord((cudaEvent_t)stage_events[0], cs);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
+                    w.accept,      w.labels,     w.posflags,   w.stats};
+    PCG_DISPATCH_DTYPE(dtype, position_kernel<LogitT><<<B * K, kPosThreads, 0, cs>>>(pa, G));
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
+    if (stage_events) {
+        e = cudaEventRecord((cudaEvent_t)stage_events[1], cs);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    }
+    ThinArgs ta{target_logits, draft_logits, draft_tokens, uniforms,        thin_uniforms, n_trials,
+                K,             s,            w.accept,     w.labels,        w.posflags,    w.stats,
+                w.fallback_rows, out_accept_len, out_tokens, out_groups,    out_flags,     out_trials};
+    auto launch = [&](auto kern) -> cudaError_t {
+        cudaError_t le = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (le != cudaSuccess) return le;
+        kern<<<B, kThinThreads, smem, cs>>>(ta, G);
+        return cudaGetLastError();
+    };
+    PCG_DISPATCH_DTYPE(dtype, e = launch(thinning_kernel<LogitT>));
+    if (e != cudaSuccess) return cuda_fail(e, "launching thinning_kernel");
     if (stage_events) {
         e = cudaEventRecord((cudaEvent_t)stage_events[2], cs);
         if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");

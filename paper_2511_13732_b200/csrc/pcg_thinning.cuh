@@ -1,0 +1,350 @@
+// Terminal group by thinning ("Residual sampling via thinning", Sec. 2.2) -- included by pcg_kernels.cu inside
+// namespace pcg, after the helpers of the batched terminal stage.
+//
+// The paper's sampler never enumerates the groups: a candidate (y, k) is drawn with y ~ target and k ~ w_{.,y}
+// (so k follows the target's coarse distribution) and kept with probability [1 - Q(k)/P(k)]_+, which needs the
+// two masses of group k only.  One block per sequence:
+//   1. first rejection n from the accept bits (warp ballots); row statistics from the position kernel, or, when
+//      every position was accepted, one pass over the bonus row;
+//   2. one streaming pass over the target row of position n: the sum of 2^(l s - RS) over every tile of
+//      32 x 16 bytes, kept in shared memory as an inclusive prefix (double) -- the token-level CDF at tile
+//      granularity;
+//   3. trials, one WARP per trial and all warps at once: binary search for the tile, re-read of that tile (it
+//      sits in L2), in-tile scan for y, label k, the two masses of group k by a warp gather, keep test.  The
+//      first kept candidate in trial order wins, so the result is the sequential sampler's although several
+//      trials run side by side;
+//   4. token inside the kept group and outputs, as in the enumerated path.
+// If all supplied trials are turned down, the block enumerates the residual itself (one thread per group,
+// staged in a row of the workspace) and draws from it with the sequence's terminal-group uniform: same law,
+// flagged PCG_FLAG_THINNING_EXHAUSTED.
+
+constexpr int kThinThreads = 512;
+
+struct ThinArgs {
+    const void *target;           // [B, K+1, V]
+    const void *draft;            // [B, K, V]
+    const int32_t *draft_tokens;  // [B, K]
+    const float *uniforms;        // [B, K+1, 2]
+    const float *thin;            // [B, n_trials, 3]: token, label and keep uniform of every trial
+    int n_trials;
+    int K;
+    float s;
+    const int32_t *accept, *labels, *posflags;  // [B*K] from the position kernel
+    const float4 *stats;                        // [B*K]
+    float *fallback_rows;                       // [B, M] staging for sequences whose trials ran out
+    int32_t *out_accept_len, *out_tokens, *out_groups, *out_flags, *out_trials;
+};
+
+static size_t thin_smem_bytes(int V, size_t esz) {
+    const size_t ts = 32 * (16 / esz);
+    return ((size_t)V + ts - 1) / ts * 8 + 32 * 8 + 64 * 4 + 8 * 4 + (kThinThreads / 32) * 4;
+}
+
+// 2^(l s - rs) of this lane's share (one 16-byte vector) of tile `tile` of `row`; zero past the end of the row.
+template <typename T>
+__device__ __forceinline__ void thin_lane_terms(const T *row, int V, int tile, int lane, bool vec_ok, float s, float rs,
+                                                float (&e)[Elem<T>::kPerVec]) {
+    constexpr int NV = Elem<T>::kPerVec;
+    const int t0 = (tile * 32 + lane) * NV;
+    if (vec_ok && t0 + NV <= V) {
+        float v[NV];
+        Elem<T>::unpack(ld_stream(reinterpret_cast<const uint4 *>(row + t0)), v);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) e[i] = ex2(__fmaf_rn(v[i], s, -rs));
+    } else {
+#pragma unroll
+        for (int i = 0; i < NV; ++i) e[i] = t0 + i < V ? ex2(__fmaf_rn(Elem<T>::widen(row[t0 + i]), s, -rs)) : 0.f;
+    }
+}
+
+template <int NV>
+__device__ __forceinline__ float thin_lane_sum(const float (&e)[NV]) {
+    float v = e[0];
+#pragma unroll
+    for (int i = 1; i < NV; ++i) v += e[i];
+    return v;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, GroupsDev G) {
+    constexpr int NT = kThinThreads, NW = NT / 32, NV = Elem<T>::kPerVec, TS = 32 * NV;
+    extern __shared__ __align__(16) unsigned char raw[];
+    __shared__ int s_n, s_flags;
+    const int V = G.V, M = G.M, K = a.K;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int ntiles = (V + TS - 1) / TS;
+    double *tile_incl = reinterpret_cast<double *>(raw);        // [ntiles] inclusive prefix of the tile sums
+    double *dscratch = tile_incl + ntiles;                      // 32 doubles
+    float *scratch = reinterpret_cast<float *>(dscratch + 32);  // 64 floats
+    int *ibox = reinterpret_cast<int *>(scratch + 64);          // 8 ints
+    int *cand = ibox + 8;                                       // NW ints: group kept by each warp's trial, or -1
+
+    // ---- 1. first rejected position and the flags of the positions up to it ----
+    if (tid < 32) {
+        int n = K, flags = 0;
+        for (int base = 0; base < K && n == K; base += 32) {
+            const int i = base + tid;
+            const int rej = (i < K) && (a.accept[b * K + i] == 0);
+            const unsigned mask = __ballot_sync(0xffffffffu, rej);
+            if (mask) n = base + __ffs(mask) - 1;
+        }
+        for (int base = 0; base < K && base <= n; base += 32) {
+            const int i = base + tid;
+            const int f = (i < K && i <= n) ? a.posflags[b * K + i] : 0;
+            flags |= __reduce_or_sync(0xffffffffu, f);
+        }
+        if (tid == 0) {
+            s_n = n;
+            s_flags = flags;
+        }
+    }
+    __syncthreads();
+    const int n = s_n;
+    int flags = s_flags;
+    const bool residual = n < K;  // false: every position accepted, the terminal draw is the bonus token
+    const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
+    const T *qrow = reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(n, K - 1)) * V;
+    const bool vec_ok = ((uintptr_t)trow & 15u) == 0;
+    float rs_p, iz_p, rs_q = 0.f, iz_q = 0.f;
+    if (residual) {
+        const float4 st = a.stats[b * K + n];
+        rs_p = st.x, iz_p = st.y, rs_q = st.z, iz_q = st.w;
+    } else {
+        // statistics of the bonus row: one pass with a per-thread reference, merged over the block
+        RefSum st{kRefInit * a.s, 0.f};
+        for (int tile = warp; tile < ntiles; tile += NW) {
+            const int t0 = (tile * 32 + lane) * NV;
+            if (vec_ok && t0 + NV <= V) {
+                float v[NV];
+                Elem<T>::unpack(ld_stream(reinterpret_cast<const uint4 *>(trow + t0)), v);
+                absorb<NV>(st, v, a.s);
+            } else {
+                for (int i = 0; i < NV && t0 + i < V; ++i) absorb1(st, Elem<T>::widen(trow[t0 + i]), a.s);
+            }
+        }
+        float rs = st.rs, Z = st.acc;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) merge(rs, Z, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, Z, o));
+        if (lane == 0) {
+            scratch[2 * warp] = rs;
+            scratch[2 * warp + 1] = Z;
+        }
+        __syncthreads();
+        rs = scratch[0];
+        Z = scratch[1];
+        for (int w = 1; w < NW; ++w) merge(rs, Z, scratch[2 * w], scratch[2 * w + 1]);
+        __syncthreads();
+        if (!(Z > 0.f) || isinf(Z) || isinf(rs)) flags |= PCG_FLAG_NONFINITE;
+        rs_p = rs;
+        iz_p = 1.0f / Z;
+    }
+
+    // ---- 2. tile sums of the target row (four tiles of loads in flight per warp), then their prefix ----
+    for (int base = warp; base < ntiles; base += 4 * NW) {
+        uint4 r[4];
+        bool fast[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int tile = base + j * NW;
+            const int t0 = (tile * 32 + lane) * NV;
+            fast[j] = tile < ntiles && vec_ok && t0 + NV <= V;
+            if (fast[j]) r[j] = ld_stream(reinterpret_cast<const uint4 *>(trow + t0));
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int tile = base + j * NW;
+            if (tile >= ntiles) continue;  // (warp-uniform)
+            float e[NV];
+            if (fast[j]) {
+                float v[NV];
+                Elem<T>::unpack(r[j], v);
+#pragma unroll
+                for (int i = 0; i < NV; ++i) e[i] = ex2(__fmaf_rn(v[i], a.s, -rs_p));
+            } else {
+                thin_lane_terms<T>(trow, V, tile, lane, false, a.s, rs_p, e);
+            }
+            float sum = thin_lane_sum<NV>(e);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (lane == 0) tile_incl[tile] = (double)sum;
+        }
+    }
+    __syncthreads();
+    double Ztot;
+    {
+        const int per = (ntiles + NT - 1) / NT;
+        const int i0 = min(ntiles, tid * per), i1 = min(ntiles, i0 + per);
+        double my = 0.0, excl, incl;
+        for (int j = i0; j < i1; ++j) my += tile_incl[j];
+        block_scan<NT>(my, dscratch, &excl, &incl, &Ztot);
+        double run = excl;
+        for (int j = i0; j < i1; ++j) {
+            run += tile_incl[j];
+            tile_incl[j] = run;
+        }
+    }
+    __syncthreads();
+
+    // ---- 3. trials: warp w of round r0 runs trial r0 + w; the first kept candidate in trial order wins ----
+    int gsel = -1, used = 0;
+    const bool usable = Ztot > 0.0 && Ztot < (double)__builtin_huge_valf();
+    if (!usable) flags |= PCG_FLAG_NONFINITE;
+    const float *tu = a.thin + (size_t)b * a.n_trials * 3;
+    const int max_trials = usable ? (residual ? a.n_trials : 1) : 0;
+    for (int r0 = 0; r0 < max_trials && gsel < 0; r0 += NW) {
+        const int r = r0 + warp;
+        int kept = -1;
+        if (r < max_trials) {
+            const float u_tok = tu[3 * r], u_lab = tu[3 * r + 1], u_keep = tu[3 * r + 2];
+            // token y ~ target: tile by binary search over the prefix, then a scan inside the tile
+            const double target = (double)u_tok * Ztot;
+            int lo = 0, hi = ntiles - 1;  // the last tile's prefix is the total, which exceeds u * total for u < 1
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (tile_incl[mid] > target)
+                    hi = mid;
+                else
+                    lo = mid + 1;
+            }
+            const int tile = lo;
+            const double tl = target - (tile > 0 ? tile_incl[tile - 1] : 0.0);
+            float e[NV];
+            thin_lane_terms<T>(trow, V, tile, lane, vec_ok, a.s, rs_p, e);
+            const float lsum = thin_lane_sum<NV>(e);
+            double inc = (double)lsum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += up;
+            }
+            const unsigned above = __ballot_sync(0xffffffffu, lsum > 0.f && inc > tl);
+            const unsigned massy = __ballot_sync(0xffffffffu, lsum > 0.f);
+            // rounding may leave no lane above the target: then the last lane with mass, and its last element with mass
+            const int L = above ? __ffs(above) - 1 : (massy ? 31 - __clz(massy) : 0);
+            int pick = 0;
+            if (lane == L) {
+                double loc = inc - (double)lsum;
+                int last = 0;
+                bool found = false;
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    loc += (double)e[i];
+                    if (e[i] > 0.f) {
+                        if (!found) last = i;
+                        if (!found && loc > tl) found = true;
+                    }
+                }
+                pick = last;
+            }
+            pick = __shfl_sync(0xffffffffu, pick, L);
+            int y = (tile * 32 + L) * NV + pick;
+            if (y >= V) y = V - 1;
+            // label k ~ w_{.,y}
+            const int rv0 = G.rev_ptr[y];
+            const int g = draw_label(G, rv0, G.rev_ptr[y + 1] - rv0, u_lab);
+            bool keep = true;
+            if (residual) {
+                // the two masses of group g (a warp gather over its tokens), then u < [1 - Q/P]_+ without a division
+                const int k_lo = G.group_ptr[g], k_hi = G.group_ptr[g + 1];
+                float Sp = 0.f, Sq = 0.f;
+                for (int k = k_lo + lane; k < k_hi; k += 32) {
+                    const int t = G.group_tok[k];
+                    const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
+                    Sp += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs_p)), w);
+                    Sq += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), a.s, -rs_q)), w);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    Sp += __shfl_xor_sync(0xffffffffu, Sp, o);
+                    Sq += __shfl_xor_sync(0xffffffffu, Sq, o);
+                }
+                const float P = __fmul_rn(Sp, iz_p), Q = __fmul_rn(Sq, iz_q);
+                keep = __fmul_rn(u_keep, P) < P - Q;
+            }
+            kept = keep ? g : -1;
+        }
+        if (lane == 0) cand[warp] = kept;
+        __syncthreads();
+        used = min(r0 + NW, max_trials);
+        for (int w = 0; w < NW; ++w)
+            if (cand[w] >= 0) {
+                gsel = cand[w];
+                used = r0 + w + 1;
+                break;
+            }
+        __syncthreads();
+    }
+
+    // ---- every supplied trial was turned down: enumerate the residual and invert its CDF (same law) ----
+    if (usable && gsel < 0) {
+        flags |= PCG_FLAG_THINNING_EXHAUSTED;
+        float *own = a.fallback_rows + (size_t)b * M;
+        const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
+        const int per = (M + NT - 1) / NT;
+        const int i0 = min(M, tid * per), i1 = min(M, i0 + per);
+        double Zr = 0.0, excl = 0.0, incl = 0.0, my = 0.0;
+        bool minus_q = true;
+        for (int attempt = 0; attempt < 2; ++attempt) {
+            for (int g = tid; g < M; g += NT) {
+                float acc = 0.f;
+                for (int k = G.group_ptr[g]; k < G.group_ptr[g + 1]; ++k) {
+                    const int t = G.group_tok[k];
+                    const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
+                    float d = __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs_p)), iz_p);
+                    if (minus_q) d -= __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), a.s, -rs_q)), iz_q);
+                    acc += __fmul_rn(d, w);
+                }
+                own[g] = fmaxf(acc, 0.f);
+            }
+            __syncthreads();
+            my = 0.0;
+            for (int j = i0; j < i1; ++j) my += (double)own[j];
+            block_scan<NT>(my, dscratch, &excl, &incl, &Zr);
+            if (Zr > 0.0 || !minus_q) break;
+            flags |= PCG_FLAG_ZERO_RESIDUAL;  // the residual vanished (P == Q to rounding): draw from P instead
+            minus_q = false;
+            __syncthreads();
+        }
+        const double target = (double)u_group * Zr;
+        if (tid == 0) {
+            ibox[2] = NT;
+            ibox[3] = -1;
+            ibox[4] = -1;
+        }
+        __syncthreads();
+        int my_last = -1;
+        for (int j = i0; j < i1; ++j)
+            if (own[j] > 0.f) my_last = j;
+        if (my_last >= 0) atomicMax(&ibox[3], my_last);
+        if (my > 0.0 && incl > target) atomicMin(&ibox[2], tid);
+        __syncthreads();
+        if (ibox[2] == tid) {
+            double loc = 0.0;
+            int pick = my_last;
+            for (int j = i0; j < i1; ++j) {
+                loc += (double)own[j];
+                if (excl + loc > target) {
+                    pick = j;
+                    break;
+                }
+            }
+            ibox[4] = pick;
+        }
+        __syncthreads();
+        gsel = ibox[4] >= 0 ? ibox[4] : ibox[3];
+        __syncthreads();
+    }
+
+    // ---- 4. token inside the kept group, outputs ----
+    int z = 0;
+    if (gsel < 0) {  // no mass anywhere (non-finite inputs): emit group 0 / token 0 and flag it
+        gsel = 0;
+        flags |= PCG_FLAG_NONFINITE;
+    } else {
+        const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
+        z = draw_token_in_group<T, NT>(G, trow, gsel, a.s, u_token, dscratch, scratch, ibox, flags);
+    }
+    emit_sequence<NT>(G, b, K, n, z, gsel, flags, a.draft_tokens, a.labels, a.out_accept_len, a.out_tokens, a.out_groups,
+                      a.out_flags);
+    if (tid == 0 && a.out_trials) a.out_trials[b] = used;
+}

@@ -22,7 +22,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 SEED0 = 251113732
-_STREAM_EMB, _STREAM_CENT, _STREAM_SEQ, _STREAM_GROUPS = 0, 1, 2, 3
+_STREAM_EMB, _STREAM_CENT, _STREAM_SEQ, _STREAM_GROUPS, _STREAM_THIN = 0, 1, 2, 3, 4
 
 
 @dataclass(frozen=True)
@@ -309,6 +309,19 @@ def make_batch(cfg: Config, B: Optional[int] = None, seqs: Optional[Sequence[int
         for i in range(n):
             fill(i)
     return Batch(tl, dl, x, u, cfg.temperature, cfg.dtype)
+
+
+def make_thin_uniforms(cfg: Config, n_trials: int, B: Optional[int] = None, seqs: Optional[Sequence[int]] = None) -> np.ndarray:
+    """Uniforms of the thinning trials, [n, n_trials, 3] float32 multiples of 2^-24 in [0, 1): per trial the
+    token, label and keep draw.  A pure function of (config, sequence index), like the other inputs."""
+    if seqs is None:
+        seqs = range(cfg.B if B is None else B)
+    seqs = list(seqs)
+    out = np.empty((len(seqs), n_trials, 3), np.float32)
+    for i, b in enumerate(seqs):
+        rng = _rng(cfg.cfg_id, _STREAM_THIN, b)
+        out[i] = rng.integers(0, 1 << 24, size=(n_trials, 3)).astype(np.float32) * np.float32(2.0 ** -24)
+    return out
 
 
 def scaled(cfg: Config, **kw) -> Config:
