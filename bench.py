@@ -34,7 +34,7 @@ UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
 # dram__bytes_read.sum + dram__bytes_write.sum of one position_kernel launch, from the ncu capture summarised in
 # profiles/ (null until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {"C5": 1076212992 + 12269056}
+NCU_TRAFFIC_BYTES = {"C5": 1076079104 + 12456448}
 
 
 def hbm_peak():
@@ -186,8 +186,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C5", choices=sorted(W.CONFIGS))
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size B (profiling only)")
-    ap.add_argument("--mode", default="default", choices=["default", "dense", "cluster", "batched"],
-                    help="pcg_verify mode of the timed steps (the headline is 'default')")
+    ap.add_argument("--mode", default="default", choices=["default", "dense", "cluster", "batched", "thinning"],
+                    help="pcg_verify mode of the timed steps (the headline is 'default'); 'thinning' times "
+                         "pcg_verify_thinning (the paper's sampler for the terminal group) instead")
+    ap.add_argument("--thin-trials", type=int, default=32, help="trials supplied per sequence to pcg_verify_thinning")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-modes", action="store_true", help="skip the brief timing of the other pcg_verify modes")
@@ -242,13 +244,24 @@ def main():
     dt_code = binding.PCG_BF16 if bf16 else binding.PCG_F32
     mode_codes = {"default": binding.VERIFY_DEFAULT, "dense": binding.VERIFY_DENSE,
                   "cluster": binding.VERIFY_CLUSTER_TERMINAL, "batched": binding.VERIFY_BATCHED_TERMINAL}
-    mode = mode_codes[args.mode]
+    thinning = args.mode == "thinning"
+    mode = mode_codes.get(args.mode, binding.VERIFY_DEFAULT)
     ws = torch.empty(binding.pcg_verify_workspace_bytes(B, K, V, M, dt_code, mode), dtype=torch.uint8, device="cuda")
     out = (torch.empty(B, dtype=torch.int32, device="cuda"), torch.empty((B, K + 1), dtype=torch.int32, device="cuda"),
            torch.empty((B, K + 1), dtype=torch.int32, device="cuda"), torch.empty(B, dtype=torch.int32, device="cuda"))
     esz = 2 if bf16 else 4
+    # pcg_verify_thinning: its own trial uniforms, workspace and a fifth output (trials drawn per sequence)
+    thin_u = torch.from_numpy(W.make_thin_uniforms(cfg, args.thin_trials, seqs=seqs)).cuda()
+    thin_ws = torch.empty(binding.pcg_verify_thinning_workspace_bytes(B, K, V, M, dt_code), dtype=torch.uint8, device="cuda")
+    thin_out = tuple(torch.empty_like(t) for t in out) + (torch.empty(B, dtype=torch.int32, device="cuda"),)
+
+    def thin_step(events=None):
+        binding.pcg_verify_thinning(tl, dl, x, handle, u, thin_u, cfg.temperature, workspace=thin_ws, out=thin_out,
+                                    stage_events=events)
 
     def step(events=None):
+        if thinning:
+            return thin_step(events)
         binding.pcg_verify(tl, dl, x, handle, u, cfg.temperature, workspace=ws, out=out, stage_events=events,
                            mode=mode)
 
@@ -259,8 +272,10 @@ def main():
 
     for _ in range(max(args.warmup, 3)):
         step()
-    # stage events of every timed step (recorded once here so that their handles exist)
-    stage = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    # stage events on every 8th timed step (recorded once here so that their handles exist): an event between two
+    # kernels costs a drain of the first one, 7 us per call at C5 when every step carries them
+    STAGE_EVERY = 8
+    stage = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(-(-args.steps // STAGE_EVERY))]
     for evs in stage:
         for e in evs:
             e.record()
@@ -269,7 +284,7 @@ def main():
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_begin.record()
     for i in range(args.steps):
-        step(stage[i])
+        step(stage[i // STAGE_EVERY] if i % STAGE_EVERY == 0 else None)
     t_end.record()
     barrier()
     clocks = sampler.stop()
@@ -277,7 +292,7 @@ def main():
     ms_step = ms_total / args.steps
     pos_ms = statistics.fmean(e[0].elapsed_time(e[1]) for e in stage)
     term_ms = statistics.fmean(e[1].elapsed_time(e[2]) for e in stage)
-    accept_len = out[0].cpu().numpy()
+    accept_len = (thin_out if thinning else out)[0].cpu().numpy()
 
     # ---- end to end through the host entry point: pinned host inputs in, host outputs back, every step ----
     arena = torch.empty(binding.pcg_verify_host_arena_bytes(B, K, V, M, dt_code), dtype=torch.uint8, device="cuda")
@@ -308,7 +323,7 @@ def main():
     sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
     default_is_cluster = B * info.slices <= 2 * sm_count  # the library's rule for PCG_VERIFY_DEFAULT
     launches_per_step = {"default": 2 if default_is_cluster else batched, "cluster": 2, "batched": batched,
-                         "dense": 2 + 1 + 1 + 1}[args.mode]
+                         "dense": 2 + 1 + 1 + 1, "thinning": 2}[args.mode]
 
     # the other modes, briefly (same inputs, same outputs): context for the headline mode
     other_modes = {}
@@ -327,9 +342,12 @@ def main():
                 binding.pcg_verify(tl, dl, x, handle, u, cfg.temperature, workspace=ws_m, out=out_m, mode=m)
             m1.record()
             torch.cuda.synchronize()
-            same = all(torch.equal(a_, b_) for a_, b_ in zip(out, out_m))
+            if thinning:  # other draws for the terminal token: only the accept lengths must agree
+                same = torch.equal(thin_out[0], out_m[0])
+            else:
+                same = all(torch.equal(a_, b_) for a_, b_ in zip(out, out_m))
             other_modes[name] = {"ms_per_step": m0.elapsed_time(m1) / reps, "steps": reps,
-                                 "outputs_equal_to_timed_mode": bool(same)}
+                                 ("accept_lengths_equal_to_timed_mode" if thinning else "outputs_equal_to_timed_mode"): bool(same)}
             del ws_m
 
     # the timed mode once more, captured in a CUDA graph and replayed (launch overhead off the host)
@@ -371,6 +389,31 @@ def main():
         extras["group_probs"] = {"rows": rows, "ms": gp_ms, "rows_per_s": rows / (gp_ms * 1e-3),
                                  "counted_gbs": rows * (V * esz + M * 4) / (gp_ms * 1e-3) / 1e9,
                                  "row_sum_max_error": float((P.sum(dim=1) - 1).abs().max())}
+        # the paper's thinning sampler for the terminal group instead of the enumerated residual
+        if not thinning:
+            for _ in range(3):
+                thin_step()
+            reps = 200
+            tev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            for e in tev:
+                e.record()
+            torch.cuda.synchronize()
+            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            q0.record()
+            for i in range(reps):
+                thin_step(tev if i == reps - 1 else None)
+            q1.record()
+            torch.cuda.synchronize()
+            th_ms = q0.elapsed_time(q1) / reps
+            tr = thin_out[4].float()
+            extras["verify_thinning"] = {
+                "ms_per_step": th_ms, "steps": reps, "value": B * K / (th_ms * 1e-3), "unit": UNIT,
+                "whole_step_gbs": B * (2 * K + 1) * V * esz / (th_ms * 1e-3) / 1e9,
+                "whole_step_frac_of_measured_peak": B * (2 * K + 1) * V * esz / (th_ms * 1e-3) / 1e9 / hbm_peak()[0],
+                "per_sequence_stage_ms_last_step": tev[1].elapsed_time(tev[2]),
+                "trials_supplied": args.thin_trials, "trials_mean": float(tr.mean()), "trials_max": int(tr.max()),
+                "sequences_exhausted": int((thin_out[3] & binding.FLAG_THINNING_EXHAUSTED).ne(0).sum()),
+                "accept_lengths_equal_to_timed_mode": bool(torch.equal(thin_out[0], out[0]))}
         d_emb = 512 if V >= 32768 else 128
         gen = torch.Generator(device="cuda")
         gen.manual_seed(2511)
@@ -403,9 +446,11 @@ def main():
                          "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": alg_bytes,
                          "avg_launch_ms": pos_ms},
-            "stages_ms": {"per_position_stage": pos_ms, "per_sequence_stage": term_ms},
+            "stages_ms": {"per_position_stage": pos_ms, "per_sequence_stage": term_ms,
+                          "sampled_on_every_nth_timed_step": STAGE_EVERY},
             "mode": args.mode + (" (per-sequence stage: " + ("cluster" if default_is_cluster else "batched") + ")"
-                                 if args.mode == "default" else ""),
+                                 if args.mode == "default" else
+                                 f" (pcg_verify_thinning, {args.thin_trials} trials supplied)" if thinning else ""),
             "other_modes": other_modes,
             "other_entry_points": extras,
             "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,

@@ -137,6 +137,17 @@ struct Elem<f16_t> {
 };
 
 // Streaming 128-bit load that does not allocate in L1 (each logit is read once per kernel).
+// Programmatic dependent launch.  A kernel launched with cudaLaunchAttributeProgrammaticStreamSerialization may
+// be scheduled while the kernel before it on the stream is still draining: pdl_enter() first lets the NEXT kernel
+// do the same with respect to this one, then waits until the previous grid has completed and its writes are
+// visible.  Nothing a previous kernel wrote may be read before it.  Without the launch attribute both are no-ops.
+__device__ __forceinline__ void pdl_enter() {
+#ifndef PCG_NO_PDL
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
+}
+
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
     uint4 r;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"

@@ -70,6 +70,7 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
     constexpr int NT = kThinThreads, NW = NT / 32, NV = Elem<T>::kPerVec, TS = 32 * NV;
     extern __shared__ __align__(16) unsigned char raw[];
     __shared__ int s_n, s_flags;
+    __shared__ float4 s_stats;
     const int V = G.V, M = G.M, K = a.K;
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int ntiles = (V + TS - 1) / TS;
@@ -79,9 +80,21 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
     int *ibox = reinterpret_cast<int *>(scratch + 64);          // 8 ints
     int *cand = ibox + 8;                                       // NW ints: group kept by each warp's trial, or -1
 
+    // the first trial of this warp: its uniforms are inputs of the call, so they can be fetched before the
+    // position kernel's results are waited for
+    const float *tu = a.thin + (size_t)b * a.n_trials * 3;
+    float u_first[3] = {0.f, 0.f, 0.f};
+    if (warp < a.n_trials) {
+#pragma unroll
+        for (int j = 0; j < 3; ++j) u_first[j] = tu[3 * warp + j];
+    }
+    pdl_enter();  // everything above may overlap the tail of the position kernel; none of its results is read before here
+
     // ---- 1. first rejected position and the flags of the positions up to it ----
     if (tid < 32) {
         int n = K, flags = 0;
+        // the statistics of the first 32 positions travel with their accept bits (one hop fewer for most sequences)
+        const float4 early = tid < K ? a.stats[b * K + tid] : make_float4(0.f, 0.f, 0.f, 0.f);
         for (int base = 0; base < K && n == K; base += 32) {
             const int i = base + tid;
             const int rej = (i < K) && (a.accept[b * K + i] == 0);
@@ -93,9 +106,16 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
             const int f = (i < K && i <= n) ? a.posflags[b * K + i] : 0;
             flags |= __reduce_or_sync(0xffffffffu, f);
         }
+        const int src = n < 32 ? n : 0;
+        float4 st;
+        st.x = __shfl_sync(0xffffffffu, early.x, src);
+        st.y = __shfl_sync(0xffffffffu, early.y, src);
+        st.z = __shfl_sync(0xffffffffu, early.z, src);
+        st.w = __shfl_sync(0xffffffffu, early.w, src);
         if (tid == 0) {
             s_n = n;
             s_flags = flags;
+            s_stats = (n < K && n >= 32) ? a.stats[b * K + n] : st;
         }
     }
     __syncthreads();
@@ -107,7 +127,7 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
     const bool vec_ok = ((uintptr_t)trow & 15u) == 0;
     float rs_p, iz_p, rs_q = 0.f, iz_q = 0.f;
     if (residual) {
-        const float4 st = a.stats[b * K + n];
+        const float4 st = s_stats;
         rs_p = st.x, iz_p = st.y, rs_q = st.z, iz_q = st.w;
     } else {
         // statistics of the bonus row: one pass with a per-thread reference, merged over the block
@@ -189,13 +209,13 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
     int gsel = -1, used = 0;
     const bool usable = Ztot > 0.0 && Ztot < (double)__builtin_huge_valf();
     if (!usable) flags |= PCG_FLAG_NONFINITE;
-    const float *tu = a.thin + (size_t)b * a.n_trials * 3;
     const int max_trials = usable ? (residual ? a.n_trials : 1) : 0;
     for (int r0 = 0; r0 < max_trials && gsel < 0; r0 += NW) {
         const int r = r0 + warp;
         int kept = -1;
         if (r < max_trials) {
-            const float u_tok = tu[3 * r], u_lab = tu[3 * r + 1], u_keep = tu[3 * r + 2];
+            const float u_tok = r0 ? tu[3 * r] : u_first[0], u_lab = r0 ? tu[3 * r + 1] : u_first[1];
+            const float u_keep = r0 ? tu[3 * r + 2] : u_first[2];
             // token y ~ target: tile by binary search over the prefix, then a scan inside the tile
             const double target = (double)u_tok * Ztot;
             int lo = 0, hi = ntiles - 1;  // the last tile's prefix is the total, which exceeds u * total for u < 1
