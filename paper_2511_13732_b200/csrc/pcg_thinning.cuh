@@ -37,7 +37,7 @@ struct ThinArgs {
 
 static size_t thin_smem_bytes(int V, size_t esz) {
     const size_t ts = 32 * (16 / esz);
-    return ((size_t)V + ts - 1) / ts * 8 + 32 * 8 + 64 * 4 + 8 * 4 + (kThinThreads / 32) * 4;
+    return ((size_t)V + ts - 1) / ts * 8 + 32 * 8 + 64 * 4 + 8 * 4 + 2 * (kThinThreads / 32) * 4;
 }
 
 // 2^(l s - rs) of this lane's share (one 16-byte vector) of tile `tile` of `row`; zero past the end of the row.
@@ -65,8 +65,47 @@ __device__ __forceinline__ float thin_lane_sum(const float (&e)[NV]) {
     return v;
 }
 
+// Token inside group g by ONE WARP: inverse CDF with u_token over p(t) w_{g,t} in the group's CSR order (the
+// target-conditional; the common factor 1/Z cancels).  Terms are taken relative to the row reference rs, which is
+// fine for a group that was just kept: its mass under that reference is positive.  Returns -1 if no term is positive.
 template <typename T>
-__global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, GroupsDev G) {
+__device__ __forceinline__ int warp_token_in_group(const GroupsDev &G, const T *trow, int g, float s, float rs,
+                                                   float u_token, int lane) {
+    const int lo = G.group_ptr[g], len = G.group_ptr[g + 1] - lo;
+    auto omega = [&](int k) -> float {
+        if (k >= len) return 0.f;
+        const int t = G.group_tok[lo + k];
+        const float w = G.pair_w ? G.pair_w[lo + k] : G.inv_deg[t];
+        return __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs)), w);
+    };
+    double total = 0.0;
+    for (int k = lane; k < len; k += 32) total += (double)omega(k);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    total = __shfl_sync(0xffffffffu, total, 0);  // one value for the whole warp
+    const double target = (double)u_token * total;
+    double carry = 0.0;
+    int pick = -1, last = -1;
+    for (int base = 0; base < len && pick < 0; base += 32) {
+        const float w = omega(base + lane);
+        double inc = (double)w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += up;
+        }
+        const unsigned hit = __ballot_sync(0xffffffffu, w > 0.f && carry + inc > target);
+        const unsigned pos = __ballot_sync(0xffffffffu, w > 0.f);
+        if (pos) last = base + 31 - __clz(pos);
+        if (hit) pick = base + __ffs(hit) - 1;
+        carry += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    const int ksel = pick >= 0 ? pick : last;  // rounding left no prefix above the target: last token with mass
+    return ksel >= 0 ? G.group_tok[lo + ksel] : -1;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, GroupsDev G) {
     constexpr int NT = kThinThreads, NW = NT / 32, NV = Elem<T>::kPerVec, TS = 32 * NV;
     extern __shared__ __align__(16) unsigned char raw[];
     __shared__ int s_n, s_flags;
@@ -79,6 +118,7 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
     float *scratch = reinterpret_cast<float *>(dscratch + 32);  // 64 floats
     int *ibox = reinterpret_cast<int *>(scratch + 64);          // 8 ints
     int *cand = ibox + 8;                                       // NW ints: group kept by each warp's trial, or -1
+    int *cand_tok = cand + NW;                                  // NW ints: the token drawn inside that group
 
     // the first trial of this warp: its uniforms are inputs of the call, so they can be fetched before the
     // position kernel's results are waited for
@@ -88,6 +128,8 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
 #pragma unroll
         for (int j = 0; j < 3; ++j) u_first[j] = tu[3 * warp + j];
     }
+    const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
+    const int pre_tok = tid < K ? a.draft_tokens[b * K + tid] : -1;  // for the emission at the end
     pdl_enter();  // everything above may overlap the tail of the position kernel; none of its results is read before here
 
     // ---- 1. first rejected position and the flags of the positions up to it ----
@@ -159,21 +201,28 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
         iz_p = 1.0f / Z;
     }
 
-    // ---- 2. tile sums of the target row (four tiles of loads in flight per warp), then their prefix ----
-    for (int base = warp; base < ntiles; base += 4 * NW) {
-        uint4 r[4];
-        bool fast[4];
+    // ---- 2. tile sums of the target row, then their prefix.  A warp walks a contiguous run of tiles, kInFlight
+    // tiles of loads in flight at a time (deeper or double-buffered variants measured the same) ----
+#ifndef PCG_THIN_INFLIGHT
+#define PCG_THIN_INFLIGHT 4
+#endif
+    constexpr int kInFlight = PCG_THIN_INFLIGHT;
+    const int tiles_per_warp = (ntiles + NW - 1) / NW;
+    const int tile_first = warp * tiles_per_warp, tile_end = min(ntiles, tile_first + tiles_per_warp);
+    auto issue = [&](int base, uint4(&r)[kInFlight], bool(&fast)[kInFlight]) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int tile = base + j * NW;
+        for (int j = 0; j < kInFlight; ++j) {
+            const int tile = base + j;
             const int t0 = (tile * 32 + lane) * NV;
-            fast[j] = tile < ntiles && vec_ok && t0 + NV <= V;
+            fast[j] = tile < tile_end && vec_ok && t0 + NV <= V;
             if (fast[j]) r[j] = ld_stream(reinterpret_cast<const uint4 *>(trow + t0));
         }
+    };
+    auto consume = [&](int base, const uint4(&r)[kInFlight], const bool(&fast)[kInFlight]) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int tile = base + j * NW;
-            if (tile >= ntiles) continue;  // (warp-uniform)
+        for (int j = 0; j < kInFlight; ++j) {
+            const int tile = base + j;
+            if (tile >= tile_end) continue;  // (warp-uniform)
             float e[NV];
             if (fast[j]) {
                 float v[NV];
@@ -188,6 +237,12 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
             for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
             if (lane == 0) tile_incl[tile] = (double)sum;
         }
+    };
+    for (int base = tile_first; base < tile_end; base += kInFlight) {
+        uint4 r[kInFlight];
+        bool fast[kInFlight];
+        issue(base, r, fast);
+        consume(base, r, fast);
     }
     __syncthreads();
     double Ztot;
@@ -206,7 +261,7 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
     __syncthreads();
 
     // ---- 3. trials: warp w of round r0 runs trial r0 + w; the first kept candidate in trial order wins ----
-    int gsel = -1, used = 0;
+    int gsel = -1, used = 0, z = -1;
     const bool usable = Ztot > 0.0 && Ztot < (double)__builtin_huge_valf();
     if (!usable) flags |= PCG_FLAG_NONFINITE;
     const int max_trials = usable ? (residual ? a.n_trials : 1) : 0;
@@ -282,6 +337,10 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
                 keep = __fmul_rn(u_keep, P) < P - Q;
             }
             kept = keep ? g : -1;
+            if (keep) {  // the token inside the kept group, by this warp (used only if this trial wins)
+                const int zt = warp_token_in_group<T>(G, trow, g, a.s, rs_p, u_token, lane);
+                if (lane == 0) cand_tok[warp] = zt;
+            }
         }
         if (lane == 0) cand[warp] = kept;
         __syncthreads();
@@ -289,6 +348,7 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
         for (int w = 0; w < NW; ++w)
             if (cand[w] >= 0) {
                 gsel = cand[w];
+                z = cand_tok[w];
                 used = r0 + w + 1;
                 break;
             }
@@ -355,16 +415,30 @@ __global__ void __launch_bounds__(kThinThreads) thinning_kernel(ThinArgs a, Grou
         __syncthreads();
     }
 
-    // ---- 4. token inside the kept group, outputs ----
-    int z = 0;
+    // ---- 4. outputs (the token was drawn by the winning warp; block-wide after the enumerated fallback) ----
     if (gsel < 0) {  // no mass anywhere (non-finite inputs): emit group 0 / token 0 and flag it
         gsel = 0;
+        z = 0;
         flags |= PCG_FLAG_NONFINITE;
-    } else {
-        const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
+    } else if (z < 0) {
         z = draw_token_in_group<T, NT>(G, trow, gsel, a.s, u_token, dscratch, scratch, ibox, flags);
     }
-    emit_sequence<NT>(G, b, K, n, z, gsel, flags, a.draft_tokens, a.labels, a.out_accept_len, a.out_tokens, a.out_groups,
-                      a.out_flags);
-    if (tid == 0 && a.out_trials) a.out_trials[b] = used;
+    for (int i = tid; i <= K; i += NT) {
+        int tok = -1, grp = -1;
+        if (i < n) {
+            tok = i == tid ? pre_tok : a.draft_tokens[b * K + i];
+            if (tok < 0 || tok >= V) tok = 0;  // verified as token 0 (and flagged), so emitted as token 0
+            grp = a.labels[b * K + i];
+        } else if (i == n) {
+            tok = z;
+            grp = gsel;
+        }
+        a.out_tokens[(int64_t)b * (K + 1) + i] = tok;
+        if (a.out_groups) a.out_groups[(int64_t)b * (K + 1) + i] = grp;
+    }
+    if (tid == 0) {
+        a.out_accept_len[b] = n;
+        if (a.out_flags) a.out_flags[b] = flags;
+        if (a.out_trials) a.out_trials[b] = used;
+    }
 }
