@@ -26,7 +26,7 @@ EXPORTS = [
     "pcg_status_string", "pcg_last_error", "pcg_groups_create", "pcg_groups_destroy", "pcg_groups_info",
     "pcg_groups_set_accept_bias",
     "pcg_group_probs", "pcg_verify_workspace_bytes", "pcg_verify", "pcg_verify_host_arena_bytes", "pcg_verify_host",
-    "pcg_verify_static", "pcg_asg_create", "pcg_asg_info", "pcg_asg_csr", "pcg_asg_destroy",
+    "pcg_verify_static", "pcg_verify_thinning_workspace_bytes", "pcg_verify_thinning", "pcg_asg_create", "pcg_asg_info", "pcg_asg_csr", "pcg_asg_destroy",
 ]
 
 

@@ -92,6 +92,10 @@ def test_workspace_queries():
     assert a >= 256 * 16 * 28 and b >= 256 and a % 256 == 0 and b % 256 == 0
     arena = lib.pcg_verify_host_arena_bytes(256, 16, 65536, 16384, 1, 0)
     assert arena >= 256 * 33 * 65536 * 2 + a
+    t = lib.pcg_verify_thinning_workspace_bytes(256, 16, 65536, 16384, 1)
+    assert t >= 256 * 16 * 28 + 256 * 16384 * 4 and t % 256 == 0
+    assert lib.pcg_verify_thinning(None, None, 0, 1, 1, None, None, None, None, 4, 1.0, None, None, None, None, None,
+                                   None, 0, None, None) == 1  # null handle
 
 
 def test_binding_has_no_fallback(monkeypatch):
