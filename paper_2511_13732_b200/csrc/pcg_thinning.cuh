@@ -365,14 +365,34 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
         double Zr = 0.0, excl = 0.0, incl = 0.0, my = 0.0;
         bool minus_q = true;
         for (int attempt = 0; attempt < 2; ++attempt) {
+            // one thread per group, its tokens eight at a time: ids first, then the gathers they address, then the
+            // sum in CSR order (the dependent loads of a batch are in flight together)
+            constexpr int FB = 8;
             for (int g = tid; g < M; g += NT) {
                 float acc = 0.f;
-                for (int k = G.group_ptr[g]; k < G.group_ptr[g + 1]; ++k) {
-                    const int t = G.group_tok[k];
-                    const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
-                    float d = __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs_p)), iz_p);
-                    if (minus_q) d -= __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), a.s, -rs_q)), iz_q);
-                    acc += __fmul_rn(d, w);
+                const int k_end = G.group_ptr[g + 1];
+                for (int k = G.group_ptr[g]; k < k_end; k += FB) {
+                    int t[FB];
+                    float lp[FB], lq[FB], w[FB];
+#pragma unroll
+                    for (int j = 0; j < FB; ++j) t[j] = k + j < k_end ? G.group_tok[k + j] : -1;
+#pragma unroll
+                    for (int j = 0; j < FB; ++j) {
+                        lp[j] = lq[j] = kNegInf;
+                        w[j] = 0.f;
+                        if (t[j] >= 0) {
+                            lp[j] = Elem<T>::widen(trow[t[j]]);
+                            if (minus_q) lq[j] = Elem<T>::widen(qrow[t[j]]);
+                            w[j] = G.pair_w ? G.pair_w[k + j] : G.inv_deg[t[j]];
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < FB; ++j) {
+                        if (t[j] < 0) continue;
+                        float d = __fmul_rn(ex2(__fmaf_rn(lp[j], a.s, -rs_p)), iz_p);
+                        if (minus_q) d -= __fmul_rn(ex2(__fmaf_rn(lq[j], a.s, -rs_q)), iz_q);
+                        acc += __fmul_rn(d, w[j]);
+                    }
                 }
                 own[g] = fmaxf(acc, 0.f);
             }
