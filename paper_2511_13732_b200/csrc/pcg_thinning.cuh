@@ -299,17 +299,16 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
             int pick = 0;
             if (lane == L) {
                 double loc = inc - (double)lsum;
-                int last = 0;
-                bool found = false;
+                int first_above = -1, last = 0;
 #pragma unroll
                 for (int i = 0; i < NV; ++i) {
                     loc += (double)e[i];
                     if (e[i] > 0.f) {
-                        if (!found) last = i;
-                        if (!found && loc > tl) found = true;
+                        last = i;
+                        if (first_above < 0 && loc > tl) first_above = i;
                     }
                 }
-                pick = last;
+                pick = first_above >= 0 ? first_above : last;
             }
             pick = __shfl_sync(0xffffffffu, pick, L);
             int y = (tile * 32 + L) * NV + pick;
