@@ -317,7 +317,7 @@ def main():
 
     # kernels launched by one pcg_verify call (see pcg_verify in csrc/pcg_kernels.cu)
     info = handle.info
-    chunk_unit = 128 if B >= 128 else 32
+    chunk_unit = 256 if (B >= 256 and (64 << 20) // (V * 4) >= 256) else 128 if B >= 128 else 32
     chunk = min(-(-B // chunk_unit) * chunk_unit, max(chunk_unit, ((64 << 20) // (V * 4)) // chunk_unit * chunk_unit))
     batched = 1 + 1 + 2 * (-(-B // chunk)) + 1  # position, prepare, (transpose, sparse product) per chunk, draw
     sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count

@@ -729,7 +729,7 @@ constexpr int kSpmmThreads = PCG_SPMM_THREADS;  // group_spmm_kernel: warps of 8
 #define PCG_SPMM_DEPTH 8  // tokens per batch of the sparse product; two batches of loads are in flight per lane
 #endif
 #ifndef PCG_SPMM_GW
-#define PCG_SPMM_GW 8  // consecutive groups per warp of the sparse product
+#define PCG_SPMM_GW 4  // consecutive groups per warp of the sparse product
 #endif
 constexpr int kSpmmGroupsPerWarp = PCG_SPMM_GW;
 constexpr int kSpmmWide = PCG_SPMM_SPL;
@@ -1033,14 +1033,24 @@ struct SeqVec<4> {
     }
 };
 
-// Grid (ceil(M / (8 * warps per block)), bpad / (32 * SPL)).  A warp owns 8 consecutive groups -- their token
+template <>
+struct SeqVec<8> {  // one 256-bit load per lane
+    float v[8];
+    __device__ __forceinline__ void load(const float *p) {
+        asm volatile("ld.global.cg.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                     : "l"(p));
+    }
+};
+
+// Grid (ceil(M / (GW * warps per block)), bpad / (32 * SPL)).  A warp owns GW (4) consecutive groups -- their token
 // lists are one contiguous range of the CSR -- and a block of 32 * SPL sequences; a lane holds SPL consecutive
-// sequences (one 4-, 8- or 16-byte load per token).  The range is walked in batches of DEPTH tokens with two
+// sequences (one 4-, 16- or 32-byte load per token).  The range is walked in batches of DEPTH tokens with two
 // register buffers: the loads of batch i+1 are issued before batch i is added, so a warp keeps up to 2 * DEPTH
 // lines of Dt in flight at all times (random L2 gathers need on the order of 150 KB in flight per SM to
 // reach the L2's bandwidth).  Token ids are fetched 32 at a time, one block of 32 ahead.  Sums run in CSR
-// order; a group ends where the running entry index reaches the next group pointer.  The warp's 8 x (32 * SPL)
-// sums are turned in shared memory so that R is written along the group index, 32 bytes per sequence.
+// order; a group ends where the running entry index reaches the next group pointer.  The warp's GW x (32 * SPL)
+// sums are turned in shared memory so that R is written along the group index, 4 * GW bytes per sequence.
 template <int SPL, int DEPTH, bool HAS_W>
 __global__ void __launch_bounds__(kSpmmThreads) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
     pdl_enter();
@@ -1134,7 +1144,7 @@ __global__ void __launch_bounds__(kSpmmThreads) group_spmm_kernel(SpmmArgs a, Gr
     close_groups(e1);  // trailing empty groups (gi reaches ng)
     __syncwarp();
     const int bbase = a.b0 + blockIdx.y * NS;
-    for (int i = lane; i < NS * GW; i += 32) {  // 8 consecutive lanes: the 8 groups of one sequence
+    for (int i = lane; i < NS * GW; i += 32) {  // GW consecutive lanes: the GW groups of one sequence
         const int sq = i / GW, t = i - sq * GW;
         if (bbase + sq < a.B && t < ng) a.R[(size_t)(bbase + sq) * G.M + g0 + t] = tile[t * TS + sq];
     }
@@ -1459,10 +1469,17 @@ static cudaError_t launch_cluster(Kern kern, int blocks, int cluster, size_t sme
 #endif
 constexpr size_t kDtBudgetBytes = (size_t)PCG_DT_BUDGET_MB << 20;  // Dt of one chunk of sequences must stay inside the L2
 
-// Sequences per chunk of the batched terminal stage: a multiple of 32 * kSpmmWide (one warp of the sparse
-// product covers that many sequences with vector loads) once the batch has that many, of 32 below that.
+// Sequences per lane of the sparse product: 8 (one 256-bit load per token and lane) from 256 sequences on if
+// that many fit the budget of the transposed operand, kSpmmWide (4) from 128 on, else 1.
+static int spmm_lanes(int B, int V) {
+    if (B >= 256 && kDtBudgetBytes / ((size_t)V * 4) >= 256) return 8;
+    return B >= 32 * kSpmmWide ? kSpmmWide : 1;
+}
+
+// Sequences per chunk of the batched terminal stage: a multiple of what one warp of the sparse product covers
+// (32 sequences per lane-sequence).
 static int terminal_chunk(int B, int V) {
-    const int64_t unit = B >= 32 * kSpmmWide ? 32 * kSpmmWide : 32;
+    const int64_t unit = 32 * spmm_lanes(B, V);
     const int64_t bpad = ((int64_t)B + unit - 1) / unit * unit;
     int64_t fit = (int64_t)(kDtBudgetBytes / ((size_t)V * 4)) / unit * unit;
     if (fit < unit) fit = unit;
@@ -1509,12 +1526,18 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
     return w;
 }
 
-// The sparse product over nb blocks of 32 sequences (nb a multiple of kSpmmWide when `wide`).
-static void launch_spmm(const SpmmArgs &sp, int nb, bool wide, const GroupsDev &G, cudaStream_t cs) {
+// The sparse product over nb blocks of 32 sequences (nb a multiple of `lanes`, the sequences per lane: 8, 4 or 1).
+static void launch_spmm(const SpmmArgs &sp, int nb, int lanes, const GroupsDev &G, cudaStream_t cs) {
     const int gpb = kSpmmGroupsPerWarp * (kSpmmThreads / 32);  // groups per block
     const unsigned gx = (unsigned)((G.M + gpb - 1) / gpb);
     const bool has_w = G.pair_w != nullptr;
-    if (wide) {
+    if (lanes == 8) {
+        const dim3 grid(gx, (unsigned)(nb / 8));
+        if (has_w)
+            launch_after(group_spmm_kernel<8, 4, true>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+        else
+            launch_after(group_spmm_kernel<8, 4, false>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+    } else if (lanes == kSpmmWide) {
         const dim3 grid(gx, (unsigned)(nb / kSpmmWide));
         if (has_w)
             launch_after(group_spmm_kernel<kSpmmWide, kSpmmDepth, true>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
@@ -1567,7 +1590,7 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
             TransposeArgs tr{base, base, nr, 0, 0, chunk, s, groups->probs_zero, groups->probs_stats, groups->probs_dt};
             const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
             PCG_DISPATCH_DTYPE(dtype, launch_after(residual_transpose_kernel<LogitT>, tgrid, dim3(kTrThreads), 0, cs, tr, G));
-            launch_spmm(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M}, nb, true, G, cs);
+            launch_spmm(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M}, nb, kSpmmWide, G, cs);
         }
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching the batched group-probability kernels");
@@ -1686,17 +1709,17 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         if (!dense) {
             const int chunk = terminal_chunk(B, G.V);
             const int tt = 32 * (int)(16 / dtype_bytes(dtype));
-            const bool wide = B >= 32 * kSpmmWide;  // several sequences per lane in the sparse product
+            const int lanes = spmm_lanes(B, G.V);  // sequences per lane in the sparse product
             for (int b0 = 0; b0 < B; b0 += chunk) {
-                // blocks of 32 sequences in this chunk, rounded up to what one block of the sparse product reads
-                const int unit = wide ? 32 * kSpmmWide : 32;
+                // blocks of 32 sequences in this chunk, rounded up to what one warp of the sparse product reads
+                const int unit = 32 * lanes;
                 const int nb = (std::min(B - b0, chunk) + unit - 1) / unit * (unit / 32);
                 TransposeArgs tr{target_logits, draft_logits, B, K, b0, chunk, s, w.term_n, w.term_stats, w.Dt};
                 const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
                 PCG_DISPATCH_DTYPE(dtype, launch_after(residual_transpose_kernel<LogitT>, tgrid, dim3(kTrThreads), 0, cs, tr, G));
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
-                launch_spmm(SpmmArgs{w.Dt, B, b0, chunk, w.R}, nb, wide, G, cs);
+                launch_spmm(SpmmArgs{w.Dt, B, b0, chunk, w.R}, nb, lanes, G, cs);
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
             }
