@@ -1585,12 +1585,13 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
             const char *base = (const char *)logits + (size_t)r0 * G.V * dtype_bytes(dtype);
             PCG_DISPATCH_DTYPE(dtype, launch_after(row_stats_kernel<LogitT>, dim3((unsigned)nr), dim3(kPrepThreads), 0, cs,
                                                    (const void *)base, s, groups->probs_stats, G));
-            const int nb = (nr + 127) / 128 * 4;  // blocks of 32 rows, whole warps of the sparse product
+            const int lanes = (chunk % 256 == 0 && nr >= 256) ? 8 : kSpmmWide;      // rows per lane of the sparse product
+            const int nb = (nr + 32 * lanes - 1) / (32 * lanes) * lanes;          // blocks of 32 rows, whole warps of it
             // every row is "a sequence whose only row is accepted": K = 0 makes the kernel form p alone
             TransposeArgs tr{base, base, nr, 0, 0, chunk, s, groups->probs_zero, groups->probs_stats, groups->probs_dt};
             const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
             PCG_DISPATCH_DTYPE(dtype, launch_after(residual_transpose_kernel<LogitT>, tgrid, dim3(kTrThreads), 0, cs, tr, G));
-            launch_spmm(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M}, nb, kSpmmWide, G, cs);
+            launch_spmm(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M}, nb, lanes, G, cs);
         }
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching the batched group-probability kernels");
