@@ -1175,61 +1175,64 @@ struct DrawArgs {
 
 __device__ __forceinline__ int own_slot(int j) { return j + (j >> 5); }  // one pad word per 32: chunked reads spread over banks
 
-// Token inside the drawn group `gsel`: target-conditional p(t) w / P[g] over the group's CSR order, by inverse
-// CDF with `u_token` (whole block; dscratch: 32 doubles, scratch: 64 floats, ibox: 8 ints of shared memory).
-// Only ratios inside the group matter, so the terms are taken relative to the group's largest logit.
-template <typename T, int NT>
-__device__ __forceinline__ int draw_token_in_group(const GroupsDev &G, const T *trow, int gsel, float s, float u_token,
-                                                   double *dscratch, float *scratch, int *ibox, int &flags) {
-    const int tid = threadIdx.x;
-    const int lo = G.group_ptr[gsel], hi = G.group_ptr[gsel + 1], len = hi - lo;
-    const int per2 = (len + NT - 1) / NT;
-    const int k0 = min(len, tid * per2), k1 = min(len, k0 + per2);
+// Token inside group g by ONE WARP: inverse CDF with u_token over p(t) w_{g,t} in the group's CSR order (the
+// target-conditional; the common factor 1/Z cancels, and only ratios inside the group matter, so the terms are
+// taken relative to the group's largest logit).  Sums in double by chunked warp scans.  Returns -1 if no term is
+// positive (non-finite inputs).
+template <typename T>
+__device__ __forceinline__ int warp_token_in_group(const GroupsDev &G, const T *trow, int g, float s, float u_token,
+                                                   int lane) {
+    const int lo = G.group_ptr[g], len = G.group_ptr[g + 1] - lo;
     float mloc = kNegInf;
-    for (int k = k0; k < k1; ++k) mloc = fmaxf(mloc, Elem<T>::widen(trow[G.group_tok[lo + k]]));
-    const float mg = block_max<NT>(mloc, scratch);
-    const float rs = mg > kNegInf ? mg * s : 0.f;
+    for (int k = lane; k < len; k += 32) mloc = fmaxf(mloc, Elem<T>::widen(trow[G.group_tok[lo + k]]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o));
+    const float rs = mloc > kNegInf ? mloc * s : 0.f;
     auto omega = [&](int k) -> float {
+        if (k >= len) return 0.f;
         const int t = G.group_tok[lo + k];
         const float w = G.pair_w ? G.pair_w[lo + k] : G.inv_deg[t];
         return __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs)), w);
     };
-    double wsum = 0.0;
-    int wlast = -1;
-    for (int k = k0; k < k1; ++k) {
-        const float w = omega(k);
-        wsum += (double)w;
-        if (w > 0.f) wlast = k;
-    }
-    double excl, incl, wtot;
-    block_scan<NT>(wsum, dscratch, &excl, &incl, &wtot);
-    if (tid == 0) {
-        ibox[2] = NT;
-        ibox[3] = -1;
-        ibox[4] = -1;
-    }
-    __syncthreads();
-    const double target2 = (double)u_token * wtot;
-    if (wlast >= 0) atomicMax(&ibox[3], wlast);
-    if (wsum > 0.0 && incl > target2) atomicMin(&ibox[2], tid);
-    __syncthreads();
-    if (ibox[2] == tid) {
-        double loc = 0.0;
-        int pick = wlast;
-        for (int k = k0; k < k1; ++k) {
-            loc += (double)omega(k);
-            if (excl + loc > target2) {
-                pick = k;
-                break;
-            }
+    double total = 0.0;
+    for (int k = lane; k < len; k += 32) total += (double)omega(k);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    total = __shfl_sync(0xffffffffu, total, 0);  // one value for the whole warp
+    const double target = (double)u_token * total;
+    double carry = 0.0;
+    int pick = -1, last = -1;
+    for (int base = 0; base < len && pick < 0; base += 32) {
+        const float w = omega(base + lane);
+        double inc = (double)w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += up;
         }
-        ibox[4] = pick;
+        const unsigned hit = __ballot_sync(0xffffffffu, w > 0.f && carry + inc > target);
+        const unsigned pos = __ballot_sync(0xffffffffu, w > 0.f);
+        if (pos) last = base + 31 - __clz(pos);
+        if (hit) pick = base + __ffs(hit) - 1;
+        carry += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    const int ksel = pick >= 0 ? pick : last;  // rounding left no prefix above the target: last token with mass
+    return ksel >= 0 ? G.group_tok[lo + ksel] : -1;
+}
+
+// The same from inside a block-wide code path: warp 0 draws, everybody gets the token (ibox: shared ints).
+template <typename T>
+__device__ __forceinline__ int block_token_in_group(const GroupsDev &G, const T *trow, int g, float s, float u_token,
+                                                    int *ibox, int &flags) {
+    if (threadIdx.x < 32) {
+        const int zt = warp_token_in_group<T>(G, trow, g, s, u_token, (int)threadIdx.x);
+        if (threadIdx.x == 0) ibox[5] = zt;
     }
     __syncthreads();
-    const int ksel = ibox[4] >= 0 ? ibox[4] : ibox[3];
-    if (ksel >= 0) return G.group_tok[lo + ksel];
+    const int z = ibox[5];
+    if (z >= 0) return z;
     flags |= PCG_FLAG_NONFINITE;  // the drawn group has no token with target mass (non-finite inputs)
-    return len > 0 ? G.group_tok[lo] : 0;
+    return G.group_ptr[g + 1] > G.group_ptr[g] ? G.group_tok[G.group_ptr[g]] : 0;
 }
 
 // Outputs of sequence b: accepted draft tokens, the drawn token z of group gsel at position n, then filler.
@@ -1300,7 +1303,16 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
         } else if (attempt == 0) {
             // R holds sum_t (p - q)/N for a rejection and sum_t p/N for the bonus row
             const float *Rb = a.R + (size_t)b * M;  // (with global staging this is `own` itself: clamped in place)
-            for (int g = tid; g < M; g += NT) own[slot(g)] = fmaxf(Rb[g], 0.f);
+            // eight loads in flight per thread before the first is used (one at a time, this loop was 10 of the
+            // kernel's 23 microseconds)
+            for (int g0 = tid; g0 < M; g0 += 8 * NT) {
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = g0 + j * NT < M ? Rb[g0 + j * NT] : 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (g0 + j * NT < M) own[slot(g0 + j * NT)] = fmaxf(v[j], 0.f);
+            }
         } else {
             // slow path of the zero-residual fallback: the target masses straight from the row
             const float rs = a.term_stats[b].x;
@@ -1359,7 +1371,7 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
         gsel = 0;
         flags |= PCG_FLAG_NONFINITE;
     } else {
-        z = draw_token_in_group<T, NT>(G, trow, gsel, a.s, u_token, dscratch, scratch, ibox, flags);
+        z = block_token_in_group<T>(G, trow, gsel, a.s, u_token, ibox, flags);
     }
     emit_sequence<NT>(G, b, K, n, z, gsel, flags, a.draft_tokens, a.labels, a.out_accept_len, a.out_tokens, a.out_groups,
                       a.out_flags);

@@ -65,45 +65,6 @@ __device__ __forceinline__ float thin_lane_sum(const float (&e)[NV]) {
     return v;
 }
 
-// Token inside group g by ONE WARP: inverse CDF with u_token over p(t) w_{g,t} in the group's CSR order (the
-// target-conditional; the common factor 1/Z cancels).  Terms are taken relative to the row reference rs, which is
-// fine for a group that was just kept: its mass under that reference is positive.  Returns -1 if no term is positive.
-template <typename T>
-__device__ __forceinline__ int warp_token_in_group(const GroupsDev &G, const T *trow, int g, float s, float rs,
-                                                   float u_token, int lane) {
-    const int lo = G.group_ptr[g], len = G.group_ptr[g + 1] - lo;
-    auto omega = [&](int k) -> float {
-        if (k >= len) return 0.f;
-        const int t = G.group_tok[lo + k];
-        const float w = G.pair_w ? G.pair_w[lo + k] : G.inv_deg[t];
-        return __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs)), w);
-    };
-    double total = 0.0;
-    for (int k = lane; k < len; k += 32) total += (double)omega(k);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-    total = __shfl_sync(0xffffffffu, total, 0);  // one value for the whole warp
-    const double target = (double)u_token * total;
-    double carry = 0.0;
-    int pick = -1, last = -1;
-    for (int base = 0; base < len && pick < 0; base += 32) {
-        const float w = omega(base + lane);
-        double inc = (double)w;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const double up = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += up;
-        }
-        const unsigned hit = __ballot_sync(0xffffffffu, w > 0.f && carry + inc > target);
-        const unsigned pos = __ballot_sync(0xffffffffu, w > 0.f);
-        if (pos) last = base + 31 - __clz(pos);
-        if (hit) pick = base + __ffs(hit) - 1;
-        carry += __shfl_sync(0xffffffffu, inc, 31);
-    }
-    const int ksel = pick >= 0 ? pick : last;  // rounding left no prefix above the target: last token with mass
-    return ksel >= 0 ? G.group_tok[lo + ksel] : -1;
-}
-
 template <typename T>
 __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, GroupsDev G) {
     constexpr int NT = kThinThreads, NW = NT / 32, NV = Elem<T>::kPerVec, TS = 32 * NV;
@@ -337,7 +298,7 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
             }
             kept = keep ? g : -1;
             if (keep) {  // the token inside the kept group, by this warp (used only if this trial wins)
-                const int zt = warp_token_in_group<T>(G, trow, g, a.s, rs_p, u_token, lane);
+                const int zt = warp_token_in_group<T>(G, trow, g, a.s, u_token, lane);
                 if (lane == 0) cand_tok[warp] = zt;
             }
         }
@@ -440,7 +401,7 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
         z = 0;
         flags |= PCG_FLAG_NONFINITE;
     } else if (z < 0) {
-        z = draw_token_in_group<T, NT>(G, trow, gsel, a.s, u_token, dscratch, scratch, ibox, flags);
+        z = block_token_in_group<T>(G, trow, gsel, a.s, u_token, ibox, flags);
     }
     for (int i = tid; i <= K; i += NT) {
         int tok = -1, grp = -1;
