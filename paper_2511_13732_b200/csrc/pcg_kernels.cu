@@ -1296,6 +1296,12 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
     const int per = (M + NT - 1) / NT;
     const int i0 = min(M, tid * per), i1 = min(M, i0 + per);
     double Ztot = 0.0, my_excl = 0.0, my_incl = 0.0, my_sum = 0.0;
+    int my_last = -1;  // last group with mass in this thread's chunk
+    if (tid == 0) {
+        ibox[2] = NT;  // selected thread (minimum)
+        ibox[3] = -1;  // last group with mass (maximum)
+        ibox[4] = -1;  // drawn group
+    }
     for (int attempt = 0; attempt < 2; ++attempt) {
         if (DENSE) {
             for (int g = tid; g < M; g += NT)
@@ -1303,14 +1309,14 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
         } else if (attempt == 0) {
             // R holds sum_t (p - q)/N for a rejection and sum_t p/N for the bonus row
             const float *Rb = a.R + (size_t)b * M;  // (with global staging this is `own` itself: clamped in place)
-            // eight loads in flight per thread before the first is used (one at a time, this loop was 10 of the
-            // kernel's 23 microseconds)
-            for (int g0 = tid; g0 < M; g0 += 8 * NT) {
-                float v[8];
+            // sixteen loads in flight per thread before the first is used (one at a time, this loop was 10 of
+            // the kernel's 23 microseconds)
+            for (int g0 = tid; g0 < M; g0 += 16 * NT) {
+                float v[16];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = g0 + j * NT < M ? Rb[g0 + j * NT] : 0.f;
+                for (int j = 0; j < 16; ++j) v[j] = g0 + j * NT < M ? Rb[g0 + j * NT] : 0.f;
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
+                for (int j = 0; j < 16; ++j)
                     if (g0 + j * NT < M) own[slot(g0 + j * NT)] = fmaxf(v[j], 0.f);
             }
         } else {
@@ -1329,7 +1335,12 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
         __syncthreads();
         // ---- prefix sums over the groups (double): a contiguous chunk per thread, then a block scan ----
         my_sum = 0.0;
-        for (int j = i0; j < i1; ++j) my_sum += (double)own[slot(j)];
+        my_last = -1;
+        for (int j = i0; j < i1; ++j) {
+            const float v = own[slot(j)];
+            my_sum += (double)v;
+            if (v > 0.f) my_last = j;
+        }
         block_scan<NT>(my_sum, dscratch, &my_excl, &my_incl, &Ztot);
         if (Ztot > 0.0 || !residual) break;
         // a rejection whose residual vanished (P == Q to rounding): draw from P instead
@@ -1339,16 +1350,7 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
     }
 
     // ---- group draw: first group whose inclusive prefix exceeds u * Z ----
-    const double target = (double)u_group * Ztot;
-    if (tid == 0) {
-        ibox[2] = NT;  // selected thread (minimum)
-        ibox[3] = -1;  // last group with mass (maximum)
-        ibox[4] = -1;  // drawn group
-    }
-    __syncthreads();
-    int my_last = -1;
-    for (int j = i0; j < i1; ++j)
-        if (own[slot(j)] > 0.f) my_last = j;
+    const double target = (double)u_group * Ztot;  // (ibox was initialised before the barriers of the scan)
     if (my_last >= 0) atomicMax(&ibox[3], my_last);
     if (my_sum > 0.0 && my_incl > target) atomicMin(&ibox[2], tid);
     __syncthreads();
