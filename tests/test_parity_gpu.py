@@ -184,6 +184,35 @@ def test_verify_batch_spanning_several_sequence_blocks(oracle):
         _assert_parity(run_verify(bt, h, mode=mode), ref)
 
 
+@pytest.mark.parametrize("B", [130, 300])
+def test_verify_wide_sparse_product_forms(oracle, B):
+    """From 128 sequences on a lane of the sparse product holds 4 sequences (128-bit loads), from 256 on 8 (256-bit
+    loads): ragged batches in both forms, with a group count that is not a multiple of a block's groups, with and
+    without general weights, bonus rows included; pcg_group_probs over 300 rows takes the 256-bit form too."""
+    from paper_2511_13732_b200 import binding
+
+    cfg = W.scaled(W.CONFIGS["C3"], B=B, V=2500, M=611, K=2)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    bt.draft_logits[::5] = bt.target_logits[::5, :cfg.K]
+    ref = run_oracle(oracle, bt, groups)
+    assert np.any(ref.accept_len == cfg.K) and np.any(ref.accept_len == 0)
+    _assert_parity(run_verify(bt, make_handle(groups), mode=4), ref)
+    rng = np.random.default_rng(9)
+    raw = rng.random(groups.nnz) + 0.05
+    tot = np.zeros(cfg.V)
+    np.add.at(tot, groups.group_tok, raw)
+    w = (raw / tot[groups.group_tok]).astype(np.float32)
+    ref_w = run_oracle(oracle, bt, groups, weights=w.astype(np.float64))
+    hw = make_handle(groups, weights=w)
+    _assert_parity(run_verify(bt, hw, mode=4), ref_w, max_excused=1)
+    x = np.ascontiguousarray(bt.target_logits.reshape(-1, cfg.V)[:B])
+    want = oracle.group_probs(x, groups.group_ptr, groups.group_tok, groups.tok_degree, cfg.temperature,
+                              weights=w.astype(np.float64))
+    got = binding.pcg_group_probs(logits_to_device(x), hw, cfg.temperature).cpu().numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-5, atol=1e-37)
+
+
 @pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("hint", [1, 2, 4, 8])
 def test_verify_any_slicing(oracle, hint, mode):
