@@ -289,7 +289,7 @@ pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits
                              int32_t *out_flags, pcg_stream stream);
 
 /*
- * pcg_verify with the paper's own sampler for the terminal group: "Residual sampling via thinning" (Sec. 2.2).
+ * pcg_verify with the paper's own sampler for the terminal group: the thinning sampler of Sec. 2.2.
  *
  * Everything up to the first rejection is pcg_verify's per-position stage (label, acceptance, first-reject scan).
  * The group at the rejected position is then drawn WITHOUT enumerating the groups.  Trial r = 0, 1, ... draws a

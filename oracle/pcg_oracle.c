@@ -214,7 +214,7 @@ static int32_t draw_label(int32_t x, double u, const double *weights, const int3
  * uniforms[K][1]        : terminal within-group token draw
  *
  * Terminal group, two ways.  thin == NULL: enumerate the residual over all groups and invert its CDF with
- * uniforms[K][0].  thin != NULL ([B, n_trials, 3]): the paper's own sampler, "Residual sampling via thinning"
+ * uniforms[K][0].  thin != NULL ([B, n_trials, 3]): the thinning sampler of the paper
  * (Sec. 2.2), which never enumerates the groups.  Trial r uses thin[r][0] to draw a token y from the target
  * row by inverse CDF in token order, thin[r][1] to draw y's label k ~ w_{.,y} (so that k ~ the target's coarse
  * distribution), and keeps k if thin[r][2] < [1 - draft mass(k) / target mass(k)]_+; otherwise the next trial

@@ -1,4 +1,4 @@
-// Terminal group by thinning ("Residual sampling via thinning", Sec. 2.2) -- included by pcg_kernels.cu inside
+// Terminal group by thinning (the thinning paragraph of Sec. 2.2) -- included by pcg_kernels.cu inside
 // namespace pcg, after the helpers of the batched terminal stage.
 //
 // The paper's sampler never enumerates the groups: a candidate (y, k) is drawn with y ~ target and k ~ w_{.,y}

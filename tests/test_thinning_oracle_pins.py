@@ -1,4 +1,4 @@
-"""Pins for the oracle's thinning sampler (the paper's "Residual sampling via thinning", Sec. 2.2).
+"""Pins for the oracle's thinning sampler (the thinning paragraph of the paper's Sec. 2.2).
 
 Nothing here re-types the sampler.  The checks are the facts the paper states about it, measured on the oracle's
 output over many seeded random uniforms (tolerances are five standard deviations of the estimate):
