@@ -729,9 +729,10 @@ constexpr int kSpmmThreads = PCG_SPMM_THREADS;  // group_spmm_kernel: warps of 8
 #define PCG_SPMM_DEPTH 8  // tokens per batch of the sparse product; two batches of loads are in flight per lane
 #endif
 #ifndef PCG_SPMM_GW
-#define PCG_SPMM_GW 4  // consecutive groups per warp of the sparse product
+#define PCG_SPMM_GW 4  // consecutive groups per warp of the sparse product when the launch has many waves
 #endif
 constexpr int kSpmmGroupsPerWarp = PCG_SPMM_GW;
+constexpr int kSpmmMaxGroupsPerWarp = 8;  // chosen per launch between 2 and this (see launch_spmm)
 constexpr int kSpmmWide = PCG_SPMM_SPL;
 constexpr int kSpmmDepth = PCG_SPMM_DEPTH;
 constexpr int kDrawThreads = 512;  // terminal_draw_kernel
@@ -1008,6 +1009,7 @@ struct SpmmArgs {
     int b0;           // first sequence of this chunk
     int bpad;
     float *R;         // [B, M] (raw sums; the consumer clamps at zero)
+    int gw;           // consecutive groups per warp, at most kSpmmMaxGroupsPerWarp
 };
 
 template <int SPL>
@@ -1043,7 +1045,7 @@ struct SeqVec<8> {  // one 256-bit load per lane
     }
 };
 
-// Grid (ceil(M / (GW * warps per block)), bpad / (32 * SPL)).  A warp owns GW (4) consecutive groups -- their token
+// Grid (ceil(M / (GW * warps per block)), bpad / (32 * SPL)).  A warp owns GW = a.gw consecutive groups -- their token
 // lists are one contiguous range of the CSR -- and a block of 32 * SPL sequences; a lane holds SPL consecutive
 // sequences (one 4-, 16- or 32-byte load per token).  The range is walked in batches of DEPTH tokens with two
 // register buffers: the loads of batch i+1 are issued before batch i is added, so a warp keeps up to 2 * DEPTH
@@ -1055,12 +1057,12 @@ template <int SPL, int DEPTH, bool HAS_W>
 __global__ void __launch_bounds__(kSpmmThreads) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
     pdl_enter();
     constexpr int NS = 32 * SPL;  // sequences per warp
-    constexpr int GW = kSpmmGroupsPerWarp;
+    const int GW = a.gw;
     constexpr int TS = NS + 4;    // row stride of the result tile (keeps 16-byte alignment, spreads banks)
     static_assert(32 % DEPTH == 0, "a batch never straddles two blocks of 32 token ids");
-    __shared__ __align__(16) float tiles[(kSpmmThreads / 32) * GW * TS];
+    __shared__ __align__(16) float tiles[(kSpmmThreads / 32) * kSpmmMaxGroupsPerWarp * TS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float *tile = tiles + warp * GW * TS;
+    float *tile = tiles + warp * kSpmmMaxGroupsPerWarp * TS;
     const int g0 = (blockIdx.x * (kSpmmThreads / 32) + warp) * GW;
     if (g0 >= G.M) return;  // warp-uniform; the kernel has no block-wide barrier
     const int ng = min(GW, G.M - g0);
@@ -1540,29 +1542,58 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
     return w;
 }
 
+// Groups per warp for a launch of `warps_y` warp rows over M groups.  All warps take about the same time, so a
+// launch of 1.7 waves costs two: with few waves the groups per warp are chosen to fill whole waves (C5: 7 groups
+// per warp = 586 blocks on 592 resident ones, instead of 4 = 1024 blocks = 1.73 waves); with many waves the
+// measured best, kSpmmGroupsPerWarp.
+static int spmm_groups_per_warp(int M, int64_t warps_y, int64_t resident_blocks) {
+    const int wpb = kSpmmThreads / 32;
+    auto waves = [&](int gw) {
+        const int64_t blocks = ((M + gw - 1) / gw + wpb - 1) / wpb * warps_y;
+        return (blocks + resident_blocks - 1) / resident_blocks;
+    };
+    if (waves(kSpmmGroupsPerWarp) > 4) return kSpmmGroupsPerWarp;  // many waves: the tail no longer matters
+    int best = kSpmmGroupsPerWarp;
+    int64_t best_cost = waves(best) * best;  // time ~ waves x work per warp
+    for (int gw = kSpmmMaxGroupsPerWarp; gw >= 2; --gw)
+        if (waves(gw) * gw < best_cost) {
+            best = gw;
+            best_cost = waves(gw) * gw;
+        }
+    return best;
+}
+
 // The sparse product over nb blocks of 32 sequences (nb a multiple of `lanes`, the sequences per lane: 8, 4 or 1).
-static void launch_spmm(const SpmmArgs &sp, int nb, int lanes, const GroupsDev &G, cudaStream_t cs) {
-    const int gpb = kSpmmGroupsPerWarp * (kSpmmThreads / 32);  // groups per block
-    const unsigned gx = (unsigned)((G.M + gpb - 1) / gpb);
+static void launch_spmm(SpmmArgs sp, int nb, int lanes, const GroupsDev &G, int sm_count, cudaStream_t cs) {
     const bool has_w = G.pair_w != nullptr;
+    auto go = [&](auto kern, int slot) {
+        static int occupancy[6];  // resident blocks per SM of each variant (0 = not asked yet; a benign race)
+        if (occupancy[slot] == 0) {
+            int occ = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kSpmmThreads, 0) != cudaSuccess || occ < 1) occ = 4;
+            occupancy[slot] = occ;
+        }
+        const int64_t wy = nb / lanes;
+        sp.gw = spmm_groups_per_warp(G.M, wy, (int64_t)occupancy[slot] * sm_count);
+        const int gpb = sp.gw * (kSpmmThreads / 32);  // groups per block
+        const dim3 grid((unsigned)((G.M + gpb - 1) / gpb), (unsigned)wy);
+        launch_after(kern, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+    };
     if (lanes == 8) {
-        const dim3 grid(gx, (unsigned)(nb / 8));
         if (has_w)
-            launch_after(group_spmm_kernel<8, 4, true>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+            go(group_spmm_kernel<8, 4, true>, 0);
         else
-            launch_after(group_spmm_kernel<8, 4, false>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+            go(group_spmm_kernel<8, 4, false>, 1);
     } else if (lanes == kSpmmWide) {
-        const dim3 grid(gx, (unsigned)(nb / kSpmmWide));
         if (has_w)
-            launch_after(group_spmm_kernel<kSpmmWide, kSpmmDepth, true>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+            go(group_spmm_kernel<kSpmmWide, kSpmmDepth, true>, 2);
         else
-            launch_after(group_spmm_kernel<kSpmmWide, kSpmmDepth, false>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+            go(group_spmm_kernel<kSpmmWide, kSpmmDepth, false>, 3);
     } else {
-        const dim3 grid(gx, (unsigned)nb);
         if (has_w)
-            launch_after(group_spmm_kernel<1, 16, true>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+            go(group_spmm_kernel<1, 16, true>, 4);
         else
-            launch_after(group_spmm_kernel<1, 16, false>, grid, dim3(kSpmmThreads), 0, cs, sp, G);
+            go(group_spmm_kernel<1, 16, false>, 5);
     }
 }
 
@@ -1605,7 +1636,7 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
             TransposeArgs tr{base, base, nr, 0, 0, chunk, s, groups->probs_zero, groups->probs_stats, groups->probs_dt};
             const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
             PCG_DISPATCH_DTYPE(dtype, launch_after(residual_transpose_kernel<LogitT>, tgrid, dim3(kTrThreads), 0, cs, tr, G));
-            launch_spmm(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M}, nb, lanes, G, cs);
+            launch_spmm(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M, 0}, nb, lanes, G, groups->sm_count, cs);
         }
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching the batched group-probability kernels");
@@ -1734,7 +1765,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
                 PCG_DISPATCH_DTYPE(dtype, launch_after(residual_transpose_kernel<LogitT>, tgrid, dim3(kTrThreads), 0, cs, tr, G));
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
-                launch_spmm(SpmmArgs{w.Dt, B, b0, chunk, w.R}, nb, lanes, G, cs);
+                launch_spmm(SpmmArgs{w.Dt, B, b0, chunk, w.R, 0}, nb, lanes, G, groups->sm_count, cs);
                 e = cudaGetLastError();
                 if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
             }
