@@ -110,7 +110,7 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
-def oracle_leg(cfg, groups, batch, min_seconds=2.0, max_passes=200):
+def oracle_leg(cfg, groups, batch, min_seconds=2.0, max_passes=200, timed_outputs=None):
     """Time the CPU oracle, as it stands, with all host cores: whole passes over (a bounded sample of) the batch,
     repeated until about `min_seconds` of wall time (tens of core-seconds of CPU work) have been spent."""
     import oracle
@@ -119,11 +119,13 @@ def oracle_leg(cfg, groups, batch, min_seconds=2.0, max_passes=200):
     cores = oracle.max_threads()
     B = batch.draft_tokens.shape[0]
 
+    last = {}
+
     def one_pass(nseq):
         t0 = time.perf_counter()
-        oracle.verify(batch.target_logits[:nseq], batch.draft_logits[:nseq], batch.draft_tokens[:nseq],
-                      groups.group_ptr, groups.group_tok, groups.tok_degree, batch.uniforms[:nseq], batch.temperature,
-                      threads=cores)
+        last["ref"] = oracle.verify(batch.target_logits[:nseq], batch.draft_logits[:nseq], batch.draft_tokens[:nseq],
+                                    groups.group_ptr, groups.group_tok, groups.tok_degree, batch.uniforms[:nseq],
+                                    batch.temperature, threads=cores)
         return time.perf_counter() - t0
 
     probe = max(one_pass(min(B, 8)), 1e-5)  # sizes the sample so that one pass stays below ~min_seconds
@@ -132,10 +134,19 @@ def oracle_leg(cfg, groups, batch, min_seconds=2.0, max_passes=200):
     while passes < max_passes and (spent < min_seconds or passes < 2):
         spent += one_pass(nseq)
         passes += 1
-    return {"value": nseq * cfg.K * passes / spent, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {nseq} of {B} sequences of {cfg.name} ({nseq * cfg.K} drafted positions), {passes} "
-                      f"passes, {spent:.3f} s wall on {cores} threads (OpenMP over sequences; the oracle stops a "
-                      f"sequence at its first rejection, as Algorithm 1 does)"}
+    out = {"value": nseq * cfg.K * passes / spent, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"first {nseq} of {B} sequences of {cfg.name} ({nseq * cfg.K} drafted positions), {passes} "
+                     f"passes, {spent:.3f} s wall on {cores} threads (OpenMP over sequences; the oracle stops a "
+                     f"sequence at its first rejection, as Algorithm 1 does)"}
+    if timed_outputs is not None:
+        # the oracle's results on that sample against what the timed GPU steps produced, decision by decision
+        from oracle.compare import compare_verify
+
+        n, tok, grp = (a[:nseq] for a in timed_outputs)
+        cmp = compare_verify(n, tok, grp, last["ref"], band=1e-6)
+        out["parity_of_timed_outputs"] = {"sequences": int(nseq), "hard_mismatches": int(cmp.hard),
+                                          "excused_within_1e-6": int(cmp.excused)}
+    return out
 
 
 def run_reference(args, cfg, rank):
@@ -414,6 +425,19 @@ def main():
                 "trials_supplied": args.thin_trials, "trials_mean": float(tr.mean()), "trials_max": int(tr.max()),
                 "sequences_exhausted": int((thin_out[3] & binding.FLAG_THINNING_EXHAUSTED).ne(0).sum()),
                 "accept_lengths_equal_to_timed_mode": bool(torch.equal(thin_out[0], out[0]))}
+        # workload statistics on a sample of drafted positions: how much coarse-graining raises the overlap of the
+        # two models (sum_g min(P, Q) against sum_t min(p, q); the former is the group-level acceptance probability)
+        ns = min(B, 64)
+        t_rows = tl[:ns, 0].contiguous()
+        d_rows = dl[:ns, 0].contiguous()
+        Pg = binding.pcg_group_probs(t_rows, handle, cfg.temperature)
+        Qg = binding.pcg_group_probs(d_rows, handle, cfg.temperature)
+        pt = torch.softmax(t_rows.float() / cfg.temperature, dim=1)
+        qt = torch.softmax(d_rows.float() / cfg.temperature, dim=1)
+        extras["workload_statistics"] = {
+            "positions_sampled": ns,
+            "group_overlap_sum_min_PQ": float(torch.minimum(Pg, Qg).sum(dim=1).mean()),
+            "token_overlap_sum_min_pq": float(torch.minimum(pt, qt).sum(dim=1).mean())}
         d_emb = 512 if V >= 32768 else 128
         gen = torch.Generator(device="cuda")
         gen.manual_seed(2511)
@@ -461,7 +485,9 @@ def main():
             "mean_accept_len": float(accept_len.mean()),
         }
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = oracle_leg(cfg, groups, batch)
+            line["cpu_baseline"] = oracle_leg(
+                cfg, groups, batch,
+                timed_outputs=None if thinning else tuple(t.cpu().numpy() for t in out[:3]))
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
