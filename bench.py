@@ -34,7 +34,7 @@ UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
 # dram__bytes_read.sum + dram__bytes_write.sum of one position_kernel launch, from the ncu capture summarised in
 # profiles/ (null until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {"C5": 1076235520 + 12602880}
+NCU_TRAFFIC_BYTES = {"C5": 1076131840 + 12466432}
 
 
 def hbm_peak():
