@@ -183,10 +183,31 @@ def run_reference(args, cfg, rank):
     print(json.dumps(line), flush=True)
 
 
+L2_BYTES = 126 << 20
+
+
+def input_copies(cfg):
+    """How many rotating copies of the inputs the timed steps walk through: one when a batch alone exceeds the L2,
+    else enough for twice the L2 (at most 64)."""
+    esz = 4 if cfg.dtype == "f32" else 2
+    nbytes = cfg.B * (2 * cfg.K + 1) * cfg.V * esz
+    return 1 if nbytes > L2_BYTES else int(min(64, -(-2 * L2_BYTES // nbytes)))
+
+
 def workload_config(cfg):
+    esz = 4 if cfg.dtype == "f32" else 2
+    nbytes = cfg.B * (2 * cfg.K + 1) * cfg.V * esz
+    copies = input_copies(cfg)
+    if copies == 1:
+        l2 = "not flushed: each step streams the whole batch, larger than the 126 MB L2"
+    elif copies * nbytes > L2_BYTES:
+        l2 = (f"not flushed: the timed steps rotate over {copies} copies of the inputs, {copies * nbytes / 2**20:.0f} MB "
+              f"in all, larger than the 126 MB L2")
+    else:
+        l2 = (f"not flushed: the timed steps rotate over {copies} copies of the inputs, only {copies * nbytes / 2**20:.1f} MB "
+              f"in all, so the inputs stay in the 126 MB L2 (launch-latency-bound case, not a bandwidth figure)")
     return {"workload": cfg.name, "B": cfg.B, "K": cfg.K, "V": cfg.V, "M": cfg.M, "logits_dtype": cfg.dtype,
-            "temperature": cfg.temperature, "membership": f"{cfg.groups} (mean degree {cfg.degree})",
-            "l2": "not flushed: each step streams the whole batch, larger than the 126 MB L2"}
+            "temperature": cfg.temperature, "membership": f"{cfg.groups} (mean degree {cfg.degree})", "l2": l2}
 
 
 def main():
@@ -266,14 +287,22 @@ def main():
     thin_ws = torch.empty(binding.pcg_verify_thinning_workspace_bytes(B, K, V, M, dt_code), dtype=torch.uint8, device="cuda")
     thin_out = tuple(torch.empty_like(t) for t in out) + (torch.empty(B, dtype=torch.int32, device="cuda"),)
 
+    # small workloads: rotate over several copies of the inputs so that they are not simply served from the L2
+    rotation = [(tl, dl, x, u)] + [(tl.clone(), dl.clone(), x.clone(), u.clone()) for _ in range(input_copies(cfg) - 1)]
+    turn = [0]
+
     def thin_step(events=None):
-        binding.pcg_verify_thinning(tl, dl, x, handle, u, thin_u, cfg.temperature, workspace=thin_ws, out=thin_out,
-                                    stage_events=events)
+        a_tl, a_dl, a_x, a_u = rotation[turn[0] % len(rotation)]
+        turn[0] += 1
+        binding.pcg_verify_thinning(a_tl, a_dl, a_x, handle, a_u, thin_u, cfg.temperature, workspace=thin_ws,
+                                    out=thin_out, stage_events=events)
 
     def step(events=None):
         if thinning:
             return thin_step(events)
-        binding.pcg_verify(tl, dl, x, handle, u, cfg.temperature, workspace=ws, out=out, stage_events=events,
+        a_tl, a_dl, a_x, a_u = rotation[turn[0] % len(rotation)]
+        turn[0] += 1
+        binding.pcg_verify(a_tl, a_dl, a_x, handle, a_u, cfg.temperature, workspace=ws, out=out, stage_events=events,
                            mode=mode)
 
     def barrier():
