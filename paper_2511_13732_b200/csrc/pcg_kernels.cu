@@ -15,6 +15,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <atomic>
 #include <mutex>
 
 #include "pcg_common.cuh"
@@ -1567,14 +1568,14 @@ static int spmm_groups_per_warp(int M, int64_t warps_y, int64_t resident_blocks)
 static void launch_spmm(SpmmArgs sp, int nb, int lanes, const GroupsDev &G, int sm_count, cudaStream_t cs) {
     const bool has_w = G.pair_w != nullptr;
     auto go = [&](auto kern, int slot) {
-        static int occupancy[6];  // resident blocks per SM of each variant (0 = not asked yet; a benign race)
-        if (occupancy[slot] == 0) {
-            int occ = 0;
+        static std::atomic<int> occupancy[6];  // resident blocks per SM of each variant (0 = not asked yet)
+        int occ = occupancy[slot].load(std::memory_order_relaxed);
+        if (occ == 0) {
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kSpmmThreads, 0) != cudaSuccess || occ < 1) occ = 4;
-            occupancy[slot] = occ;
+            occupancy[slot].store(occ, std::memory_order_relaxed);
         }
         const int64_t wy = nb / lanes;
-        sp.gw = spmm_groups_per_warp(G.M, wy, (int64_t)occupancy[slot] * sm_count);
+        sp.gw = spmm_groups_per_warp(G.M, wy, (int64_t)occ * sm_count);
         const int gpb = sp.gw * (kSpmmThreads / 32);  // groups per block
         const dim3 grid((unsigned)((G.M + gpb - 1) / gpb), (unsigned)wy);
         launch_after(kern, grid, dim3(kSpmmThreads), 0, cs, sp, G);
