@@ -1,21 +1,23 @@
 // Kernels and entry points of libpcg: PCG group-level verification on sm_100a.
 //
-// Two kernels make up pcg_verify:
 //   position_kernel  one thread block per drafted position (b,i).  Streams the target and the draft row once
-//                    (online max/sum softmax statistics, 128-bit loads), draws the group label of the draft
+//                    (softmax statistics with a lazy reference, 128-bit loads), draws the group label of the draft
 //                    token, forms the label group's target and draft mass from a handful of gathered logits and
 //                    takes the accept decision.  This kernel moves ~all of the bytes.
-//   terminal_kernel  one thread-block cluster per sequence.  Finds the first rejected position with a warp
-//                    ballot, re-reads that position's rows, builds the residual (P-Q)_+ (or P for the bonus
-//                    token) of ALL groups with a token-sliced segmented reduction in shared memory, combines the
-//                    slices over distributed shared memory, scans it, draws the group, draws the token inside
-//                    it and writes the outputs.
-// pcg_group_probs uses the same token-sliced aggregation to write P of every row.
+// The per-sequence stage of pcg_verify (first rejection, residual (P-Q)_+ of ALL groups at that position, group
+// draw, token draw, outputs) exists in two forms:
+//   terminal_kernel  one thread-block cluster per sequence: a token-sliced segmented reduction in shared memory,
+//                    slices combined over distributed shared memory (a handful of sequences: lowest latency).
+//   batched          terminal_prepare_kernel, residual_transpose_kernel, group_spmm_kernel, terminal_draw_kernel:
+//                    the residual of all sequences as one sparse product over a transposed, L2-resident operand.
+// pcg_group_probs writes P of every row with the same two aggregations; pcg_verify_thinning replaces the
+// per-sequence stage by thinning_kernel (pcg_thinning.cuh), which enumerates nothing.  Every kernel after the
+// first of a call is launched with programmatic stream serialisation (pdl_enter, launch_after).
 #include <cooperative_groups.h>
 
 #include <algorithm>
-#include <cmath>
 #include <atomic>
+#include <cmath>
 #include <mutex>
 
 #include "pcg_common.cuh"
@@ -710,8 +712,8 @@ __global__ void __launch_bounds__(kAggThreads, 2) terminal_kernel(TerminalArgs a
 //                              if everything was accepted, the softmax statistics of the bonus row
 //   residual_transpose_kernel  re-reads the two rows of every sequence's terminal position and writes D
 //                              TRANSPOSED, Dt[t, b]: the sequences of a chunk side by side in one line
-//   group_spmm_kernel          one warp per (4 groups, block of sequences): walks the groups' token lists once
-//                              and adds one fully used line of Dt per token (Dt stays in L2)
+//   group_spmm_kernel          one warp per (a few consecutive groups, block of 32 to 256 sequences): walks the
+//                              groups' token lists once and adds one row segment of Dt per token (Dt stays in L2)
 //   terminal_draw_kernel       one block per sequence: prefix scan over the M residual masses, group draw,
 //                              within-group token draw, outputs
 // Sequences are processed in chunks whose Dt fits in L2.
@@ -722,12 +724,12 @@ constexpr int kTrThreads = 256;    // residual_transpose_kernel
 #ifndef PCG_SPMM_THREADS
 #define PCG_SPMM_THREADS 128
 #endif
-constexpr int kSpmmThreads = PCG_SPMM_THREADS;  // group_spmm_kernel: warps of 8 groups each
+constexpr int kSpmmThreads = PCG_SPMM_THREADS;  // group_spmm_kernel
 #ifndef PCG_SPMM_SPL
-#define PCG_SPMM_SPL 4    // sequences per lane of the sparse product for batches of at least 32 * PCG_SPMM_SPL
+#define PCG_SPMM_SPL 4    // sequences per lane of the sparse product for batches of 128 to 255 sequences (8 beyond, 1 below)
 #endif
 #ifndef PCG_SPMM_DEPTH
-#define PCG_SPMM_DEPTH 8  // tokens per batch of the sparse product; two batches of loads are in flight per lane
+#define PCG_SPMM_DEPTH 8  // tokens per batch of that form of the sparse product; two batches of loads are in flight per lane
 #endif
 #ifndef PCG_SPMM_GW
 #define PCG_SPMM_GW 4  // consecutive groups per warp of the sparse product when the launch has many waves
