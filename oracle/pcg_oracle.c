@@ -47,6 +47,11 @@
 
 /* flag bits written per sequence */
 #define ORACLE_FLAG_ZERO_RESIDUAL 2 /* reject taken but sum of (P-Q)_+ was <= 0 */
+/* Candidate-token order of the thinning sampler (the paper fixes the law y ~ target, not how a uniform is mapped
+ * to y).  Reading of this library: the inverse CDF runs over the tokens taken slot by slot, where the slot of
+ * token t is (t div W) mod 128 and W is the number of logits in 16 bytes (4 for float, 8 for the 16-bit types);
+ * inside a slot tokens ascend. */
+#define ORACLE_CANDIDATE_SLOTS 128
 #define ORACLE_FLAG_THINNING_EXHAUSTED 8 /* every supplied thinning trial was turned down; enumerated draw used */
 
 /* IEEE binary16 bit pattern to double, from the format's definition: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
@@ -216,7 +221,7 @@ static int32_t draw_label(int32_t x, double u, const double *weights, const int3
  * Terminal group, two ways.  thin == NULL: enumerate the residual over all groups and invert its CDF with
  * uniforms[K][0].  thin != NULL ([B, n_trials, 3]): the thinning sampler of the paper
  * (Sec. 2.2), which never enumerates the groups.  Trial r uses thin[r][0] to draw a token y from the target
- * row by inverse CDF in token order, thin[r][1] to draw y's label k ~ w_{.,y} (so that k ~ the target's coarse
+ * row by inverse CDF over the tokens in candidate order (cand_order, see ORACLE_CANDIDATE_SLOTS), thin[r][1] to draw y's label k ~ w_{.,y} (so that k ~ the target's coarse
  * distribution), and keeps k if thin[r][2] < [1 - draft mass(k) / target mass(k)]_+; otherwise the next trial
  * draws a new (y, k).  After all accepted positions (no rejection) there is no draft mass: the first candidate
  * is kept, which draws the bonus group from the target's coarse distribution.  The paper's sampler is not
@@ -231,9 +236,10 @@ static void verify_sequence(const void *target_logits, const void *draft_logits,
                             double T, const int32_t *draft_tokens, int M, const int32_t *group_ptr,
                             const int32_t *group_tok, const int32_t *tok_degree, const double *weights,
                             const int32_t *rev_ptr, const int32_t *rev_grp, const int32_t *rev_nz,
-                            const float *uniforms, const float *thin, int n_trials, double accept_bias,
-                            int32_t *accept_len, int32_t *tokens, int32_t *groups, int32_t *flags, int32_t *trials,
-                            double *margins, double *p, double *q, double *P, double *Q, double *R) {
+                            const float *uniforms, const float *thin, int n_trials, const int32_t *cand_order,
+                            double *pm, double accept_bias, int32_t *accept_len, int32_t *tokens, int32_t *groups,
+                            int32_t *flags, int32_t *trials, double *margins, double *p, double *q, double *P,
+                            double *Q, double *R) {
     const float *u = uniforms + b * (int64_t)(K + 1) * 2;
     int32_t *tok_out = tokens + b * (int64_t)(K + 1);
     int32_t *grp_out = groups + b * (int64_t)(K + 1);
@@ -278,9 +284,10 @@ static void verify_sequence(const void *target_logits, const void *draft_logits,
     if (thin) {
         const float *tu = thin + b * (int64_t)n_trials * 3;
         int used = 0;
+        for (int t = 0; t < V; ++t) pm[t] = p[cand_order[t]]; /* target masses in candidate order */
         for (int r = 0; r < n_trials && gs < 0; ++r) {
             double m_tok = INFINITY, m_lab = INFINITY, m_keep = INFINITY;
-            int y = inverse_cdf(p, V, (double)tu[3 * r], NULL, &m_tok);            /* y ~ target */
+            int y = cand_order[inverse_cdf(pm, V, (double)tu[3 * r], NULL, &m_tok)]; /* y ~ target */
             int32_t k = draw_label(y, (double)tu[3 * r + 1], weights, rev_ptr, rev_grp, rev_nz, &m_lab); /* k ~ w_{.,y} */
             int keep = 1;
             if (have_Q) { /* thinning probability a(k) = [1 - draft mass / target mass]_+ */
@@ -374,6 +381,17 @@ static int verify_batch(const void *target_logits, const void *draft_logits, int
         }
     for (int64_t k = 0; k < (int64_t)B * K; ++k)
         if (draft_tokens[k] < 0 || draft_tokens[k] >= V) return 4;
+    /* candidate order of the thinning sampler: slot-major, ascending inside a slot */
+    int32_t *cand_order = NULL;
+    if (thin) {
+        cand_order = (int32_t *)malloc(sizeof(int32_t) * (size_t)V);
+        if (!cand_order) return 2;
+        const int W = dtype == ORACLE_F32 ? 4 : 8;
+        int n = 0;
+        for (int slot = 0; slot < ORACLE_CANDIDATE_SLOTS; ++slot)
+            for (int t = 0; t < V; ++t)
+                if ((t / W) % ORACLE_CANDIDATE_SLOTS == slot) cand_order[n++] = t;
+    }
     int nthreads = threads;
 #ifdef _OPENMP
     if (nthreads <= 0) nthreads = omp_get_max_threads();
@@ -388,7 +406,8 @@ static int verify_batch(const void *target_logits, const void *draft_logits, int
         double *P = (double *)malloc(sizeof(double) * (size_t)M);
         double *Q = (double *)malloc(sizeof(double) * (size_t)M);
         double *R = (double *)malloc(sizeof(double) * (size_t)M);
-        if (!p || !q || !P || !Q || !R) {
+        double *pm = (double *)malloc(sizeof(double) * (size_t)V);
+        if (!p || !q || !P || !Q || !R || !pm) {
 #pragma omp atomic write
             failed = 1;
         } else {
@@ -396,19 +415,21 @@ static int verify_batch(const void *target_logits, const void *draft_logits, int
             for (int b = 0; b < B; ++b)
                 verify_sequence(target_logits, draft_logits, dtype, b, K, V, (double)temperature, draft_tokens, M,
                                 group_ptr, group_tok, tok_degree, weights, rev_ptr, rev_grp, rev_nz, uniforms,
-                                thin, n_trials, accept_bias, accept_len, tokens, groups, flags, trials, margins,
-                                p, q, P, Q, R);
+                                thin, n_trials, cand_order, pm, accept_bias, accept_len, tokens, groups, flags,
+                                trials, margins, p, q, P, Q, R);
         }
         free(p);
         free(q);
         free(P);
         free(Q);
         free(R);
+        free(pm);
     }
     free(rev_ptr);
     free(rev_grp);
     free(rev_nz);
     free(fill);
+    free(cand_order);
     return failed ? 2 : 0;
 }
 

@@ -56,8 +56,9 @@ PIN_CALLS = (
 THIN_MUTATIONS = [
     ("thinning_ratio_inverted", "double a = P[k] > 0.0 ? 1.0 - Q[k] / P[k] : 0.0;",
      "double a = Q[k] > 0.0 ? 1.0 - P[k] / Q[k] : 0.0;", 0),
-    ("thinning_candidate_from_draft", "int y = inverse_cdf(p, V, (double)tu[3 * r], NULL, &m_tok);",
-     "int y = inverse_cdf(have_Q ? q : p, V, (double)tu[3 * r], NULL, &m_tok);", 0),
+    ("thinning_candidate_from_draft", "pm[t] = p[cand_order[t]];", "pm[t] = (have_Q ? q : p)[cand_order[t]];", 0),
+    ("thinning_candidate_order_is_plain_token_order", "if ((t / W) % ORACLE_CANDIDATE_SLOTS == slot) cand_order[n++] = t;",
+     "if (slot == 0) cand_order[n++] = t;", 0),
     ("thinning_keep_uses_label_uniform", "keep = (double)tu[3 * r + 2] < a;", "keep = (double)tu[3 * r + 1] < a;", 0),
     ("thinning_label_uses_token_uniform", "draw_label(y, (double)tu[3 * r + 1], weights,", "draw_label(y, (double)tu[3 * r], weights,", 0),
     ("thinning_bonus_is_thinned_too", "if (have_Q) { /* thinning probability", "if (1) { /* thinning probability", 0),
@@ -71,7 +72,8 @@ THIN_PIN_CALLS = (
     + [lambda o, s=s: thin_pins.test_thinning_bonus_is_one_candidate_from_the_target(o, s) for s in (11,)]
     + [lambda o: thin_pins.test_thinning_with_singleton_groups_is_token_level_residual_sampling(o),
        lambda o: thin_pins.test_thinning_exhaustion_falls_back_to_the_enumerated_draw(o),
-       lambda o: thin_pins.test_thinning_never_reads_trials_it_does_not_reach(o)]
+       lambda o: thin_pins.test_thinning_never_reads_trials_it_does_not_reach(o),
+       lambda o: thin_pins.test_thinning_candidate_order_is_slot_major(o, thin_pins.np.float32, 4)]
 )
 
 

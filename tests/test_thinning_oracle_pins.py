@@ -9,7 +9,10 @@ output over many seeded random uniforms (tolerances are five standard deviations
   * after an all-accepted sequence one candidate is drawn and the bonus token follows the target p;
   * singleton groups give token-level residual sampling (p - q)_+;
   * when every supplied trial is turned down the result is the enumerated draw (pinned on its own elsewhere);
-  * uniforms of trials that are never reached do not matter.
+  * uniforms of trials that are never reached do not matter;
+  * the mapping from the token uniform to the candidate is the documented one: inverse CDF over the tokens taken
+    slot by slot (slot = (t div W) mod 128, W logits per 16 bytes), checked on a uniform target where the candidate
+    is simply the floor(u V)-th token of that order.
 """
 import numpy as np
 import pytest
@@ -158,3 +161,24 @@ def test_thinning_never_reads_trials_it_does_not_reach(oracle):
     tu3[:, 0, 0] = _uniforms(rng, (N,))
     res3 = _run(oracle, groups, tl, dl, x, u, tu3)
     assert not np.array_equal(res3.groups, res.groups)
+
+
+@pytest.mark.parametrize("dtype,W_", [(np.float32, 4), (np.float16, 8)])
+def test_thinning_candidate_order_is_slot_major(oracle, dtype, W_):
+    """Uniform target, singleton groups, draft == target (every position accepted): the bonus token is the first
+    candidate itself, which must be the floor(u V)-th token in slot-major order."""
+    V = 2600  # more than 128 * W tokens, not a multiple of it
+    order = sorted(range(V), key=lambda t: ((t // W_) % 128, t))
+    assert order[:3] == [0, 1, 2] and order[W_] == 128 * W_  # after the first 16-byte word comes the word 128 further on
+    g = W.groups_from_lists(V, [[t] for t in range(V)])
+    idx = np.array([0, 1, W_, W_ + 1, 777, 1300, V - 2, V - 1])
+    N = idx.size
+    tl = np.zeros((N, 2, V), dtype)
+    dl = np.zeros((N, 1, V), dtype)
+    u = np.zeros((N, 2, 2), np.float32)
+    u[:, 1, 1] = 0.5
+    tu = np.zeros((N, 2, 3), np.float32)
+    tu[:, 0, 0] = ((idx + 0.5) / V).astype(np.float32)
+    res = oracle.verify(tl, dl, np.zeros((N, 1), np.int32), g.group_ptr, g.group_tok, g.tok_degree, u, thin_uniforms=tu)
+    assert np.all(res.accept_len == 1) and np.all(res.trials == 1)
+    assert res.tokens[:, 1].tolist() == [order[i] for i in idx]
