@@ -293,7 +293,9 @@ pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits
  *
  * Everything up to the first rejection is pcg_verify's per-position stage (label, acceptance, first-reject scan).
  * The group at the rejected position is then drawn WITHOUT enumerating the groups.  Trial r = 0, 1, ... draws a
- * token y from the target row by inverse CDF in token order with thin_uniforms[b, r, 0], a label k ~ w_{.,y} over
+ * token y from the target row by inverse CDF with thin_uniforms[b, r, 0] over the tokens taken slot by slot (the
+ * slot of token t is (t div W) mod 128 with W = 16 bytes / bytes per logit, tokens ascending inside a slot: the
+ * order in which the library's streaming kernel sums a row, so that the slot masses cost nothing), a label k ~ w_{.,y} over
  * the groups containing y with thin_uniforms[b, r, 1] (so k follows the target's coarse distribution), and keeps
  * k if thin_uniforms[b, r, 2] < [1 - Q(k)/P(k)]_+ (draft mass over target mass of group k alone); otherwise the
  * next trial draws a new candidate.  The kept group's law is the normalised residual (P - Q)_+ exactly; the
@@ -311,11 +313,12 @@ pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits
  *
  *   thin_uniforms [B, n_trials, 3] float in [0,1), device, read-only; 1 <= n_trials <= 65536
  *   out_trials    [B] int32 or NULL: candidates drawn (1 after an all-accepted sequence; n_trials when exhausted)
- *   workspace     device, 256-byte aligned, at least pcg_verify_thinning_workspace_bytes(...) bytes (28 bytes per
+ *   workspace     device, 256-byte aligned, at least pcg_verify_thinning_workspace_bytes(...) bytes (1052 bytes per
  *                 drafted position plus B*M*4 for sequences whose trials run out); contents need no initialisation
  *   the remaining arguments, ownership, asynchrony (no allocation, no synchronisation, the caller's stream only)
- *   and errors are pcg_verify's; V is limited by the shared memory the tile prefix needs (8 bytes per 16-byte
- *   vector of a row: V <= 3.6 million for 16-bit logits), beyond that PCG_ERR_UNSUPPORTED.
+ *   and errors are pcg_verify's.  Rows that do not start on 16-byte boundaries or are not whole 16-byte words
+ *   long (V * bytes per logit not a multiple of 16) give the same results, a little slower (their slot masses
+ *   are summed by the thinning kernel itself).
  */
 size_t pcg_verify_thinning_workspace_bytes(int32_t B, int32_t K, int32_t V, int32_t M, pcg_dtype dtype);
 pcg_status pcg_verify_thinning(const void *target_logits, const void *draft_logits, pcg_dtype dtype, int32_t B, int32_t K,

@@ -109,6 +109,8 @@ struct PositionArgs {
     int32_t *labels;         // [B*K] group label of the draft token
     int32_t *posflags;       // [B*K]
     float4 *stats;           // [B*K] (RS_p, 1/Z_p, RS_q, 1/Z_q): scaled reference and reciprocal normaliser
+    float2 *strata;          // [B*K, kHalf] or null: every target-row thread's own (reference, sum); thread h has
+                             // summed the 16-byte words h, h + 128, h + 256, ... of the row (see pcg_thinning.cuh)
 };
 
 // Group-label coupling: the label of draft token x is drawn from the groups containing x (reverse membership
@@ -234,6 +236,7 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
         for (int t = head + nvec * NV + htid; t < V; t += H) absorb1(st, Elem<T>::widen(row[t]), s);
     }
     while (chained < kChainSteps) chain(chained++);
+    if (a.strata && half == 0) a.strata[(size_t)pos * H + htid] = make_float2(st.rs, st.acc);  // a free by-product
 
     // ---- per-row (rs, Z): xor butterfly inside a warp, then a fixed-order pass over each half's warps ----
     float rs = st.rs, Z = st.acc;
@@ -1733,7 +1736,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         if (e != cudaSuccess) return cuda_fail(e, "launching dense_accept_kernel");
     } else {
         PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
-                        w.accept,      w.labels,     w.posflags,   w.stats};
+                        w.accept,      w.labels,     w.posflags,   w.stats,  nullptr};
         PCG_DISPATCH_DTYPE(dtype, position_kernel<LogitT><<<B * K, kPosThreads, 0, cs>>>(pa, G));
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
@@ -1801,6 +1804,7 @@ struct ThinWorkspace {
     int32_t *accept, *labels, *posflags;
     float4 *stats;
     float *fallback_rows;
+    float2 *strata;
     size_t bytes;
 };
 static ThinWorkspace carve_thin_workspace(void *base, int64_t B, int64_t K, int64_t M) {
@@ -1817,6 +1821,7 @@ static ThinWorkspace carve_thin_workspace(void *base, int64_t B, int64_t K, int6
     w.labels = (int32_t *)(p + take((size_t)(B * K) * 4));
     w.posflags = (int32_t *)(p + take((size_t)(B * K) * 4));
     w.fallback_rows = (float *)(p + take((size_t)(B * M) * 4));
+    w.strata = (float2 *)(p + take((size_t)(B * K) * kHalf * 8));
     w.bytes = off ? off : 256;
     return w;
 }
@@ -1859,12 +1864,7 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
         set_error("pcg_verify_thinning: B*K too large for one launch");
         return PCG_ERR_UNSUPPORTED;
     }
-    const size_t smem = thin_smem_bytes(G.V, esz);
-    if (smem > kMaxDynSmem) {
-        set_error("pcg_verify_thinning: V=%d needs %zu bytes of shared memory for the tile prefix (limit %zu)", G.V, smem,
-                  kMaxDynSmem);
-        return PCG_ERR_UNSUPPORTED;
-    }
+    const size_t smem = thin_smem_bytes();
     const size_t need = pcg_verify_thinning_workspace_bytes(B, K, G.V, G.M, dtype);
     if (!workspace || ((uintptr_t)workspace & 255u) || workspace_bytes < need) {
         set_error("pcg_verify_thinning: workspace must be 256-byte aligned and hold %zu bytes (got %zu)", need,
@@ -1877,8 +1877,12 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
     cudaError_t e = cudaSuccess;
     if (stage_events) e = cudaEventRecord((cudaEvent_t)stage_events[0], cs);
     if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
+    // Rows that start on 16-byte boundaries and consist of whole 16-byte words: the partial sums the position
+    // kernel's threads hold anyway are exactly the slot masses the candidate draw needs (slot of token t =
+    // (t div W) mod 128), so the thinning kernel needs no pass of its own over the row.
+    const bool strata = ((uintptr_t)target_logits & 15u) == 0 && ((size_t)G.V * esz) % 16 == 0;
     PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
-                    w.accept,      w.labels,     w.posflags,   w.stats};
+                    w.accept,      w.labels,     w.posflags,   w.stats,  strata ? w.strata : nullptr};
     PCG_DISPATCH_DTYPE(dtype, position_kernel<LogitT><<<B * K, kPosThreads, 0, cs>>>(pa, G));
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
@@ -1888,7 +1892,8 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
     }
     ThinArgs ta{target_logits, draft_logits, draft_tokens, uniforms,        thin_uniforms, n_trials,
                 K,             s,            w.accept,     w.labels,        w.posflags,    w.stats,
-                w.fallback_rows, out_accept_len, out_tokens, out_groups,    out_flags,     out_trials};
+                w.fallback_rows, out_accept_len, out_tokens, out_groups,    out_flags,     out_trials,
+                strata ? w.strata : nullptr};
     auto launch = [&](auto kern) -> cudaError_t {
         cudaError_t le = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (le != cudaSuccess) return le;

@@ -3,17 +3,19 @@
 //
 // The paper's sampler never enumerates the groups: a candidate (y, k) is drawn with y ~ target and k ~ w_{.,y}
 // (so k follows the target's coarse distribution) and kept with probability [1 - Q(k)/P(k)]_+, which needs the
-// two masses of group k only.  One block per sequence:
+// two masses of group k only.  The candidate token is drawn by inverse CDF over the tokens taken slot by slot:
+// the slot of token t is (t div W) mod 128, W = logits per 16 bytes, tokens ascending inside a slot.  That is the
+// order in which the position kernel's 128 target-row threads sum the row, so the 128 slot masses are a free
+// by-product of that kernel and no pass over the row is needed here.  One block per sequence:
 //   1. first rejection n from the accept bits (warp ballots); row statistics from the position kernel, or, when
 //      every position was accepted, one pass over the bonus row;
-//   2. one streaming pass over the target row of position n: the sum of 2^(l s - RS) over every tile of
-//      32 x 16 bytes, kept in shared memory as an inclusive prefix (double) -- the token-level CDF at tile
-//      granularity;
-//   3. trials, one WARP per trial and all warps at once: binary search for the tile, re-read of that tile (it
-//      sits in L2), in-tile scan for y, label k, the two masses of group k by a warp gather, keep test.  The
-//      first kept candidate in trial order wins, so the result is the sequential sampler's although several
-//      trials run side by side;
-//   4. token inside the kept group and outputs, as in the enumerated path.
+//   2. the 128 slot masses of the target row of position n -- from the position kernel's threads, or (bonus row,
+//      rows that are not made of aligned 16-byte words) summed here -- and their inclusive prefix in double;
+//   3. trials, one WARP per trial and all warps at once: binary search for the slot, scan of the slot's words
+//      (32 at a time, 2 KB apart) for y, label k, the two masses of group k by a warp gather, keep test, token
+//      inside a kept group.  The first kept candidate in trial order wins, so the result is the sequential
+//      sampler's although several trials run side by side;
+//   4. outputs.
 // If all supplied trials are turned down, the block enumerates the residual itself (one thread per group,
 // staged in a row of the workspace) and draws from it with the sequence's terminal-group uniform: same law,
 // flagged PCG_FLAG_THINNING_EXHAUSTED.
@@ -33,19 +35,22 @@ struct ThinArgs {
     const float4 *stats;                        // [B*K]
     float *fallback_rows;                       // [B, M] staging for sequences whose trials ran out
     int32_t *out_accept_len, *out_tokens, *out_groups, *out_flags, *out_trials;
+    const float2 *strata;  // [B*K, kThinSlots] (reference, sum) of every target row's slots from the position kernel, or null
 };
 
-static size_t thin_smem_bytes(int V, size_t esz) {
-    const size_t ts = 32 * (16 / esz);
-    return ((size_t)V + ts - 1) / ts * 8 + 32 * 8 + 64 * 4 + 8 * 4 + 2 * (kThinThreads / 32) * 4;
+constexpr int kThinSlots = kHalf;  // slots of the candidate order = target-row threads of the position kernel
+static_assert(kThinThreads % kThinSlots == 0, "the block sums the slots with a whole number of threads per slot");
+
+static size_t thin_smem_bytes() {
+    return kThinSlots * 8 + 32 * 8 + 64 * 4 + 8 * 4 + 2 * (kThinThreads / 32) * 4 + (kThinThreads / kThinSlots) * kThinSlots * 4;
 }
 
-// 2^(l s - rs) of this lane's share (one 16-byte vector) of tile `tile` of `row`; zero past the end of the row.
+// 2^(l s - rs) of the 16-byte word `word` of `row` (NV logits); zero past the end of the row.
 template <typename T>
-__device__ __forceinline__ void thin_lane_terms(const T *row, int V, int tile, int lane, bool vec_ok, float s, float rs,
+__device__ __forceinline__ void thin_word_terms(const T *row, int V, int word, bool vec_ok, float s, float rs,
                                                 float (&e)[Elem<T>::kPerVec]) {
     constexpr int NV = Elem<T>::kPerVec;
-    const int t0 = (tile * 32 + lane) * NV;
+    const int t0 = word * NV;
     if (vec_ok && t0 + NV <= V) {
         float v[NV];
         Elem<T>::unpack(ld_stream(reinterpret_cast<const uint4 *>(row + t0)), v);
@@ -67,19 +72,20 @@ __device__ __forceinline__ float thin_lane_sum(const float (&e)[NV]) {
 
 template <typename T>
 __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, GroupsDev G) {
-    constexpr int NT = kThinThreads, NW = NT / 32, NV = Elem<T>::kPerVec, TS = 32 * NV;
+    constexpr int NT = kThinThreads, NW = NT / 32, NV = Elem<T>::kPerVec, S = kThinSlots, SUB = NT / S;
     extern __shared__ __align__(16) unsigned char raw[];
     __shared__ int s_n, s_flags;
     __shared__ float4 s_stats;
     const int V = G.V, M = G.M, K = a.K;
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int ntiles = (V + TS - 1) / TS;
-    double *tile_incl = reinterpret_cast<double *>(raw);        // [ntiles] inclusive prefix of the tile sums
-    double *dscratch = tile_incl + ntiles;                      // 32 doubles
+    const int nwords = (V + NV - 1) / NV;                       // 16-byte words of a row (the last may be partial)
+    double *slot_incl = reinterpret_cast<double *>(raw);        // [S] inclusive prefix of the slot masses
+    double *dscratch = slot_incl + S;                           // 32 doubles
     float *scratch = reinterpret_cast<float *>(dscratch + 32);  // 64 floats
     int *ibox = reinterpret_cast<int *>(scratch + 64);          // 8 ints
     int *cand = ibox + 8;                                       // NW ints: group kept by each warp's trial, or -1
     int *cand_tok = cand + NW;                                  // NW ints: the token drawn inside that group
+    float *part = reinterpret_cast<float *>(cand_tok + NW);     // [SUB][S] partial slot sums of the pass below
 
     // the first trial of this warp: its uniforms are inputs of the call, so they can be fetched before the
     // position kernel's results are waited for
@@ -135,8 +141,8 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
     } else {
         // statistics of the bonus row: one pass with a per-thread reference, merged over the block
         RefSum st{kRefInit * a.s, 0.f};
-        for (int tile = warp; tile < ntiles; tile += NW) {
-            const int t0 = (tile * 32 + lane) * NV;
+        for (int word = tid; word < nwords; word += NT) {
+            const int t0 = word * NV;
             if (vec_ok && t0 + NV <= V) {
                 float v[NV];
                 Elem<T>::unpack(ld_stream(reinterpret_cast<const uint4 *>(trow + t0)), v);
@@ -162,62 +168,44 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
         iz_p = 1.0f / Z;
     }
 
-    // ---- 2. tile sums of the target row, then their prefix.  A warp walks a contiguous run of tiles, kInFlight
-    // tiles of loads in flight at a time (deeper or double-buffered variants measured the same) ----
-#ifndef PCG_THIN_INFLIGHT
-#define PCG_THIN_INFLIGHT 4
-#endif
-    constexpr int kInFlight = PCG_THIN_INFLIGHT;
-    const int tiles_per_warp = (ntiles + NW - 1) / NW;
-    const int tile_first = warp * tiles_per_warp, tile_end = min(ntiles, tile_first + tiles_per_warp);
-    auto issue = [&](int base, uint4(&r)[kInFlight], bool(&fast)[kInFlight]) {
-#pragma unroll
-        for (int j = 0; j < kInFlight; ++j) {
-            const int tile = base + j;
-            const int t0 = (tile * 32 + lane) * NV;
-            fast[j] = tile < tile_end && vec_ok && t0 + NV <= V;
-            if (fast[j]) r[j] = ld_stream(reinterpret_cast<const uint4 *>(trow + t0));
+    // ---- 2. the slot masses of the target row (slot of token t = (t div NV) mod S), then their prefix ----
+    float mass = 0.f;  // of slot tid, in threads tid < S
+    if (a.strata && residual) {
+        // the position kernel's thread h summed exactly slot h, relative to a reference of its own that is at most
+        // the row's final one
+        if (tid < S) {
+            const float2 v = a.strata[(size_t)(b * K + n) * S + tid];
+            mass = __fmul_rn(v.y, ex2(v.x - rs_p));
         }
-    };
-    auto consume = [&](int base, const uint4(&r)[kInFlight], const bool(&fast)[kInFlight]) {
+    } else {
+        // SUB threads per slot walk the slot's words, four loads in flight each; partial sums added in fixed order
+        const int h = tid % S, sub = tid / S;
+        float acc = 0.f;
+        for (int w0 = h + S * sub; w0 < nwords; w0 += 4 * S * SUB) {
+            float e[4][NV];
 #pragma unroll
-        for (int j = 0; j < kInFlight; ++j) {
-            const int tile = base + j;
-            if (tile >= tile_end) continue;  // (warp-uniform)
-            float e[NV];
-            if (fast[j]) {
-                float v[NV];
-                Elem<T>::unpack(r[j], v);
+            for (int j = 0; j < 4; ++j) {
+                const int word = w0 + j * S * SUB;
+                if (word < nwords) {
+                    thin_word_terms<T>(trow, V, word, vec_ok, a.s, rs_p, e[j]);
+                } else {
 #pragma unroll
-                for (int i = 0; i < NV; ++i) e[i] = ex2(__fmaf_rn(v[i], a.s, -rs_p));
-            } else {
-                thin_lane_terms<T>(trow, V, tile, lane, false, a.s, rs_p, e);
+                    for (int i = 0; i < NV; ++i) e[j][i] = 0.f;
+                }
             }
-            float sum = thin_lane_sum<NV>(e);
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) tile_incl[tile] = (double)sum;
+            for (int j = 0; j < 4; ++j) acc += thin_lane_sum<NV>(e[j]);
         }
-    };
-    for (int base = tile_first; base < tile_end; base += kInFlight) {
-        uint4 r[kInFlight];
-        bool fast[kInFlight];
-        issue(base, r, fast);
-        consume(base, r, fast);
+        part[sub * S + h] = acc;
+        __syncthreads();
+        if (tid < S)
+            for (int j = 0; j < SUB; ++j) mass += part[j * S + tid];
     }
-    __syncthreads();
     double Ztot;
     {
-        const int per = (ntiles + NT - 1) / NT;
-        const int i0 = min(ntiles, tid * per), i1 = min(ntiles, i0 + per);
-        double my = 0.0, excl, incl;
-        for (int j = i0; j < i1; ++j) my += tile_incl[j];
-        block_scan<NT>(my, dscratch, &excl, &incl, &Ztot);
-        double run = excl;
-        for (int j = i0; j < i1; ++j) {
-            run += tile_incl[j];
-            tile_incl[j] = run;
-        }
+        double excl, incl;
+        block_scan<NT>(tid < S ? (double)mass : 0.0, dscratch, &excl, &incl, &Ztot);
+        if (tid < S) slot_incl[tid] = incl;
     }
     __syncthreads();
 
@@ -232,47 +220,70 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
         if (r < max_trials) {
             const float u_tok = r0 ? tu[3 * r] : u_first[0], u_lab = r0 ? tu[3 * r + 1] : u_first[1];
             const float u_keep = r0 ? tu[3 * r + 2] : u_first[2];
-            // token y ~ target: tile by binary search over the prefix, then a scan inside the tile
+            // token y ~ target: slot by binary search over the prefix, then a scan over the slot's words in token
+            // order, 32 words (each S words apart) at a time with the next 32 already loading
             const double target = (double)u_tok * Ztot;
-            int lo = 0, hi = ntiles - 1;  // the last tile's prefix is the total, which exceeds u * total for u < 1
+            int lo = 0, hi = S - 1;  // the last slot's prefix is the total, which exceeds u * total for u < 1
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
-                if (tile_incl[mid] > target)
+                if (slot_incl[mid] > target)
                     hi = mid;
                 else
                     lo = mid + 1;
             }
-            const int tile = lo;
-            const double tl = target - (tile > 0 ? tile_incl[tile - 1] : 0.0);
-            float e[NV];
-            thin_lane_terms<T>(trow, V, tile, lane, vec_ok, a.s, rs_p, e);
-            const float lsum = thin_lane_sum<NV>(e);
-            double inc = (double)lsum;
+            const int h = lo;
+            const double tl = target - (h > 0 ? slot_incl[h - 1] : 0.0);
+            const int cnt = h < nwords ? (nwords - h + S - 1) / S : 0;  // words of slot h
+            double carry = 0.0;
+            int y = -1, y_last = -1;
+            float e[NV], e_next[NV];
+            if (lane < cnt) thin_word_terms<T>(trow, V, h + S * lane, vec_ok, a.s, rs_p, e);
+            for (int base = 0; base < cnt && y < 0; base += 32) {
+                const int m = base + lane;
+                if (m >= cnt) {
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double up = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc += up;
-            }
-            const unsigned above = __ballot_sync(0xffffffffu, lsum > 0.f && inc > tl);
-            const unsigned massy = __ballot_sync(0xffffffffu, lsum > 0.f);
-            // rounding may leave no lane above the target: then the last lane with mass, and its last element with mass
-            const int L = above ? __ffs(above) - 1 : (massy ? 31 - __clz(massy) : 0);
-            int pick = 0;
-            if (lane == L) {
-                double loc = inc - (double)lsum;
-                int first_above = -1, last = 0;
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    loc += (double)e[i];
-                    if (e[i] > 0.f) {
-                        last = i;
-                        if (first_above < 0 && loc > tl) first_above = i;
-                    }
+                    for (int i = 0; i < NV; ++i) e[i] = 0.f;
                 }
-                pick = first_above >= 0 ? first_above : last;
+                if (m + 32 < cnt) thin_word_terms<T>(trow, V, h + S * (m + 32), vec_ok, a.s, rs_p, e_next);
+                const float lsum = thin_lane_sum<NV>(e);
+                double inc = (double)lsum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const double up = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc += up;
+                }
+                const unsigned above = __ballot_sync(0xffffffffu, lsum > 0.f && carry + inc > tl);
+                const unsigned massy = __ballot_sync(0xffffffffu, lsum > 0.f);
+                // the lane that holds the answer of this chunk (if any), and the last lane with mass for the case
+                // that rounding leaves no prefix above the target
+                const int L = above ? __ffs(above) - 1 : (massy ? 31 - __clz(massy) : -1);
+                if (L >= 0) {
+                    int pick = 0;
+                    if (lane == L) {
+                        double loc = carry + inc - (double)lsum;
+                        int first_above = -1, last = 0;
+#pragma unroll
+                        for (int i = 0; i < NV; ++i) {
+                            loc += (double)e[i];
+                            if (e[i] > 0.f) {
+                                last = i;
+                                if (first_above < 0 && loc > tl) first_above = i;
+                            }
+                        }
+                        pick = first_above >= 0 ? first_above : last;
+                    }
+                    pick = __shfl_sync(0xffffffffu, pick, L);
+                    const int tok = (h + S * (base + L)) * NV + pick;
+                    if (above)
+                        y = tok;
+                    else
+                        y_last = tok;
+                }
+                carry += __shfl_sync(0xffffffffu, inc, 31);
+#pragma unroll
+                for (int i = 0; i < NV; ++i) e[i] = e_next[i];
             }
-            pick = __shfl_sync(0xffffffffu, pick, L);
-            int y = (tile * 32 + L) * NV + pick;
+            if (y < 0) y = y_last >= 0 ? y_last : min(h * NV, V - 1);
             if (y >= V) y = V - 1;
             // label k ~ w_{.,y}
             const int rv0 = G.rev_ptr[y];
