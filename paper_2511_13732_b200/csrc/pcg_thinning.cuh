@@ -214,10 +214,16 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
     const bool usable = Ztot > 0.0 && Ztot < (double)__builtin_huge_valf();
     if (!usable) flags |= PCG_FLAG_NONFINITE;
     const int max_trials = usable ? (residual ? a.n_trials : 1) : 0;
-    for (int r0 = 0; r0 < max_trials && gsel < 0; r0 += NW) {
+#ifndef PCG_THIN_FIRST_ROUND
+#define PCG_THIN_FIRST_ROUND 8
+#endif
+    // trials of the first round (every trial reads its slot's words, scattered over the whole row: fewer side by
+    // side means less traffic, more means fewer sequences need a second round)
+    constexpr int kFirstRound = PCG_THIN_FIRST_ROUND;
+    for (int r0 = 0, width = kFirstRound; r0 < max_trials && gsel < 0; r0 += width, width = NW) {
         const int r = r0 + warp;
         int kept = -1;
-        if (r < max_trials) {
+        if (warp < width && r < max_trials) {
             const float u_tok = r0 ? tu[3 * r] : u_first[0], u_lab = r0 ? tu[3 * r + 1] : u_first[1];
             const float u_keep = r0 ? tu[3 * r + 2] : u_first[2];
             // token y ~ target: slot by binary search over the prefix, then a scan over the slot's words in token
@@ -315,7 +321,7 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
         }
         if (lane == 0) cand[warp] = kept;
         __syncthreads();
-        used = min(r0 + NW, max_trials);
+        used = min(r0 + width, max_trials);
         for (int w = 0; w < NW; ++w)
             if (cand[w] >= 0) {
                 gsel = cand[w];
