@@ -13,7 +13,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpcg.so")
 SOURCES = ["pcg_groups.cu", "pcg_kernels.cu", "pcg_host.cu", "pcg_asg.cu"]
-HEADERS = [os.path.join(CSRC, "pcg_common.cuh"), os.path.join(ROOT, "include", "pcg.h")]
+HEADERS = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))) + [
+    os.path.join(ROOT, "include", "pcg.h")]
 
 
 def nvcc_path() -> str:
