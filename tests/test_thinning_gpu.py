@@ -41,11 +41,17 @@ def assert_thin_parity(got, ref, max_excused=0):
     assert cmp.hard == 0, f"hard mismatches: {cmp.details[:5]}"
     assert cmp.excused <= max_excused, f"excused mismatches: {cmp.details[:5]}"
     excused = {d[0] for d in cmp.details}
+    K = ref.tokens.shape[1] - 1
+    quiet = 0  # same outputs reached over a different number of trials: a keep test on its threshold
     for b in range(len(n)):
         if b in excused:
             continue
-        assert trials[b] == ref.trials[b], (b, trials[b], ref.trials[b])
-        assert flg[b] == ref.flags[b], (b, flg[b], ref.flags[b])
+        if trials[b] != ref.trials[b] or flg[b] != ref.flags[b]:
+            # with few groups a later candidate can land on the same group (and then the same token): only a
+            # decision within the band of its threshold may make the trial counts differ
+            assert ref.margins[b, K, 0] < BAND, (b, trials[b], ref.trials[b], flg[b], ref.flags[b], ref.margins[b, K, 0])
+            quiet += 1
+    assert cmp.excused + quiet <= max_excused, (cmp.excused, quiet)
     return cmp
 
 
