@@ -209,6 +209,11 @@ def _groups_heavy_tail(cfg: Config, dmax: int = 16, smax: int = 200) -> Groups:
         stubs[dup], stubs[partner] = stubs[partner].copy(), stubs[dup].copy()
     else:
         raise RuntimeError("could not resolve duplicate memberships")
+    # overlapping swaps can, at small sizes, take a token's last stub away: every token must be in a group
+    missing = np.setdiff1d(np.arange(cfg.V), stubs)
+    if missing.size:
+        slot_group = np.concatenate([slot_group, missing % cfg.M])
+        stubs = np.concatenate([stubs, missing])
     return _csr_from_pairs(cfg.V, cfg.M, slot_group, stubs)
 
 
