@@ -293,9 +293,12 @@ pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits
  *
  * Everything up to the first rejection is pcg_verify's per-position stage (label, acceptance, first-reject scan).
  * The group at the rejected position is then drawn WITHOUT enumerating the groups.  Trial r = 0, 1, ... draws a
- * token y from the target row by inverse CDF with thin_uniforms[b, r, 0] over the tokens taken slot by slot (the
- * slot of token t is (t div W) mod 128 with W = 16 bytes / bytes per logit, tokens ascending inside a slot: the
- * order in which the library's streaming kernel sums a row, so that the slot masses cost nothing), a label k ~ w_{.,y} over
+ * token y from the target row by inverse CDF with thin_uniforms[b, r, 0] (the paper fixes the law y ~ target; how a
+ * uniform is mapped to y is this interface's rule:
+ *     CANDIDATE ORDER: the inverse CDF walks the tokens in ascending order of the pair ((t div W) mod 128, t),
+ *     where W = 16 / (bytes per logit), i.e. 4 for PCG_F32 and 8 for the 16-bit types;
+ * y is the first token of that order whose inclusive running sum of p exceeds u times the total), a label
+ * k ~ w_{.,y} over
  * the groups containing y with thin_uniforms[b, r, 1] (so k follows the target's coarse distribution), and keeps
  * k if thin_uniforms[b, r, 2] < [1 - Q(k)/P(k)]_+ (draft mass over target mass of group k alone); otherwise the
  * next trial draws a new candidate.  The kept group's law is the normalised residual (P - Q)_+ exactly; the
@@ -306,8 +309,8 @@ pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits
  * are turned down, draws the group from the enumerated residual with uniforms[b, K, 0] (what pcg_verify does;
  * same law) and sets PCG_FLAG_THINNING_EXHAUSTED for that sequence.  That fallback is slow -- one thread block
  * walks all nnz memberships of the sequence, 0.47 ms at V = 65536, M = 16384, nnz = 393216 on a B200, more than
- * the rest of a 256-sequence call -- whereas trials are cheap: they run 16 at a time, and a further round (about
- * 4 microseconds) is entered only by sequences whose earlier candidates were all turned down.  So supply trials
+ * the rest of a 256-sequence call -- whereas trials are cheap: they run side by side (8 in the first round, 16 in
+ * each later one), and a further round (about 4 microseconds) is entered only by sequences whose earlier candidates were all turned down.  So supply trials
  * generously: a rejected sequence runs out of n_trials with probability (1 - TV(P,Q))^n_trials.  Results are a deterministic function of
  * the inputs; they equal pcg_verify's in distribution, not draw by draw (the two consume different uniforms).
  *

@@ -23,7 +23,11 @@
  * facts that do not come from this file (a library softmax, dense-matrix brute
  * force in exact rationals, the exactness proposition checked by enumeration,
  * a separately written token-level speculative-sampling verifier).  The
- * thinning sampler of pcg_oracle_verify_thinning is pinned by the laws the
+ * general-weights branches (coarse-graining, label draw, within-group draw)
+ * and the constant acceptance bias are pinned with unequal hand-made weights
+ * the same way (exact rationals, hand-written labels, the coupling identity,
+ * min(Q, P + bias Q) on a grid of uniforms).  The thinning sampler of
+ * pcg_oracle_verify_thinning is pinned by the laws the
  * paper states for it, measured over many seeded uniforms (kept group ~
  * normalised residual, emitted group ~ target coarse distribution, mean
  * number of trials = 1/TV, token ~ target-conditional), by its singleton-group
@@ -47,11 +51,6 @@
 
 /* flag bits written per sequence */
 #define ORACLE_FLAG_ZERO_RESIDUAL 2 /* reject taken but sum of (P-Q)_+ was <= 0 */
-/* Candidate-token order of the thinning sampler (the paper fixes the law y ~ target, not how a uniform is mapped
- * to y).  Reading of this library: the inverse CDF runs over the tokens taken slot by slot, where the slot of
- * token t is (t div W) mod 128 and W is the number of logits in 16 bytes (4 for float, 8 for the 16-bit types);
- * inside a slot tokens ascend. */
-#define ORACLE_CANDIDATE_SLOTS 128
 #define ORACLE_FLAG_THINNING_EXHAUSTED 8 /* every supplied thinning trial was turned down; enumerated draw used */
 
 /* IEEE binary16 bit pattern to double, from the format's definition: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
@@ -221,7 +220,9 @@ static int32_t draw_label(int32_t x, double u, const double *weights, const int3
  * Terminal group, two ways.  thin == NULL: enumerate the residual over all groups and invert its CDF with
  * uniforms[K][0].  thin != NULL ([B, n_trials, 3]): the thinning sampler of the paper
  * (Sec. 2.2), which never enumerates the groups.  Trial r uses thin[r][0] to draw a token y from the target
- * row by inverse CDF over the tokens in candidate order (cand_order, see ORACLE_CANDIDATE_SLOTS), thin[r][1] to draw y's label k ~ w_{.,y} (so that k ~ the target's coarse
+ * row by inverse CDF over the tokens taken in the order cand_order[0], cand_order[1], ... (a permutation of the tokens
+ * supplied by the caller, NULL = ascending token id: the paper fixes the law y ~ target, which no order can change,
+ * not how a uniform is mapped to y), thin[r][1] to draw y's label k ~ w_{.,y} (so that k ~ the target's coarse
  * distribution), and keeps k if thin[r][2] < [1 - draft mass(k) / target mass(k)]_+; otherwise the next trial
  * draws a new (y, k).  After all accepted positions (no rejection) there is no draft mass: the first candidate
  * is kept, which draws the bonus group from the target's coarse distribution.  The paper's sampler is not
@@ -284,10 +285,11 @@ static void verify_sequence(const void *target_logits, const void *draft_logits,
     if (thin) {
         const float *tu = thin + b * (int64_t)n_trials * 3;
         int used = 0;
-        for (int t = 0; t < V; ++t) pm[t] = p[cand_order[t]]; /* target masses in candidate order */
+        for (int t = 0; t < V; ++t) pm[t] = p[cand_order ? cand_order[t] : t]; /* target masses in candidate order */
         for (int r = 0; r < n_trials && gs < 0; ++r) {
             double m_tok = INFINITY, m_lab = INFINITY, m_keep = INFINITY;
-            int y = cand_order[inverse_cdf(pm, V, (double)tu[3 * r], NULL, &m_tok)]; /* y ~ target */
+            int y = inverse_cdf(pm, V, (double)tu[3 * r], NULL, &m_tok); /* y ~ target */
+            if (cand_order) y = cand_order[y];
             int32_t k = draw_label(y, (double)tu[3 * r + 1], weights, rev_ptr, rev_grp, rev_nz, &m_lab); /* k ~ w_{.,y} */
             int keep = 1;
             if (have_Q) { /* thinning probability a(k) = [1 - draft mass / target mass]_+ */
@@ -351,8 +353,9 @@ static void verify_sequence(const void *target_logits, const void *draft_logits,
 static int verify_batch(const void *target_logits, const void *draft_logits, int dtype, int B, int K, int V,
                         const int32_t *draft_tokens, int M, const int32_t *group_ptr, const int32_t *group_tok,
                         const int32_t *tok_degree, const double *weights, const float *uniforms, const float *thin,
-                        int n_trials, float temperature, double accept_bias, int32_t *accept_len, int32_t *tokens,
-                        int32_t *groups, int32_t *flags, int32_t *trials, double *margins, int threads) {
+                        int n_trials, const int32_t *cand_order, float temperature, double accept_bias,
+                        int32_t *accept_len, int32_t *tokens, int32_t *groups, int32_t *flags, int32_t *trials,
+                        double *margins, int threads) {
     if (!target_logits || !draft_logits || !draft_tokens || !group_ptr || !group_tok || !tok_degree || !uniforms ||
         !accept_len || !tokens || !groups)
         return 1;
@@ -381,16 +384,20 @@ static int verify_batch(const void *target_logits, const void *draft_logits, int
         }
     for (int64_t k = 0; k < (int64_t)B * K; ++k)
         if (draft_tokens[k] < 0 || draft_tokens[k] >= V) return 4;
-    /* candidate order of the thinning sampler: slot-major, ascending inside a slot */
-    int32_t *cand_order = NULL;
-    if (thin) {
-        cand_order = (int32_t *)malloc(sizeof(int32_t) * (size_t)V);
-        if (!cand_order) return 2;
-        const int W = dtype == ORACLE_F32 ? 4 : 8;
-        int n = 0;
-        for (int slot = 0; slot < ORACLE_CANDIDATE_SLOTS; ++slot)
-            for (int t = 0; t < V; ++t)
-                if ((t / W) % ORACLE_CANDIDATE_SLOTS == slot) cand_order[n++] = t;
+    /* the candidate order of the thinning sampler must be a permutation of the tokens */
+    if (thin && cand_order) {
+        int bad = 0;
+        for (int t = 0; t < V; ++t) fill[t] = 0;
+        for (int t = 0; t < V; ++t) {
+            if (cand_order[t] < 0 || cand_order[t] >= V || fill[cand_order[t]]++) bad = 1;
+        }
+        if (bad) {
+            free(rev_ptr);
+            free(rev_grp);
+            free(rev_nz);
+            free(fill);
+            return 5;
+        }
     }
     int nthreads = threads;
 #ifdef _OPENMP
@@ -429,7 +436,6 @@ static int verify_batch(const void *target_logits, const void *draft_logits, int
     free(rev_grp);
     free(rev_nz);
     free(fill);
-    free(cand_order);
     return failed ? 2 : 0;
 }
 
@@ -439,26 +445,28 @@ int pcg_oracle_verify(const void *target_logits, const void *draft_logits, int d
                       double accept_bias, int32_t *accept_len, int32_t *tokens, int32_t *groups, int32_t *flags,
                       double *margins, int threads) {
     return verify_batch(target_logits, draft_logits, dtype, B, K, V, draft_tokens, M, group_ptr, group_tok,
-                        tok_degree, weights, uniforms, NULL, 0, temperature, accept_bias, accept_len, tokens, groups,
+                        tok_degree, weights, uniforms, NULL, 0, NULL, temperature, accept_bias, accept_len, tokens, groups,
                         flags, NULL, margins, threads);
 }
 
 /*
  * Batched verification with the thinning sampler for the terminal group (see verify_sequence).
- * thin_uniforms [B, n_trials, 3] floats in [0,1), n_trials >= 1; trials [B] (may be NULL) receives the number
- * of candidates drawn (1 after an all-accepted sequence).  margins[b][K][0] is the smallest margin over every
+ * thin_uniforms [B, n_trials, 3] floats in [0,1), n_trials >= 1; cand_order [V]: the order in which the
+ * candidate draw walks the tokens, a permutation of 0..V-1, or NULL for ascending token id; trials [B] (may be
+ * NULL) receives the number of candidates drawn (1 after an all-accepted sequence).  margins[b][K][0] is the smallest margin over every
  * decision that led to the terminal group.  Everything else as pcg_oracle_verify.
  */
 int pcg_oracle_verify_thinning(const void *target_logits, const void *draft_logits, int dtype, int B, int K, int V,
                                const int32_t *draft_tokens, int M, const int32_t *group_ptr,
                                const int32_t *group_tok, const int32_t *tok_degree, const double *weights,
-                               const float *uniforms, const float *thin_uniforms, int n_trials, float temperature,
-                               double accept_bias, int32_t *accept_len, int32_t *tokens, int32_t *groups,
-                               int32_t *flags, int32_t *trials, double *margins, int threads) {
+                               const float *uniforms, const float *thin_uniforms, int n_trials,
+                               const int32_t *cand_order, float temperature, double accept_bias,
+                               int32_t *accept_len, int32_t *tokens, int32_t *groups, int32_t *flags,
+                               int32_t *trials, double *margins, int threads) {
     if (!thin_uniforms || n_trials < 1) return 1;
     return verify_batch(target_logits, draft_logits, dtype, B, K, V, draft_tokens, M, group_ptr, group_tok,
-                        tok_degree, weights, uniforms, thin_uniforms, n_trials, temperature, accept_bias, accept_len,
-                        tokens, groups, flags, trials, margins, threads);
+                        tok_degree, weights, uniforms, thin_uniforms, n_trials, cand_order, temperature, accept_bias,
+                        accept_len, tokens, groups, flags, trials, margins, threads);
 }
 
 /* Number of threads pcg_oracle_verify uses for threads <= 0. */

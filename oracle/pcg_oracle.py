@@ -48,7 +48,7 @@ def _load():
                                           c_f, c_d, c_vp, c_vp, c_vp, c_vp, c_vp, c_i]
         lib.pcg_oracle_verify.restype = c_i
         lib.pcg_oracle_verify_thinning.argtypes = [c_vp, c_vp, c_i, c_i, c_i, c_i, c_vp, c_i, c_vp, c_vp, c_vp, c_vp,
-                                                   c_vp, c_vp, c_i, c_f, c_d, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_i]
+                                                   c_vp, c_vp, c_i, c_vp, c_f, c_d, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_i]
         lib.pcg_oracle_verify_thinning.restype = c_i
         lib.pcg_oracle_max_threads.argtypes = []
         lib.pcg_oracle_max_threads.restype = c_i
@@ -117,11 +117,12 @@ class OracleResult:
 
 def verify(target_logits, draft_logits, draft_tokens, group_ptr, group_tok, tok_degree, uniforms,
            temperature: float = 1.0, weights=None, accept_bias: float = 0.0, threads: int = 1,
-           thin_uniforms=None) -> OracleResult:
+           thin_uniforms=None, cand_order=None) -> OracleResult:
     """Run Algorithm 1's verification for a batch; see pcg_oracle.c for the layouts.
 
     With ``thin_uniforms`` ([B, n_trials, 3]) the terminal group comes from the thinning sampler of Sec. 2.2
-    instead of the enumerated inverse CDF, and ``trials`` is filled in.
+    instead of the enumerated inverse CDF, and ``trials`` is filled in.  ``cand_order`` ([V], a permutation of the
+    token ids; None = ascending token id) is the order in which the sampler's candidate draw walks the tokens.
     """
     tl, dt = _logits(target_logits)
     dl, dt2 = _logits(draft_logits)
@@ -150,8 +151,11 @@ def verify(target_logits, draft_logits, draft_tokens, group_ptr, group_tok, tok_
         if tu.ndim != 3 or tu.shape[0] != B or tu.shape[1] < 1 or tu.shape[2] != 3:
             raise ValueError("thin_uniforms must be [B, n_trials >= 1, 3]")
         res.trials = np.zeros(B, np.int32)
+        order = None if cand_order is None else _i32(cand_order)
+        if order is not None and order.shape != (V,):
+            raise ValueError("cand_order must be [V]")
         rc = _load().pcg_oracle_verify_thinning(_ptr(tl), _ptr(dl), dt, B, K, V, _ptr(x), M, _ptr(gp), _ptr(gt), _ptr(dg),
-                                                _ptr(w), _ptr(u), _ptr(tu), tu.shape[1], temperature, accept_bias,
+                                                _ptr(w), _ptr(u), _ptr(tu), tu.shape[1], _ptr(order), temperature, accept_bias,
                                                 _ptr(res.accept_len), _ptr(res.tokens), _ptr(res.groups),
                                                 _ptr(res.flags), _ptr(res.trials), _ptr(res.margins), threads)
         if rc:

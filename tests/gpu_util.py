@@ -30,3 +30,12 @@ def run_oracle(oracle, batch, groups, weights=None):
     return oracle.verify(batch.target_logits, batch.draft_logits, batch.draft_tokens, groups.group_ptr,
                          groups.group_tok, groups.tok_degree, batch.uniforms, batch.temperature, weights=weights,
                          threads=0)
+
+
+def library_candidate_order(V: int, logits: np.ndarray) -> np.ndarray:
+    """The order in which pcg_verify_thinning's candidate draw walks the tokens, built here from the rule its
+    header states: ascending ((t div W) mod 128, t) with W = 16 bytes / bytes per logit.  The oracle takes the
+    order as an input; nothing of it is built into the oracle."""
+    W = 16 // logits.dtype.itemsize
+    t = np.arange(V)
+    return np.lexsort((t, (t // W) % 128)).astype(np.int32)

@@ -49,7 +49,7 @@ def test_captured_thinning_call_replays_on_new_inputs(oracle):
     from oracle.compare import compare_verify
     from paper_2511_13732_b200 import binding
 
-    from gpu_util import logits_to_device, make_handle
+    from gpu_util import library_candidate_order, logits_to_device, make_handle
 
     cfg = W.scaled(W.CONFIGS["C3"], B=40, K=4, V=4096, M=1000)
     groups = W.make_groups(cfg)
@@ -82,7 +82,7 @@ def test_captured_thinning_call_replays_on_new_inputs(oracle):
         torch.cuda.synchronize()
         ref = oracle.verify(batch.target_logits, batch.draft_logits, batch.draft_tokens, groups.group_ptr,
                             groups.group_tok, groups.tok_degree, batch.uniforms, batch.temperature, threads=0,
-                            thin_uniforms=thin)
+                            thin_uniforms=thin, cand_order=library_candidate_order(groups.V, batch.target_logits))
         cmp = compare_verify(out[0].cpu().numpy(), out[1].cpu().numpy(), out[2].cpu().numpy(), ref)
         assert cmp.hard == 0 and cmp.excused == 0, cmp.details[:3]
         assert np.array_equal(out[4].cpu().numpy(), ref.trials)

@@ -11,6 +11,7 @@ import pytest
 
 import test_oracle_pins as pins
 import test_thinning_oracle_pins as thin_pins
+import test_weighted_oracle_pins as w_pins
 
 ORACLE_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle")
 
@@ -56,9 +57,10 @@ PIN_CALLS = (
 THIN_MUTATIONS = [
     ("thinning_ratio_inverted", "double a = P[k] > 0.0 ? 1.0 - Q[k] / P[k] : 0.0;",
      "double a = Q[k] > 0.0 ? 1.0 - P[k] / Q[k] : 0.0;", 0),
-    ("thinning_candidate_from_draft", "pm[t] = p[cand_order[t]];", "pm[t] = (have_Q ? q : p)[cand_order[t]];", 0),
-    ("thinning_candidate_order_is_plain_token_order", "if ((t / W) % ORACLE_CANDIDATE_SLOTS == slot) cand_order[n++] = t;",
-     "if (slot == 0) cand_order[n++] = t;", 0),
+    ("thinning_candidate_from_draft", "pm[t] = p[cand_order ? cand_order[t] : t];",
+     "pm[t] = (have_Q ? q : p)[cand_order ? cand_order[t] : t];", 0),
+    ("thinning_candidate_not_mapped_back_through_the_order", "if (cand_order) y = cand_order[y];", "", 0),
+    ("thinning_masses_not_taken_in_the_given_order", "pm[t] = p[cand_order ? cand_order[t] : t];", "pm[t] = p[t];", 0),
     ("thinning_keep_uses_label_uniform", "keep = (double)tu[3 * r + 2] < a;", "keep = (double)tu[3 * r + 1] < a;", 0),
     ("thinning_label_uses_token_uniform", "draw_label(y, (double)tu[3 * r + 1], weights,", "draw_label(y, (double)tu[3 * r], weights,", 0),
     ("thinning_bonus_is_thinned_too", "if (have_Q) { /* thinning probability", "if (1) { /* thinning probability", 0),
@@ -68,12 +70,38 @@ THIN_MUTATIONS = [
 ]
 
 THIN_PIN_CALLS = (
-    [lambda o, s=s: thin_pins.test_thinning_group_law_trials_and_token_law(o, s) for s in (11, 13)]
-    + [lambda o, s=s: thin_pins.test_thinning_bonus_is_one_candidate_from_the_target(o, s) for s in (11,)]
-    + [lambda o: thin_pins.test_thinning_with_singleton_groups_is_token_level_residual_sampling(o),
+    [lambda o, s=s, r=r: thin_pins.test_thinning_group_law_trials_and_token_law(o, s, r) for s, r in ((11, None), (13, 102))]
+    + [lambda o, s=s: thin_pins.test_thinning_bonus_is_one_candidate_from_the_target(o, s, None) for s in (11,)]
+    + [lambda o: thin_pins.test_thinning_with_singleton_groups_is_token_level_residual_sampling(o, None),
        lambda o: thin_pins.test_thinning_exhaustion_falls_back_to_the_enumerated_draw(o),
        lambda o: thin_pins.test_thinning_never_reads_trials_it_does_not_reach(o),
-       lambda o: thin_pins.test_thinning_candidate_order_is_slot_major(o, thin_pins.np.float32, 4)]
+       lambda o: thin_pins.test_thinning_candidate_walks_the_tokens_in_the_given_order(o)]
+)
+
+
+# planted mistakes in the general-weights branches and the acceptance bias, checked against the weighted pins
+WEIGHT_MUTATIONS = [
+    ("label_weights_read_without_the_pair_index", "wx[e] = weights[rev_nz[rev_ptr[x] + e]];", "wx[e] = weights[rev_ptr[x] + e];", 0),
+    ("label_draw_ignores_weights", "    if (!weights) {\n        double uj = u * (double)N;", "    if (1) {\n        double uj = u * (double)N;", 0),
+    ("within_group_weights_not_offset_by_the_group", "w[k] = weights ? p[t] * weights[lo + k]", "w[k] = weights ? p[t] * weights[k]", 0),
+    ("within_group_draw_ignores_weights", "w[k] = weights ? p[t] * weights[lo + k] : p[t] / (double)tok_degree[t];",
+     "w[k] = p[t] / (double)tok_degree[t];", 0),
+    ("coarse_graining_weights_not_offset_by_the_group", "s += weights ? p[t] * weights[k]", "s += weights ? p[t] * weights[k - group_ptr[g]]", 0),
+    ("coarse_graining_ignores_weights", "s += weights ? p[t] * weights[k] : p[t] / (double)tok_degree[t];",
+     "s += p[t] / (double)tok_degree[t];", 0),
+    ("bias_multiplies_the_ratio", "((double)u[2 * i + 1] < ratio + accept_bias)", "((double)u[2 * i + 1] < ratio * (1.0 + accept_bias))", 0),
+    ("bias_subtracted", "((double)u[2 * i + 1] < ratio + accept_bias)", "((double)u[2 * i + 1] < ratio - accept_bias)", 0),
+    ("bias_ignored", "((double)u[2 * i + 1] < ratio + accept_bias)", "((double)u[2 * i + 1] < ratio)", 0),
+    ("bias_added_to_the_target_mass", "double ratio = Q[g] > 0.0 ? P[g] / Q[g] : INFINITY;",
+     "double ratio = Q[g] > 0.0 ? (P[g] + accept_bias) / Q[g] - accept_bias : INFINITY;", 0),
+]
+
+WEIGHT_PIN_CALLS = (
+    [lambda o: w_pins.test_weighted_group_probs_exact_rationals(o), lambda o: w_pins.test_weighted_label_draw_hand_cases(o),
+     lambda o: w_pins.test_weighted_label_law_and_acceptance_law(o),
+     lambda o: w_pins.test_weighted_emitted_group_is_target_coarse(o),
+     lambda o: w_pins.test_weighted_within_group_and_bonus_token_law(o)]
+    + [lambda o, b=b: w_pins.test_acceptance_bias_law(o, b) for b in (0.3, 0.05)]
 )
 
 
@@ -116,8 +144,20 @@ def test_every_planted_thinning_mistake_is_caught_by_a_pin(tmp_path, name, old, 
     assert caught, f"no pin noticed the planted mistake '{name}'"
 
 
+@pytest.mark.parametrize("name,old,new,occurrence", WEIGHT_MUTATIONS, ids=[m[0] for m in WEIGHT_MUTATIONS])
+def test_every_planted_weights_or_bias_mistake_is_caught_by_a_pin(tmp_path, name, old, new, occurrence):
+    mutant = _mutant(tmp_path, name, old, new, occurrence)
+    caught = []
+    for i, call in enumerate(WEIGHT_PIN_CALLS):
+        try:
+            call(mutant)
+        except AssertionError:
+            caught.append(i)
+    assert caught, f"no pin noticed the planted mistake '{name}'"
+
+
 def test_the_unmodified_copy_passes_every_pin(tmp_path):
     """Control: the same machinery with no mistake planted must pass, so a failure above means the mistake."""
     clean = _mutant(tmp_path, "clean", "double ratio", "double ratio", 0)
-    for call in PIN_CALLS + THIN_PIN_CALLS:
+    for call in PIN_CALLS + THIN_PIN_CALLS + WEIGHT_PIN_CALLS:
         call(clean)

@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 from oracle.compare import compare_verify  # noqa: E402
 
-from gpu_util import logits_to_device, make_handle  # noqa: E402
+from gpu_util import library_candidate_order, logits_to_device, make_handle  # noqa: E402
 
 BAND = 1e-6
 EXHAUSTED = 8
@@ -32,7 +32,8 @@ def run_thin(batch, handle, tu, **kw):
 def oracle_thin(oracle, batch, groups, tu, weights=None):
     return oracle.verify(batch.target_logits, batch.draft_logits, batch.draft_tokens, groups.group_ptr,
                          groups.group_tok, groups.tok_degree, batch.uniforms, batch.temperature, weights=weights,
-                         threads=0, thin_uniforms=tu)
+                         threads=0, thin_uniforms=tu,
+                         cand_order=library_candidate_order(groups.V, batch.target_logits))
 
 
 def assert_thin_parity(got, ref, max_excused=0):

@@ -10,9 +10,10 @@ output over many seeded random uniforms (tolerances are five standard deviations
   * singleton groups give token-level residual sampling (p - q)_+;
   * when every supplied trial is turned down the result is the enumerated draw (pinned on its own elsewhere);
   * uniforms of trials that are never reached do not matter;
-  * the mapping from the token uniform to the candidate is the documented one: inverse CDF over the tokens taken
-    slot by slot (slot = (t div W) mod 128, W logits per 16 bytes), checked on a uniform target where the candidate
-    is simply the floor(u V)-th token of that order.
+  * the order in which the candidate draw walks the tokens is an INPUT (a permutation; None = ascending token id).
+    The paper fixes the law y ~ target, which no order can change: the law pins run under the identity and under
+    seeded random permutations; that the given order is really the one walked is checked against literal expected
+    tokens on hand-made targets.
 """
 import numpy as np
 import pytest
@@ -28,20 +29,28 @@ def _uniforms(rng, shape):
     return (rng.integers(0, 1 << 24, size=shape) * 2.0 ** -24).astype(np.float32)
 
 
-def _run(oracle, groups, tl, dl, x, u, tu):
+# candidate orders the law pins run under: ascending token id, and two seeded random permutations
+ORDERS = [None, 101, 102]
+
+
+def _order(which, V):
+    return None if which is None else np.random.default_rng(which).permutation(V).astype(np.int32)
+
+
+def _run(oracle, groups, tl, dl, x, u, tu, order=None):
     B = x.shape[0]
     V = tl.shape[-1]
     return oracle.verify(np.broadcast_to(tl, (B,) + tl.shape[-2:]).copy(), np.broadcast_to(dl, (B,) + dl.shape[-2:]).copy(),
                          x.astype(np.int32).reshape(B, -1), groups.group_ptr, groups.group_tok, groups.tok_degree, u,
-                         thin_uniforms=tu, threads=0)
+                         thin_uniforms=tu, threads=0, cand_order=_order(order, V))
 
 
 def _five_sigma(prob, n):
     return 5.0 * np.sqrt(np.maximum(prob * (1.0 - prob), 1e-4) / n) + 1e-9
 
 
-@pytest.mark.parametrize("seed", [11, 13])
-def test_thinning_group_law_trials_and_token_law(oracle, seed):
+@pytest.mark.parametrize("seed,order", [(11, None), (13, None), (11, 101), (13, 102)])
+def test_thinning_group_law_trials_and_token_law(oracle, seed, order):
     groups, tl, dl, p, q, Wm = _tiny_problem(seed)
     P, Q = Wm @ p[0], Wm @ q
     resid = np.maximum(P - Q, 0.0)
@@ -51,7 +60,7 @@ def test_thinning_group_law_trials_and_token_law(oracle, seed):
     x = rng.choice(6, size=N, p=q)
     u = _uniforms(rng, (N, 2, 2))
     tu = _uniforms(rng, (N, NTR, 3))
-    res = _run(oracle, groups, tl, dl, x, u, tu)
+    res = _run(oracle, groups, tl, dl, x, u, tu, order)
     rej = res.accept_len == 0
     nrej = int(rej.sum())
     assert nrej > 0.5 * TV * N  # Pr(reject) = TV(P, Q)
@@ -80,8 +89,8 @@ def test_thinning_group_law_trials_and_token_law(oracle, seed):
         assert np.all(cond[Wm[g] == 0] == 0)
 
 
-@pytest.mark.parametrize("seed", [11, 14])
-def test_thinning_bonus_is_one_candidate_from_the_target(oracle, seed):
+@pytest.mark.parametrize("seed,order", [(11, None), (14, None), (14, 101)])
+def test_thinning_bonus_is_one_candidate_from_the_target(oracle, seed, order):
     groups, tl, dl, p, q, Wm = _tiny_problem(seed)
     rng = np.random.default_rng(2000 + seed)
     N = 200_000
@@ -89,7 +98,7 @@ def test_thinning_bonus_is_one_candidate_from_the_target(oracle, seed):
     u = _uniforms(rng, (N, 2, 2))
     u[:, 0, 1] = 0.0  # accept uniform 0: the drafted position is always accepted
     tu = _uniforms(rng, (N, 3, 3))
-    res = _run(oracle, groups, tl, dl, x, u, tu)
+    res = _run(oracle, groups, tl, dl, x, u, tu, order)
     assert np.all(res.accept_len == 1) and np.all(res.trials == 1) and np.all(res.flags == 0)
     grp = np.bincount(res.groups[:, 1], minlength=groups.M) / N
     np.testing.assert_allclose(grp, Wm @ p[1], atol=_five_sigma(Wm @ p[1], N).max())
@@ -98,11 +107,12 @@ def test_thinning_bonus_is_one_candidate_from_the_target(oracle, seed):
     # the bonus candidate never looks at its third uniform
     tu2 = tu.copy()
     tu2[:, 0, 2] = 1.0 - 2.0 ** -24
-    res2 = _run(oracle, groups, tl, dl, x, u, tu2)
+    res2 = _run(oracle, groups, tl, dl, x, u, tu2, order)
     assert np.array_equal(res2.tokens, res.tokens) and np.array_equal(res2.groups, res.groups)
 
 
-def test_thinning_with_singleton_groups_is_token_level_residual_sampling(oracle):
+@pytest.mark.parametrize("order", ORDERS[:2])
+def test_thinning_with_singleton_groups_is_token_level_residual_sampling(oracle, order):
     rng = np.random.default_rng(31)
     V = 7
     tl = (1.5 * rng.standard_normal((2, V))).astype(np.float32)
@@ -112,7 +122,7 @@ def test_thinning_with_singleton_groups_is_token_level_residual_sampling(oracle)
     g = W.groups_from_lists(V, [[t] for t in range(V)])
     N = 200_000
     x = rng.choice(V, size=N, p=q)
-    res = _run(oracle, g, tl, dl, x, _uniforms(rng, (N, 2, 2)), _uniforms(rng, (N, 64, 3)))
+    res = _run(oracle, g, tl, dl, x, _uniforms(rng, (N, 2, 2)), _uniforms(rng, (N, 64, 3)), order)
     rej = res.accept_len == 0
     resid = np.maximum(p - q, 0.0)
     hist = np.bincount(res.tokens[rej, 0], minlength=V) / rej.sum()
@@ -163,22 +173,43 @@ def test_thinning_never_reads_trials_it_does_not_reach(oracle):
     assert not np.array_equal(res3.groups, res.groups)
 
 
-@pytest.mark.parametrize("dtype,W_", [(np.float32, 4), (np.float16, 8)])
-def test_thinning_candidate_order_is_slot_major(oracle, dtype, W_):
-    """Uniform target, singleton groups, draft == target (every position accepted): the bonus token is the first
-    candidate itself, which must be the floor(u V)-th token in slot-major order."""
-    V = 2600  # more than 128 * W tokens, not a multiple of it
-    order = sorted(range(V), key=lambda t: ((t // W_) % 128, t))
-    assert order[:3] == [0, 1, 2] and order[W_] == 128 * W_  # after the first 16-byte word comes the word 128 further on
+def _first_candidates(oracle, p_target, order, us):
+    """Bonus tokens of all-accepted one-position sequences over singleton groups: the first candidate itself."""
+    V = len(p_target)
     g = W.groups_from_lists(V, [[t] for t in range(V)])
-    idx = np.array([0, 1, W_, W_ + 1, 777, 1300, V - 2, V - 1])
-    N = idx.size
-    tl = np.zeros((N, 2, V), dtype)
-    dl = np.zeros((N, 1, V), dtype)
+    N = len(us)
+    row = np.log(np.asarray(p_target, np.float64)).astype(np.float32)
+    tl = np.broadcast_to(row, (N, 2, V)).copy()
+    dl = tl[:, :1].copy()  # draft == target: every position is accepted
     u = np.zeros((N, 2, 2), np.float32)
     u[:, 1, 1] = 0.5
     tu = np.zeros((N, 2, 3), np.float32)
-    tu[:, 0, 0] = ((idx + 0.5) / V).astype(np.float32)
-    res = oracle.verify(tl, dl, np.zeros((N, 1), np.int32), g.group_ptr, g.group_tok, g.tok_degree, u, thin_uniforms=tu)
+    tu[:, 0, 0] = np.asarray(us, np.float32)
+    res = oracle.verify(tl, dl, np.zeros((N, 1), np.int32), g.group_ptr, g.group_tok, g.tok_degree, u, thin_uniforms=tu,
+                        cand_order=order)
     assert np.all(res.accept_len == 1) and np.all(res.trials == 1)
-    assert res.tokens[:, 1].tolist() == [order[i] for i in idx]
+    return res.tokens[:, 1].tolist()
+
+
+def test_thinning_candidate_walks_the_tokens_in_the_given_order(oracle):
+    """Expected tokens written out by hand.  Target p = (0.1, 0.2, 0.3, 0.4) over tokens 0..3.
+    Order (2, 0, 3, 1): running sums 0.3 (token 2), 0.4 (token 0), 0.8 (token 3), 1.0 (token 1).
+    Ascending order: running sums 0.1, 0.3, 0.6, 1.0."""
+    p = [0.1, 0.2, 0.3, 0.4]
+    us = [0.05, 0.29, 0.31, 0.39, 0.41, 0.79, 0.81, 0.99]
+    assert _first_candidates(oracle, p, np.array([2, 0, 3, 1], np.int32), us) == [2, 2, 0, 0, 3, 3, 1, 1]
+    assert _first_candidates(oracle, p, None, us) == [0, 1, 2, 2, 2, 3, 3, 3]
+    assert _first_candidates(oracle, p, np.arange(4, dtype=np.int32), us) == [0, 1, 2, 2, 2, 3, 3, 3]
+    # uniform target over eight tokens: the candidate is the floor(8 u)-th token of the order
+    order = np.array([5, 2, 7, 0, 3, 6, 1, 4], np.int32)
+    us8 = [(i + 0.5) / 8 for i in range(8)]
+    assert _first_candidates(oracle, [0.125] * 8, order, us8) == [5, 2, 7, 0, 3, 6, 1, 4]
+    assert _first_candidates(oracle, [0.125] * 8, None, us8) == [0, 1, 2, 3, 4, 5, 6, 7]
+
+
+def test_thinning_rejects_an_order_that_is_no_permutation(oracle):
+    for bad in ([0, 1, 1, 3], [0, 1, 2, 4], [-1, 0, 1, 2]):
+        with pytest.raises(ValueError):
+            _first_candidates(oracle, [0.25] * 4, np.array(bad, np.int32), [0.5])
+    with pytest.raises(ValueError):
+        _first_candidates(oracle, [0.25] * 4, np.arange(3, dtype=np.int32), [0.5])
