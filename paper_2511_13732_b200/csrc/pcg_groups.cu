@@ -116,13 +116,17 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
         set_error("group_ptr[0] must be 0 and group_ptr[M] must equal nnz");
         return PCG_ERR_INVALID_GROUPS;
     }
+    // the whole pointer array first: 0 <= group_ptr[g] <= group_ptr[g+1] <= nnz, so that no token list read below
+    // can leave the copy of group_tok
+    for (int g = 0; g < M; ++g) {
+        if (gptr[g] < 0 || gptr[g + 1] < gptr[g] || (int64_t)gptr[g + 1] > nnz) {
+            set_error("group_ptr decreases or leaves [0, nnz] at group %d", g);
+            return PCG_ERR_INVALID_GROUPS;
+        }
+    }
     std::vector<int32_t> count((size_t)V, 0);
     int max_group = 0;
     for (int g = 0; g < M; ++g) {
-        if (gptr[g + 1] < gptr[g]) {
-            set_error("group_ptr decreases at group %d", g);
-            return PCG_ERR_INVALID_GROUPS;
-        }
         for (int32_t k = gptr[g]; k < gptr[g + 1]; ++k) {
             int32_t t = gtok[k];
             if (t < 0 || t >= V) {

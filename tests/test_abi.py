@@ -59,6 +59,9 @@ def test_membership_validation_on_the_host():
         ([0, 2, 5, 6, 6], [0, 1, 1, 2, 3, 4], [1, 1, 1, 1, 1], "tok_degree"),  # wrong degree
         ([0, 2, 4, 5, 5], [0, 1, 1, 2, 4], [1, 2, 1, 0, 1], "tok_degree"),  # token 3 in no group
         ([0, 2, 1, 5, 5], [0, 1, 2, 3, 4], [1, 1, 1, 1, 1], "decreases"),  # pointer not monotone
+        ([0, 9, 1, 5, 5], [0, 1, 2, 3, 4], [1, 1, 1, 1, 1], "decreases"),  # pointer beyond nnz before it decreases
+        ([0, 1000, 3, 5, 5], [0, 1, 2, 3, 4], [1, 1, 1, 1, 1], "decreases"),
+        ([0, -2, 3, 5, 5], [0, 1, 2, 3, 4], [1, 1, 1, 1, 1], "decreases"),  # negative pointer
         ([1, 2, 5, 6, 6], [0, 1, 1, 2, 3, 4], [1, 2, 1, 1, 1], "group_ptr[0]"),
     ]
     for ptr, tok, deg, word in bad:
