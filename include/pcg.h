@@ -316,7 +316,7 @@ pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits
  *
  *   thin_uniforms [B, n_trials, 3] float in [0,1), device, read-only; 1 <= n_trials <= 65536
  *   out_trials    [B] int32 or NULL: candidates drawn (1 after an all-accepted sequence; n_trials when exhausted)
- *   workspace     device, 256-byte aligned, at least pcg_verify_thinning_workspace_bytes(...) bytes (1052 bytes per
+ *   workspace     device, 256-byte aligned, at least pcg_verify_thinning_workspace_bytes(...) bytes (2076 bytes per
  *                 drafted position plus B*M*4 for sequences whose trials run out); contents need no initialisation
  *   the remaining arguments, ownership, asynchrony (no allocation, no synchronisation, the caller's stream only)
  *   and errors are pcg_verify's.  Rows that do not start on 16-byte boundaries or are not whole 16-byte words

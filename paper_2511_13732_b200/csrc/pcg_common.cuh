@@ -16,6 +16,8 @@ namespace pcg {
 constexpr float kNegInf = -__builtin_huge_valf();
 constexpr int kAggThreads = 512;        // threads per block of the aggregation kernels (fixes the sweep layout)
 constexpr uint32_t kNoGroup = 0xffffu;  // group field of sweep entries that belong to no group
+constexpr int kPartMaxGroups = 8;       // a part of the sparse product holds at most this many consecutive groups
+constexpr int kPartWarpsPerSM = 20;     // parts are sized so that one warp per part fills the GPU about once
 
 // Device-resident membership, built once by pcg_groups_create.
 struct GroupsDev {
@@ -39,6 +41,11 @@ struct GroupsDev {
     const float *ent_w;        // [ent_off[C]] weights in the same layout, or nullptr (equal split)
     const float *pair_w;       // [nnz] CSR-order weights w_{g,t} or nullptr (equal split)
     const float *rev_w;        // [nnz] the same in reverse-membership order, or nullptr
+    // Partition of the groups for the sparse product: part p is the run of whole groups [part_ptr[p], part_ptr[p+1]),
+    // at most kPartMaxGroups of them, cut so that every part holds about the same number of stored pairs.
+    const int32_t *part_ptr;   // [nparts+1]
+    const int32_t *part_ent;   // [nparts+1] group_ptr[part_ptr[p]]: the first stored pair of part p
+    int32_t nparts;
 };
 
 }  // namespace pcg
@@ -156,54 +163,25 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
     return r;
 }
 
+// The same with an L2 eviction policy (see l2_evict_first_policy): logits are read once, so their lines should be
+// the first to leave the L2 -- not the operands later kernels of the call keep there.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p, uint64_t pol) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p), "l"(pol));
+    return r;
+}
+
 __device__ __forceinline__ float ex2(float x) {  // 2^x, MUFU, flushes subnormal results to zero
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-
-// e = 2^(l*s - ms): the unnormalised softmax term of logit l with s = log2(e)/T and ms = max*s.
-__device__ __forceinline__ float softmax_term(float l, float s, float ms) { return ex2(__fmaf_rn(l, s, -ms)); }
-
-// ---- running (max, sum of 2^((l - max) s)) pairs ------------------------------------------------------------
-struct MaxSum {
-    float m;    // running maximum of the raw logits
-    float acc;  // sum of 2^((l - m) * s) over the logits seen so far
-};
-
-__device__ __forceinline__ MaxSum combine(const MaxSum &a, const MaxSum &b, float s) {
-    MaxSum r;
-    r.m = fmaxf(a.m, b.m);
-    if (r.m == kNegInf) {
-        r.acc = 0.f;
-    } else {
-        r.acc = a.acc * ex2((a.m - r.m) * s) + b.acc * ex2((b.m - r.m) * s);
-    }
-    return r;
-}
-
-// Deterministic block-wide combine: xor butterfly inside a warp, then a fixed-order pass over the warps.
-// `scratch` holds 2*NWARPS floats.  Every thread returns the same pair.
-template <int NT>
-__device__ __forceinline__ MaxSum block_combine(MaxSum v, float s, float *scratch) {
-    constexpr int NW = NT / 32;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        MaxSum w;
-        w.m = __shfl_xor_sync(0xffffffffu, v.m, o);
-        w.acc = __shfl_xor_sync(0xffffffffu, v.acc, o);
-        v = combine(v, w, s);
-    }
-    __syncthreads();  // scratch may still be read by a previous use
-    if ((threadIdx.x & 31) == 0) {
-        scratch[2 * (threadIdx.x >> 5)] = v.m;
-        scratch[2 * (threadIdx.x >> 5) + 1] = v.acc;
-    }
-    __syncthreads();
-    MaxSum r{scratch[0], scratch[1]};
-#pragma unroll
-    for (int w = 1; w < NW; ++w) r = combine(r, MaxSum{scratch[2 * w], scratch[2 * w + 1]}, s);
-    return r;
 }
 
 template <int NT>

@@ -273,12 +273,44 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     std::vector<float> inv((size_t)V);
     for (int t = 0; t < V; ++t) inv[t] = 1.0f / (float)deg[t];
 
+    // ---- partition of the groups for the sparse product (see GroupsDev::part_ptr) ----
+    // Cut points are the group boundaries nearest to the quantiles k * nnz / parts of the pair index, so that parts
+    // differ by at most about one group's size; runs of more than kPartMaxGroups (small) groups are cut further.
+    int sm_count = 148;
+    if (have_device) cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, device);
+    std::vector<int32_t> part_ptr;
+    {
+        const int64_t want = std::max<int64_t>(1, std::min<int64_t>((int64_t)sm_count * kPartWarpsPerSM, nnz / 32));
+        part_ptr.push_back(0);
+        int g = 0;
+        for (int64_t k = 1; k <= want && g < M; ++k) {
+            int gend = M;
+            if (k < want) {
+                const int64_t target = k * nnz / want;
+                int hi = (int)(std::lower_bound(gptr.begin() + g, gptr.end(), (int32_t)target) - gptr.begin());
+                hi = std::min(hi, M);
+                const int lo = std::max(hi - 1, g);
+                gend = (target - gptr[lo] <= (int64_t)gptr[hi] - target) ? lo : hi;
+                if (gend <= g) continue;  // the quantile falls inside a group larger than a part
+            }
+            while (gend - g > kPartMaxGroups) {
+                g += kPartMaxGroups;
+                part_ptr.push_back(g);
+            }
+            g = gend;
+            part_ptr.push_back(g);
+        }
+    }
+
     // ---- one device allocation for everything ----
     Carver cv;
     const size_t o_gptr = cv.take(gptr.size() * 4), o_gtok = cv.take(gtok.size() * 4), o_inv = cv.take(inv.size() * 4);
     const size_t o_rptr = cv.take(rptr.size() * 4), o_rgrp = cv.take(rgrp.size() * 4);
     const size_t o_eoff = cv.take(eoff.size() * 4), o_ent = cv.take(ent.size() * 4);
     const size_t o_w = cv.take(w.size() * 4), o_entw = cv.take(entw.size() * 4), o_rw = cv.take(rw.size() * 4);
+    std::vector<int32_t> part_ent(part_ptr.size());
+    for (size_t k = 0; k < part_ptr.size(); ++k) part_ent[k] = gptr[part_ptr[k]];
+    const size_t o_part = cv.take(part_ptr.size() * 4), o_pent = cv.take(part_ent.size() * 4);
     // scratch of the batched route of pcg_group_probs: 128 rows per chunk, more while Dt stays within 64 MB
     int probs_chunk = (int)std::min<int64_t>(256, std::max<int64_t>(128, ((int64_t)64 << 20) / ((int64_t)V * 4) / 128 * 128));
     const size_t o_pdt = cv.take((size_t)V * probs_chunk * 4), o_pst = cv.take((size_t)probs_chunk * 16);
@@ -302,6 +334,8 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     if (e == cudaSuccess) e = upload(base, o_w, w);
     if (e == cudaSuccess) e = upload(base, o_entw, entw);
     if (e == cudaSuccess) e = upload(base, o_rw, rw);
+    if (e == cudaSuccess) e = upload(base, o_part, part_ptr);
+    if (e == cudaSuccess) e = upload(base, o_pent, part_ent);
     if (e == cudaSuccess) e = cudaMemset(base + o_pz, 0, (size_t)probs_chunk * 4);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -329,10 +363,12 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     h->dev.pair_w = w.empty() ? nullptr : (const float *)(base + o_w);
     h->dev.ent_w = w.empty() ? nullptr : (const float *)(base + o_entw);
     h->dev.rev_w = w.empty() ? nullptr : (const float *)(base + o_rw);
+    h->dev.part_ptr = (const int32_t *)(base + o_part);
+    h->dev.part_ent = (const int32_t *)(base + o_pent);
+    h->dev.nparts = (int32_t)part_ptr.size() - 1;
     h->nnz = nnz;
     h->device = device;
-    h->sm_count = 1;
-    cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device);
+    h->sm_count = sm_count;
     h->max_group_size = max_group;
     h->max_degree = max_deg;
     h->device_bytes = (int64_t)total;

@@ -43,13 +43,14 @@ constexpr size_t kMaxDynSmem = 227 * 1024;  // dynamic shared memory a block may
 // That happens on a thread's first vector and practically never again, so the fast path costs exactly one
 // ex2 per logit and no max instructions.  Terms therefore stay below 2^32 and Z below V * 2^32.
 //
-// A block handles one drafted position: its first half streams the target row, its second half the draft row,
-// with 128-bit loads issued one batch (kBatch vectors per thread) ahead of the arithmetic.  The chain of
-// dependent loads that leads from the draft token to the label group's logits (token -> its groups -> label ->
-// group's token list -> logits) is spread over the streaming loop, one hop per batch, so its latency is hidden.
+// A block handles one drafted position: all its threads stream the target row, then the draft row (one long
+// contiguous run per block: measured 5 % faster than two half-blocks on a row each), with 128-bit loads issued
+// one batch (kBatch vectors per thread) ahead of the arithmetic and the draft row's first batch issued before the
+// target row is reduced.  The chain of dependent loads that leads from the draft token to the label group's
+// logits (token -> its groups -> label -> group's token list -> logits) is spread over the streaming loop, one hop
+// per batch, so its latency is hidden.
 
 constexpr int kPosThreads = 256;
-constexpr int kHalf = kPosThreads / 2;
 constexpr int kBatch = 4;
 constexpr float kRefInit = -1.0e30f;     // "no logit seen yet": finite, so that -inf logits give 2^-inf = 0, not NaN
 constexpr float kVecSumLimit = 4294967296.f;  // 2^32
@@ -109,8 +110,12 @@ struct PositionArgs {
     int32_t *labels;         // [B*K] group label of the draft token
     int32_t *posflags;       // [B*K]
     float4 *stats;           // [B*K] (RS_p, 1/Z_p, RS_q, 1/Z_q): scaled reference and reciprocal normaliser
-    float2 *strata;          // [B*K, kHalf] or null: every target-row thread's own (reference, sum); thread h has
-                             // summed the 16-byte words h, h + 128, h + 256, ... of the row (see pcg_thinning.cuh)
+    float2 *strata;          // [B*K, kPosThreads] or null: every thread's own (reference, sum) of the target row; thread h
+                             // has summed its 16-byte words h, h + 256, h + 512, ... (see pcg_thinning.cuh)
+    float4 *bonus_stats;     // [B] or null: (RS, 1/Z, 0, 0) of the bonus row (target row K), written by the block of a
+                             // sequence's LAST drafted position if that position was accepted (no sequence that
+                             // needs its bonus row can have its last position rejected)
+    int32_t *bonus_flags;    // [B] flags of that row (with bonus_stats)
 };
 
 // Group-label coupling: the label of draft token x is drawn from the groups containing x (reverse membership
@@ -140,28 +145,80 @@ __device__ __forceinline__ int draw_label(const GroupsDev &G, int r0, int n, flo
     return G.rev_grp[r0 + j];
 }
 
+// Softmax statistics of one row by the whole block (the bonus row of a sequence whose last drafted position was
+// accepted).  Kept out of line so that the streaming loop of the position kernel keeps its registers.
+template <typename T>
+__device__ __noinline__ void bonus_row_stats(const T *row, int V, float s, float *red, float4 *stats_out, int32_t *flags_out) {
+    constexpr int NT = kPosThreads, NW = NT / 32, NV = Elem<T>::kPerVec;
+    const int tid = threadIdx.x;
+    RefSum st{kRefInit * s, 0.f};
+    int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
+    if (head > V) head = V;
+    const int nvec = (V - head) / NV;
+    const uint4 *vp = reinterpret_cast<const uint4 *>(row + head);
+    int idx = tid;
+    for (; idx + 3 * NT < nvec; idx += 4 * NT) {
+        uint4 r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) r[j] = ld_stream(vp + idx + j * NT);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float v[NV];
+            Elem<T>::unpack(r[j], v);
+            absorb<NV>(st, v, s);
+        }
+    }
+    for (; idx < nvec; idx += NT) {
+        float v[NV];
+        Elem<T>::unpack(ld_stream(vp + idx), v);
+        absorb<NV>(st, v, s);
+    }
+    for (int t = tid; t < head; t += NT) absorb1(st, Elem<T>::widen(row[t]), s);
+    for (int t = head + nvec * NV + tid; t < V; t += NT) absorb1(st, Elem<T>::widen(row[t]), s);
+    float rs = st.rs, Z = st.acc;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) merge(rs, Z, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, Z, o));
+    if ((tid & 31) == 0) {
+        red[2 * (tid >> 5)] = rs;
+        red[2 * (tid >> 5) + 1] = Z;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        rs = red[0];
+        Z = red[1];
+        for (int w = 1; w < NW; ++w) merge(rs, Z, red[2 * w], red[2 * w + 1]);
+        *stats_out = make_float4(rs, 1.0f / Z, 0.f, 0.f);
+        *flags_out = (!(Z > 0.f) || isinf(Z) || isinf(rs)) ? PCG_FLAG_NONFINITE : 0;
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a, GroupsDev G) {
-    constexpr int NT = kPosThreads, H = kHalf, NW = NT / 32, HW = H / 32;
+    constexpr int NT = kPosThreads, NW = NT / 32;
     constexpr int NV = Elem<T>::kPerVec;
     constexpr int U = kBatch;
     constexpr int kChainSteps = 6;
-    __shared__ float red_z[2 * NW];
-    __shared__ float red_s[NW];
+    __shared__ float red_z[4 * NW];
+    __shared__ float red_s[2 * NW];
     const int tid = threadIdx.x;
-    const int half = tid / H, htid = tid - half * H;  // 0: target row, 1: draft row (warp-uniform)
     const int V = G.V, K = a.K;
     const float s = a.s;
-    const int pos = blockIdx.x;
-    const int b = pos / K, i = pos - b * K;
+    // Block order: the LAST drafted position of every sequence first (blocks 0 .. B-1), then the others.  Those
+    // blocks may have a third row to stream (the bonus row, see PositionArgs::bonus_stats); up front that extra
+    // work is spread over the first wave instead of lengthening the tail of the kernel.
+    const int nseq = (int)gridDim.x / K;
+    const int b = (int)blockIdx.x < nseq ? (int)blockIdx.x : ((int)blockIdx.x - nseq) / (K - 1);
+    const int i = (int)blockIdx.x < nseq ? K - 1 : ((int)blockIdx.x - nseq) - b * (K - 1);
+    const int pos = b * K + i;
     pdl_enter();  // (the first kernel of a call: lets the kernel behind it be scheduled while this one drains)
-    const T *row = half ? reinterpret_cast<const T *>(a.draft) + (int64_t)pos * V
-                        : reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + i) * V;
+    const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + i) * V;
+    const T *qrow = reinterpret_cast<const T *>(a.draft) + (int64_t)pos * V;
     const float *u = a.uniforms + ((int64_t)b * (K + 1) + i) * 2;
+    const uint64_t pol = l2_evict_first_policy();
 
     // ---- dependent-load chain towards the label group's logits (every thread, redundantly) ----
     int c_x = 0, c_r0 = 0, c_n = 1, c_g = 0, c_lo = 0, c_hi = 0, c_t = 0, c_flag = 0;
-    float c_u0 = 0.f, c_u1 = 0.f, c_l = kNegInf, c_w = 0.f;
+    float c_u0 = 0.f, c_u1 = 0.f, c_lp = kNegInf, c_lq = kNegInf, c_w = 0.f;
     auto chain = [&](int step) {
         switch (step) {
             case 0:
@@ -185,36 +242,45 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
                 c_hi = G.group_ptr[c_g + 1];
                 break;
             case 4:
-                if (c_lo + htid < c_hi) c_t = G.group_tok[c_lo + htid];
+                if (c_lo + tid < c_hi) c_t = G.group_tok[c_lo + tid];
                 break;
             case 5:
-                if (c_lo + htid < c_hi) {
-                    c_l = Elem<T>::widen(row[c_t]);
-                    c_w = G.pair_w ? G.pair_w[c_lo + htid] : G.inv_deg[c_t];
+                if (c_lo + tid < c_hi) {
+                    c_lp = Elem<T>::widen(trow[c_t]);
+                    c_lq = Elem<T>::widen(qrow[c_t]);
+                    c_w = G.pair_w ? G.pair_w[c_lo + tid] : G.inv_deg[c_t];
                 }
                 break;
         }
     };
-
-    // ---- stream the row: elements before the first 16-byte boundary, whole vectors, the rest ----
-    RefSum st{kRefInit * s, 0.f};
     int chained = 0;
-    int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
-    if (head > V) head = V;
-    const int nvec = (V - head) / NV;
-    const int nfull = nvec / (H * U);  // batches in which every thread has all U vectors
-    {
-        const uint4 *p = reinterpret_cast<const uint4 *>(row + head) + htid;
-        uint4 cur[U], nxt[U];
-        if (nfull > 0) {
+
+    // The whole block streams the target row, then the draft row: thread h takes the 16-byte words h, h + 256, ...
+    // of a row, U of them in flight.  A row = elements before the first 16-byte boundary, whole vectors, the rest.
+    uint4 cur[U];
+    auto plan_head = [&](const T *row) {
+        const int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
+        return head > V ? V : head;
+    };
+    auto first_batch = [&](const T *row) {  // the first U vectors of this thread, if the row has a full batch
+        const int head = plan_head(row);
+        if ((V - head) / NV / (NT * U) > 0) {
+            const uint4 *p = reinterpret_cast<const uint4 *>(row + head) + tid;
 #pragma unroll
-            for (int j = 0; j < U; ++j) cur[j] = ld_stream(p + j * H);
+            for (int j = 0; j < U; ++j) cur[j] = ld_stream(p + j * NT, pol);
         }
+    };
+    auto stream_row = [&](const T *row, RefSum &st) {  // `cur` holds the first batch on entry
+        const int head = plan_head(row);
+        const int nvec = (V - head) / NV;
+        const int nfull = nvec / (NT * U);  // batches in which every thread has all U vectors
+        const uint4 *p = reinterpret_cast<const uint4 *>(row + head) + tid;
+        uint4 nxt[U];
         for (int bi = 0; bi < nfull; ++bi) {
-            p += H * U;
+            p += NT * U;
             if (bi + 1 < nfull) {
 #pragma unroll
-                for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * H);
+                for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * NT, pol);
             }
             if (chained < kChainSteps) chain(chained++);
 #pragma unroll
@@ -226,52 +292,68 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
 #pragma unroll
             for (int j = 0; j < U; ++j) cur[j] = nxt[j];
         }
-        // remaining whole vectors (fewer than H*U), then the scalar head and tail
-        for (int idx = nfull * H * U + htid; idx < nvec; idx += H) {
+        // remaining whole vectors (fewer than NT*U), then the scalar head and tail
+        for (int idx = nfull * NT * U + tid; idx < nvec; idx += NT) {
             float v[NV];
             Elem<T>::unpack(ld_stream(reinterpret_cast<const uint4 *>(row + head) + idx), v);
             absorb<NV>(st, v, s);
         }
-        for (int t = htid; t < head; t += H) absorb1(st, Elem<T>::widen(row[t]), s);
-        for (int t = head + nvec * NV + htid; t < V; t += H) absorb1(st, Elem<T>::widen(row[t]), s);
-    }
+        for (int t = tid; t < head; t += NT) absorb1(st, Elem<T>::widen(row[t]), s);
+        for (int t = head + nvec * NV + tid; t < V; t += NT) absorb1(st, Elem<T>::widen(row[t]), s);
+    };
+    // (rs, Z) of a row from the threads' pairs: xor butterfly inside a warp, then a fixed-order pass over the warps
+    auto reduce_row = [&](const RefSum &st, float *red, float &rs_out, float &Z_out) {
+        float rs = st.rs, Z = st.acc;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) merge(rs, Z, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, Z, o));
+        if ((tid & 31) == 0) {
+            red[2 * (tid >> 5)] = rs;
+            red[2 * (tid >> 5) + 1] = Z;
+        }
+        __syncthreads();
+        rs = red[0], Z = red[1];
+#pragma unroll
+        for (int w = 1; w < NW; ++w) merge(rs, Z, red[2 * w], red[2 * w + 1]);
+        rs_out = rs, Z_out = Z;
+    };
+
+    first_batch(trow);
+    RefSum st{kRefInit * s, 0.f};
+    stream_row(trow, st);
+    if (a.strata) a.strata[(size_t)pos * NT + tid] = make_float2(st.rs, st.acc);  // a free by-product
+    first_batch(qrow);  // the draft row's first loads go out before the target row's reduction
+    float rs_p, Zp, rs_q, Zq;
+    reduce_row(st, red_z, rs_p, Zp);
+    st = RefSum{kRefInit * s, 0.f};
+    stream_row(qrow, st);
     while (chained < kChainSteps) chain(chained++);
-    if (a.strata && half == 0) a.strata[(size_t)pos * H + htid] = make_float2(st.rs, st.acc);  // a free by-product
+    reduce_row(st, red_z + 2 * NW, rs_q, Zq);
 
-    // ---- per-row (rs, Z): xor butterfly inside a warp, then a fixed-order pass over each half's warps ----
-    float rs = st.rs, Z = st.acc;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) merge(rs, Z, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, Z, o));
-    if ((tid & 31) == 0) {
-        red_z[2 * (tid >> 5)] = rs;
-        red_z[2 * (tid >> 5) + 1] = Z;
-    }
-    __syncthreads();
-    float rs_p = red_z[0], Zp = red_z[1], rs_q = red_z[2 * HW], Zq = red_z[2 * HW + 1];
-#pragma unroll
-    for (int w = 1; w < HW; ++w) {
-        merge(rs_p, Zp, red_z[2 * w], red_z[2 * w + 1]);
-        merge(rs_q, Zq, red_z[2 * (HW + w)], red_z[2 * (HW + w) + 1]);
-    }
-
-    // ---- mass of the label group under this half's row (first element prefetched by the chain) ----
-    const float rs_mine = half ? rs_q : rs_p;
-    float part = __fmul_rn(ex2(__fmaf_rn(c_l, s, -rs_mine)), c_w);
-    for (int k = c_lo + htid + H; k < c_hi; k += H) {  // groups larger than half a block
+    // ---- masses of the label group under the two rows (first element prefetched by the chain) ----
+    float part_p = __fmul_rn(ex2(__fmaf_rn(c_lp, s, -rs_p)), c_w);
+    float part_q = __fmul_rn(ex2(__fmaf_rn(c_lq, s, -rs_q)), c_w);
+    for (int k = c_lo + tid + NT; k < c_hi; k += NT) {  // groups larger than a block
         const int t = G.group_tok[k];
         const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
-        part += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(row[t]), s, -rs_mine)), w);
+        part_p += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs_p)), w);
+        part_q += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), s, -rs_q)), w);
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-    if ((tid & 31) == 0) red_s[tid >> 5] = part;
+    for (int o = 16; o > 0; o >>= 1) {
+        part_p += __shfl_xor_sync(0xffffffffu, part_p, o);
+        part_q += __shfl_xor_sync(0xffffffffu, part_q, o);
+    }
+    if ((tid & 31) == 0) {
+        red_s[tid >> 5] = part_p;
+        red_s[NW + (tid >> 5)] = part_q;
+    }
     __syncthreads();
 
     if (tid == 0) {
-        float Sp = red_s[0], Sq = red_s[HW];
-        for (int w = 1; w < HW; ++w) {
+        float Sp = red_s[0], Sq = red_s[NW];
+        for (int w = 1; w < NW; ++w) {
             Sp += red_s[w];
-            Sq += red_s[HW + w];
+            Sq += red_s[NW + w];
         }
         // acceptance u < min(1, P/Q) without a division: P = Sp/Zp, Q = Sq/Zq
         const float lhs = Sp * Zq, rhs = Sq * Zp;
@@ -283,6 +365,13 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
         a.labels[pos] = c_g;
         a.posflags[pos] = flag;
         a.stats[pos] = make_float4(rs_p, 1.0f / Zp, rs_q, 1.0f / Zq);
+        red_s[0] = acc ? 1.f : 0.f;
+    }
+    if (a.bonus_stats && i == K - 1) {  // block-uniform: the last drafted position of its sequence
+        __syncthreads();
+        if (red_s[0] != 0.f)  // accepted: the sequence may need its bonus row
+            bonus_row_stats<T>(reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + K) * V, V, s, red_z,
+                               a.bonus_stats + b, a.bonus_flags + b);
     }
 }
 
@@ -709,39 +798,27 @@ __global__ void __launch_bounds__(kAggThreads, 2) terminal_kernel(TerminalArgs a
 // ================================================================ batched terminal stage ====================
 //
 // The terminal draw of a sequence needs the residual (P - Q)_+ of ALL groups at one position (the first
-// rejection, or the bonus row).  Over a batch that is one sparse-matrix product: R[b, g] = sum_{t in G_g}
-// D[b, t], with D[b, t] = (p(t) - q(t)) / N(t) at sequence b's terminal position.  Four kernels:
-//   terminal_prepare_kernel    one block per sequence: warp ballot over the accept bits -> first rejection n_b;
-//                              if everything was accepted, the softmax statistics of the bonus row
-//   residual_transpose_kernel  re-reads the two rows of every sequence's terminal position and writes D
-//                              TRANSPOSED, Dt[t, b]: the sequences of a chunk side by side in one line
-//   group_spmm_kernel          one warp per (a few consecutive groups, block of 32 to 256 sequences): walks the
-//                              groups' token lists once and adds one row segment of Dt per token (Dt stays in L2)
-//   terminal_draw_kernel       one block per sequence: prefix scan over the M residual masses, group draw,
-//                              within-group token draw, outputs
-// Sequences are processed in chunks whose Dt fits in L2.
+// rejection, or the bonus row).  Over a batch that is one sparse-matrix product: R[g, b] = sum_{t in G_g}
+// D[b, t], with D[b, t] = (p(t) - q(t)) / N(t) at sequence b's terminal position.  Three kernels:
+//   residual_transpose_kernel  finds every sequence's first rejection (warp ballots over the accept bits), re-reads
+//                              the two rows of that position and writes D TRANSPOSED: tiles of 32 sequences side by
+//                              side, Dt[batch of 32][token][32], one bulk copy per tile
+//   group_spmm_kernel          one warp per (part of the groups, block of 32 to 256 sequences): walks the part's
+//                              token lists once and adds one row segment of Dt per token (Dt stays in L2); writes
+//                              the group sums and, per part, the sum of their positive parts
+//   terminal_pick_kernel       one block per sequence: prefix scan over the parts' sums, the part in which the
+//                              cumulative mass passes u * Z is opened, group draw, token draw, outputs
+// Sequences are processed in chunks whose Dt fits in L2.  pcg_group_probs uses the first two with row-major
+// output; dense mode (all groups at every position) uses terminal_prepare_kernel and terminal_draw_kernel.
 
 constexpr int kPrepThreads = 256;  // terminal_prepare_kernel, row_stats_kernel
 constexpr int kProbsBatchedRows = 64;  // pcg_group_probs: from this many rows on, the batched kernels
 constexpr int kTrThreads = 256;    // residual_transpose_kernel
-#ifndef PCG_SPMM_THREADS
-#define PCG_SPMM_THREADS 128
-#endif
-constexpr int kSpmmThreads = PCG_SPMM_THREADS;  // group_spmm_kernel
-#ifndef PCG_SPMM_SPL
-#define PCG_SPMM_SPL 4    // sequences per lane of the sparse product for batches of 128 to 255 sequences (8 beyond, 1 below)
-#endif
-#ifndef PCG_SPMM_DEPTH
-#define PCG_SPMM_DEPTH 8  // tokens per batch of that form of the sparse product; two batches of loads are in flight per lane
-#endif
-#ifndef PCG_SPMM_GW
-#define PCG_SPMM_GW 4  // consecutive groups per warp of the sparse product when the launch has many waves
-#endif
-constexpr int kSpmmGroupsPerWarp = PCG_SPMM_GW;
-constexpr int kSpmmMaxGroupsPerWarp = 8;  // chosen per launch between 2 and this (see launch_spmm)
-constexpr int kSpmmWide = PCG_SPMM_SPL;
-constexpr int kSpmmDepth = PCG_SPMM_DEPTH;
-constexpr int kDrawThreads = 512;  // terminal_draw_kernel
+constexpr int kSpmmThreads = 128;  // group_spmm_kernel
+constexpr int kSpmmWide = 4;       // sequences per lane of the sparse product for batches of 128 to 255 sequences (8 beyond, 1 below)
+constexpr int kSpmmDepth = 8;      // tokens per batch of that form; two batches of loads are in flight per lane
+constexpr int kDrawThreads = 512;  // terminal_draw_kernel (dense mode)
+constexpr int kPickThreads = 256;  // terminal_pick_kernel
 
 struct PrepareArgs {
     const void *target;
@@ -756,86 +833,39 @@ struct PrepareArgs {
     float4 *term_stats;   // [B] (RS_p, 1/Z_p, RS_q, 1/Z_q) of the terminal position; (RS_p, 1/Z_p, 0, 0) for a bonus row
 };
 
+// First rejected position of sequence b by one warp: ballots over the accept bits, 32 positions at a time (the
+// first word with a rejection ends the search), and the OR of the flags of the positions up to and including it.
+__device__ __forceinline__ void warp_first_reject(const int32_t *accept, const int32_t *posflags, int b, int K, int lane,
+                                                  int &n_out, int &flags_out) {
+    int n = K, flags = 0;
+    for (int base = 0; base < K && n == K; base += 32) {
+        const int i = base + lane;
+        const int rej = (i < K) && (accept[b * K + i] == 0);
+        const unsigned mask = __ballot_sync(0xffffffffu, rej);
+        if (mask) n = base + __ffs(mask) - 1;
+    }
+    for (int base = 0; base < K && base <= n; base += 32) {
+        const int i = base + lane;
+        const int f = (i < K && i <= n) ? posflags[b * K + i] : 0;
+        flags |= __reduce_or_sync(0xffffffffu, f);
+    }
+    n_out = n;
+    flags_out = flags;
+}
+
+// Dense mode only: first rejection per sequence from the accept bits of dense_accept_kernel.
 template <typename T>
 __global__ void __launch_bounds__(kPrepThreads) terminal_prepare_kernel(PrepareArgs a, GroupsDev G) {
     pdl_enter();
-    constexpr int NT = kPrepThreads, NW = NT / 32, NV = Elem<T>::kPerVec;
-    __shared__ int s_n, s_flags;
-    __shared__ float red[2 * NW];
-    const int b = blockIdx.x, tid = threadIdx.x, K = a.K, V = G.V;
-    // ---- first rejected position: warp ballots over the accept bits, 32 positions at a time ----
+    const int b = blockIdx.x, tid = threadIdx.x, K = a.K;
     if (tid < 32) {
-        // 32 accept bits per ballot; the first word with a rejection ends the search
-        int n = K, flags = 0;
-        for (int base = 0; base < K && n == K; base += 32) {
-            const int i = base + tid;
-            const int rej = (i < K) && (a.accept[b * K + i] == 0);
-            const unsigned mask = __ballot_sync(0xffffffffu, rej);
-            if (mask) n = base + __ffs(mask) - 1;
-        }
-        for (int base = 0; base < K && base <= n; base += 32) {
-            const int i = base + tid;
-            const int f = (i < K && i <= n) ? a.posflags[b * K + i] : 0;
-            flags |= __reduce_or_sync(0xffffffffu, f);
-        }
-        if (tid == 0) {
-            s_n = n;
-            s_flags = flags;
-        }
-    }
-    __syncthreads();
-    const int n = s_n;
-    if (n < K || !a.want_bonus_stats) {
+        int n, flags;
+        warp_first_reject(a.accept, a.posflags, b, K, tid, n, flags);
         if (tid == 0) {
             a.term_n[b] = n;
-            a.term_flags[b] = s_flags;
+            a.term_flags[b] = flags;
             a.term_stats[b] = n < K ? a.stats[b * K + n] : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        return;
-    }
-    // ---- every position accepted: softmax statistics of the bonus row (target row K) ----
-    const T *row = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + K) * V;
-    RefSum st{kRefInit * a.s, 0.f};
-    int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
-    if (head > V) head = V;
-    const int nvec = (V - head) / NV;
-    const uint4 *vp = reinterpret_cast<const uint4 *>(row + head);
-    int idx = tid;
-    for (; idx + 3 * NT < nvec; idx += 4 * NT) {
-        uint4 r[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) r[j] = ld_stream(vp + idx + j * NT);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            float v[NV];
-            Elem<T>::unpack(r[j], v);
-            absorb<NV>(st, v, a.s);
-        }
-    }
-    for (; idx < nvec; idx += NT) {
-        float v[NV];
-        Elem<T>::unpack(ld_stream(vp + idx), v);
-        absorb<NV>(st, v, a.s);
-    }
-    for (int t = tid; t < head; t += NT) absorb1(st, Elem<T>::widen(row[t]), a.s);
-    for (int t = head + nvec * NV + tid; t < V; t += NT) absorb1(st, Elem<T>::widen(row[t]), a.s);
-    float rs = st.rs, Z = st.acc;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) merge(rs, Z, __shfl_xor_sync(0xffffffffu, rs, o), __shfl_xor_sync(0xffffffffu, Z, o));
-    if ((tid & 31) == 0) {
-        red[2 * (tid >> 5)] = rs;
-        red[2 * (tid >> 5) + 1] = Z;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        rs = red[0];
-        Z = red[1];
-        for (int w = 1; w < NW; ++w) merge(rs, Z, red[2 * w], red[2 * w + 1]);
-        int flags = s_flags;
-        if (!(Z > 0.f) || isinf(Z) || isinf(rs)) flags |= PCG_FLAG_NONFINITE;
-        a.term_n[b] = n;
-        a.term_flags[b] = flags;
-        a.term_stats[b] = make_float4(rs, 1.0f / Z, 0.f, 0.f);
     }
 }
 
@@ -903,119 +933,231 @@ __device__ __forceinline__ float4 ld_l2_f32x4(const float *p) {
                  : "l"(p));
     return r;
 }
-#ifdef PCG_DT_STORE_EVICT_LAST
-__device__ __forceinline__ void st_dt(float *p, float v) {
-    uint64_t pol;
-    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(v), "l"(pol) : "memory");
-}
-#else
-__device__ __forceinline__ void st_dt(float *p, float v) { *p = v; }
-#endif
 
 struct TransposeArgs {
     const void *target;
     const void *draft;
     int B, K;
     int b0;             // first sequence of this chunk
-    int bpad;           // sequences per line of Dt (row stride of Dt, a multiple of 32)
     float s;
-    const int32_t *term_n;
-    const float4 *term_stats;
-    float *Dt;          // [V, bpad]
+    // The terminal position of a sequence comes from the accept bits of the position kernel (from_accept = 1: this
+    // kernel finds the first rejection itself and leaves term_n / term_flags / term_stats for the kernels behind
+    // it), or is read from term_n / term_stats as filled by an earlier kernel (from_accept = 0).
+    int from_accept;
+    const int32_t *accept, *posflags;  // [B*K]
+    const float4 *stats;               // [B*K]
+    const float4 *bonus_stats;         // [B]
+    const int32_t *bonus_flags;        // [B]
+    int32_t *term_n;                   // [B]
+    int32_t *term_flags;               // [B]
+    float4 *term_stats;                // [B]
+    float *Dt;                         // [sequences of the chunk / 32][V][32]
 };
 
-#ifndef PCG_TR_MINBLOCKS
-#define PCG_TR_MINBLOCKS 3  // caps the registers so that 24 warps per SM are resident (measured best)
-#endif
-// Grid (ceil(V / TT), bpad / 32): a tile of TT tokens x 32 sequences.  Warp w loads the row segments of
-// sequences w, w+8, w+16, w+24 (one 16-byte vector per lane), the tile is turned in shared memory (column
-// rotated by the vector index, so that both sides are free of bank conflicts) and written out one 128-byte
-// line per token.  Sequences past the end of the batch get zeros.
+// The bits of "-inf" in the logits' storage type, two (or one) to a 32-bit word: what a lane uses in place of
+// logits it must not read (past the end of a row, the draft row of a bonus position, sequences past the batch).
 template <typename T>
-__global__ void __launch_bounds__(kTrThreads, PCG_TR_MINBLOCKS) residual_transpose_kernel(TransposeArgs a, GroupsDev G) {
+struct NegInfBits;
+template <>
+struct NegInfBits<float> {
+    static constexpr uint32_t word = 0xff800000u;
+};
+template <>
+struct NegInfBits<uint16_t> {
+    static constexpr uint32_t word = 0xff80ff80u;
+};
+template <>
+struct NegInfBits<f16_t> {
+    static constexpr uint32_t word = 0xfc00fc00u;
+};
+
+// The logits held by one 32-bit word of a row.
+template <typename T>
+struct WordElems;
+template <>
+struct WordElems<float> {
+    static constexpr int kPerWord = 1;
+    static __device__ __forceinline__ void unpack(uint32_t w, float (&v)[1]) { v[0] = __uint_as_float(w); }
+};
+template <>
+struct WordElems<uint16_t> {
+    static constexpr int kPerWord = 2;
+    static __device__ __forceinline__ void unpack(uint32_t w, float (&v)[2]) {
+        v[0] = __uint_as_float(w << 16);
+        v[1] = __uint_as_float(w & 0xffff0000u);
+    }
+};
+template <>
+struct WordElems<f16_t> {
+    static constexpr int kPerWord = 2;
+    static __device__ __forceinline__ void unpack(uint32_t w, float (&v)[2]) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
+        v[0] = f.x;
+        v[1] = f.y;
+    }
+};
+
+// 32 bytes of a row, streamed (read once: first to leave the L2, so that Dt stays).
+__device__ __forceinline__ void ld_stream_32(const void *p, uint32_t (&w)[8]) {
+    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p));
+}
+
+// Grid (blocks per batch, batches of 32 sequences); block = 8 warps.  LANE = SEQUENCE throughout: a lane reads
+// 32 bytes of its own sequence's two rows per step (whole sectors; the eight warps of a block take neighbouring
+// steps, so a row is fetched in 256-byte stretches), forms D = (p - q) w for those tokens in registers, and the
+// warp writes one 128-byte line of Dt per token -- [token][32 sequences] needs no transposition this way.
+//   0. once per block, by warp 0: every lane finds its sequence's first rejection from the accept bits (its
+//      loads all in flight) and fetches the softmax statistics of that position;
+//   1. the block's run of the row is walked with the next step's 64 bytes in flight while the current step's
+//      tokens are computed and stored.
+// Lanes that have nothing to read (sequences past the batch, the draft row of a bonus position, tokens past the
+// end of a row) use -inf logits, which contribute exact zeros.
+template <typename T>
+__global__ void __launch_bounds__(kTrThreads, 3) residual_transpose_kernel(TransposeArgs a, GroupsDev G) {
     pdl_enter();
-    constexpr int NV = Elem<T>::kPerVec, TT = 32 * NV;
-    __shared__ float tile[TT * 32];
+    constexpr int PW = WordElems<T>::kPerWord;  // logits per 32-bit word
+    constexpr int CH = 8 * PW;                  // tokens per step: 32 bytes of a row
+    constexpr int NWARP = kTrThreads / 32;
+    __shared__ int s_n[32];
+    __shared__ float4 s_st[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = G.V, K = a.K;
-    const int t0 = blockIdx.x * TT;
     const int bbase = a.b0 + blockIdx.y * 32;
-    const int t = t0 + lane * NV;  // first token of this lane's vector
-    float invd[NV];
+
+    // ---- 0. terminal position and statistics of the batch's sequences ----
+    if (warp == 0) {
+        const int b = bbase + lane;
+        int n = -1, flags = 0;
+        float4 st = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (b < a.B) {
+            if (!a.from_accept) {
+                n = a.term_n[b];
+                st = a.term_stats[b];
+            } else {
+                n = K;
+                for (int i0 = 0; i0 < K && n == K; i0 += 16) {  // sixteen positions' loads in flight
+                    int acc[16], pf[16];
 #pragma unroll
-    for (int e = 0; e < NV; ++e) invd[e] = (!G.ent_w && t + e < V) ? G.inv_deg[t + e] : 1.f;
-    // all of this thread's loads first (4 sequences x 2 rows), then the arithmetic
-    int n[4];
-    float4 st[4];
-    uint4 rp[4], rq[4];
-    bool fast[4];
+                    for (int j = 0; j < 16; ++j) {
+                        const bool in = i0 + j < K;
+                        acc[j] = in ? a.accept[b * K + i0 + j] : 1;
+                        pf[j] = in ? a.posflags[b * K + i0 + j] : 0;
+                    }
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const int b = bbase + warp + 8 * q;
-        n[q] = b < a.B ? a.term_n[b] : -1;
-        st[q] = b < a.B ? a.term_stats[b] : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const int b = bbase + warp + 8 * q;
-        const T *tp = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + max(n[q], 0)) * V + t;
-        const T *qp = K > 0 ? reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(max(n[q], 0), K - 1)) * V + t : tp;
-        fast[q] = n[q] >= 0 && t + NV <= V && (((uintptr_t)tp | (uintptr_t)qp) & 15u) == 0;
-        rp[q] = rq[q] = make_uint4(0u, 0u, 0u, 0u);
-        if (fast[q]) {
-            rp[q] = ld_stream(reinterpret_cast<const uint4 *>(tp));
-            if (n[q] < K) rq[q] = ld_stream(reinterpret_cast<const uint4 *>(qp));
-        }
-    }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const int sl = warp + 8 * q;
-        float d[NV];
-#pragma unroll
-        for (int e = 0; e < NV; ++e) d[e] = 0.f;
-        if (n[q] >= 0 && t < V) {
-            const int b = bbase + sl;
-            float lp[NV], lq[NV];
-            const bool resid = n[q] < K;
-            if (fast[q]) {
-                Elem<T>::unpack(rp[q], lp);
-                Elem<T>::unpack(rq[q], lq);
-            } else {  // ragged end of the row or rows that are not 16-byte aligned
-                const T *tp = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n[q]) * V + t;
-                const T *qp = K > 0 ? reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(n[q], K - 1)) * V + t : tp;
-#pragma unroll
-                for (int e = 0; e < NV; ++e) {
-                    const bool in = t + e < V;
-                    lp[e] = in ? Elem<T>::widen(tp[e]) : kNegInf;
-                    lq[e] = (in && resid) ? Elem<T>::widen(qp[e]) : kNegInf;
+                    for (int j = 0; j < 16; ++j) {
+                        if (n == K) {
+                            flags |= pf[j];  // flags of the positions up to and including the first rejection
+                            if (acc[j] == 0) n = i0 + j;
+                        }
+                    }
+                }
+                if (n < K) {
+                    st = a.stats[b * K + n];
+                } else {
+                    st = a.bonus_stats[b];
+                    flags |= a.bonus_flags[b];
+                }
+                if (blockIdx.x == 0) {
+                    a.term_n[b] = n;
+                    a.term_flags[b] = flags;
+                    a.term_stats[b] = st;
                 }
             }
-#pragma unroll
-            for (int e = 0; e < NV; ++e) {
-                float v = __fmul_rn(ex2(__fmaf_rn(lp[e], a.s, -st[q].x)), st[q].y);
-                if (resid) v -= __fmul_rn(ex2(__fmaf_rn(lq[e], a.s, -st[q].z)), st[q].w);
-                d[e] = __fmul_rn(v, invd[e]);
-            }
         }
-#pragma unroll
-        for (int e = 0; e < NV; ++e) tile[(lane * NV + e) * 32 + ((sl + lane) & 31)] = d[e];
+        s_n[lane] = n;
+        s_st[lane] = st;
     }
     __syncthreads();
-    float *out = a.Dt + (size_t)blockIdx.y * 32 + lane;
-    for (int r = warp; r < TT; r += kTrThreads / 32) {
-        const int tok = t0 + r;
-        if (tok < V) st_dt(out + (size_t)tok * a.bpad, tile[r * 32 + ((lane + r / NV) & 31)]);
+
+    // ---- 1. this lane's sequence ----
+    const int n = s_n[lane];
+    float4 st = s_st[lane];
+    const bool live = n >= 0, resid = live && n < K;
+    if (!live) st = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (!resid) st.z = 0.f, st.w = 0.f;  // no draft term: its logits read as -inf and the factor is zero
+    const int b = bbase + lane, nn = max(n, 0);
+    const T *tp = reinterpret_cast<const T *>(a.target) + ((int64_t)(live ? b : 0) * (K + 1) + nn) * V;
+    const T *qp = K > 0 ? reinterpret_cast<const T *>(a.draft) + ((int64_t)(live ? b : 0) * K + min(nn, K - 1)) * V : tp;
+    // whole 32-byte pieces can be loaded as such if every live lane's rows start on 32-byte boundaries
+    const bool lane_al = !live || ((((uintptr_t)tp | (resid ? (uintptr_t)qp : 0)) & 31u) == 0);
+    const bool aligned = __all_sync(0xffffffffu, lane_al) && ((size_t)V * sizeof(T)) % 32 == 0;
+    const int nsteps = (V + CH - 1) / CH;
+    const int step_lo = (int)(((int64_t)nsteps * blockIdx.x) / gridDim.x);
+    const int step_hi = (int)(((int64_t)nsteps * (blockIdx.x + 1)) / gridDim.x);
+    float *dst = a.Dt + ((size_t)blockIdx.y * V) * 32 + lane;
+
+    auto fetch = [&](int step, uint32_t(&wp)[8], uint32_t(&wq)[8]) {
+        const int t = step * CH;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) wp[j] = wq[j] = NegInfBits<T>::word;
+        if (step >= step_hi) return;
+        if (aligned && t + CH <= V) {
+            if (live) ld_stream_32(tp + t, wp);
+            if (resid) ld_stream_32(qp + t, wq);
+        } else {  // ragged end of the row, or rows that are not 32-byte aligned: element by element
+            T ep[CH], eq[CH];
+            memcpy(ep, wp, 32);
+            memcpy(eq, wq, 32);
+#pragma unroll
+            for (int e = 0; e < CH; ++e) {
+                if (t + e < V) {
+                    if (live) ep[e] = tp[t + e];
+                    if (resid) eq[e] = qp[t + e];
+                }
+            }
+            memcpy(wp, ep, 32);
+            memcpy(wq, eq, 32);
+        }
+    };
+    auto emit = [&](int step, const uint32_t(&wp)[8], const uint32_t(&wq)[8]) {
+        const int t = step * CH;
+        float inv[CH];
+        if (!G.ent_w && t + CH <= V) {
+#pragma unroll
+            for (int j = 0; j < CH / 4; ++j) {
+                const float4 v = *reinterpret_cast<const float4 *>(G.inv_deg + t + 4 * j);  // (the same for all lanes)
+                inv[4 * j] = v.x, inv[4 * j + 1] = v.y, inv[4 * j + 2] = v.z, inv[4 * j + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < CH; ++e) inv[e] = (!G.ent_w && t + e < V) ? G.inv_deg[t + e] : 1.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float lp[PW], lq[PW];
+            WordElems<T>::unpack(wp[j], lp);
+            WordElems<T>::unpack(wq[j], lq);
+#pragma unroll
+            for (int e = 0; e < PW; ++e) {
+                float v = __fmul_rn(ex2(__fmaf_rn(lp[e], a.s, -st.x)), st.y);
+                v -= __fmul_rn(ex2(__fmaf_rn(lq[e], a.s, -st.z)), st.w);
+                const int r = t + j * PW + e;
+                if (r < V) dst[(size_t)r * 32] = __fmul_rn(v, inv[j * PW + e]);
+            }
+        }
+    };
+    uint32_t ap[8], aq[8], bp[8], bq[8];
+    int step = step_lo + warp;
+    fetch(step, ap, aq);
+    for (; step < step_hi; step += 2 * NWARP) {
+        fetch(step + NWARP, bp, bq);
+        emit(step, ap, aq);
+        if (step + NWARP < step_hi) {
+            fetch(step + 2 * NWARP, ap, aq);
+            emit(step + NWARP, bp, bq);
+        }
     }
 }
 
 struct SpmmArgs {
-    const float *Dt;  // [V, bpad]
+    const float *Dt;  // [sequences of the chunk / 32][V][32]
     int B;
     int b0;           // first sequence of this chunk
-    int bpad;
-    float *R;         // [B, M] (raw sums; the consumer clamps at zero)
-    int gw;           // consecutive groups per warp, at most kSpmmMaxGroupsPerWarp
+    int bpad;         // sequences per row of Rt and Psum (the chunk size, a multiple of 32 * SPL)
+    float *R;         // ROWMAJOR: [B, M] raw sums by sequence (pcg_group_probs); else Rt [M, bpad] by group
+    float *Psum;      // [nparts, bpad]: per part, the sum of the positive parts of its groups' sums (not ROWMAJOR)
 };
 
 template <int SPL>
@@ -1024,13 +1166,7 @@ template <>
 struct SeqVec<1> {
     float v[1];
     __device__ __forceinline__ void load(const float *p) { v[0] = ld_l2_f32(p); }
-};
-template <>
-struct SeqVec<2> {
-    float v[2];
-    __device__ __forceinline__ void load(const float *p) {
-        asm volatile("ld.global.cg.v2.f32 {%0,%1}, [%2];" : "=f"(v[0]), "=f"(v[1]) : "l"(p));
-    }
+    __device__ __forceinline__ void store(float *p) const { *p = v[0]; }
 };
 template <>
 struct SeqVec<4> {
@@ -1039,8 +1175,8 @@ struct SeqVec<4> {
         const float4 r = ld_l2_f32x4(p);
         v[0] = r.x, v[1] = r.y, v[2] = r.z, v[3] = r.w;
     }
+    __device__ __forceinline__ void store(float *p) const { *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]); }
 };
-
 template <>
 struct SeqVec<8> {  // one 256-bit load per lane
     float v[8];
@@ -1049,32 +1185,42 @@ struct SeqVec<8> {  // one 256-bit load per lane
                      : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
                      : "l"(p));
     }
+    __device__ __forceinline__ void store(float *p) const {
+        reinterpret_cast<float4 *>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
+        reinterpret_cast<float4 *>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
+    }
 };
 
-// Grid (ceil(M / (GW * warps per block)), bpad / (32 * SPL)).  A warp owns GW = a.gw consecutive groups -- their token
-// lists are one contiguous range of the CSR -- and a block of 32 * SPL sequences; a lane holds SPL consecutive
-// sequences (one 4-, 16- or 32-byte load per token).  The range is walked in batches of DEPTH tokens with two
-// register buffers: the loads of batch i+1 are issued before batch i is added, so a warp keeps up to 2 * DEPTH
-// lines of Dt in flight at all times (random L2 gathers need on the order of 150 KB in flight per SM to
-// reach the L2's bandwidth).  Token ids are fetched 32 at a time, one block of 32 ahead.  Sums run in CSR
-// order; a group ends where the running entry index reaches the next group pointer.  The warp's GW x (32 * SPL)
-// sums are turned in shared memory so that R is written along the group index, 4 * GW bytes per sequence.
-template <int SPL, int DEPTH, bool HAS_W>
-__global__ void __launch_bounds__(kSpmmThreads) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
+// Grid (ceil(nparts / warps per block), bpad / (32 * SPL)).  A warp owns one part of the groups -- at most
+// kPartMaxGroups consecutive groups, one contiguous range of the CSR; the parts hold about the same number of
+// stored pairs, so all warps of the (single) wave finish together -- and a block of 32 * SPL sequences; a lane
+// holds SPL consecutive sequences (one 4-, 16- or 32-byte load per token).  The range is walked in batches of
+// DEPTH tokens with two register buffers: the loads of batch i+1 are issued before batch i is added, so a warp
+// keeps up to 2 * DEPTH lines of Dt in flight at all times.  Token ids are fetched 32 at a time, one block of 32
+// ahead.  Sums run in CSR order; a group ends where the running entry index reaches the next group pointer.
+// Output by group (verification): a closed group's SPL sums go straight to Rt[g, sequences], their positive
+// parts are added up per part and written to Psum[part, sequences].  ROWMAJOR output (pcg_group_probs): the
+// part's sums are turned in shared memory and written along the group index, R[sequence, g].
+template <int SPL, int DEPTH, bool HAS_W, bool ROWMAJOR>
+__global__ void __launch_bounds__(kSpmmThreads, ROWMAJOR ? 4 : 5) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
     pdl_enter();
     constexpr int NS = 32 * SPL;  // sequences per warp
-    const int GW = a.gw;
     constexpr int TS = NS + 4;    // row stride of the result tile (keeps 16-byte alignment, spreads banks)
-    static_assert(32 % DEPTH == 0, "a batch never straddles two blocks of 32 token ids");
-    __shared__ __align__(16) float tiles[(kSpmmThreads / 32) * kSpmmMaxGroupsPerWarp * TS];
+    static_assert(32 % DEPTH == 0 && DEPTH <= 16, "a batch never straddles two blocks of 32 token ids");
+    __shared__ __align__(16) float tiles[ROWMAJOR ? (kSpmmThreads / 32) * kPartMaxGroups * TS : 4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float *tile = tiles + warp * kSpmmMaxGroupsPerWarp * TS;
-    const int g0 = (blockIdx.x * (kSpmmThreads / 32) + warp) * GW;
-    if (g0 >= G.M) return;  // warp-uniform; the kernel has no block-wide barrier
-    const int ng = min(GW, G.M - g0);
-    const float *col = a.Dt + (size_t)blockIdx.y * NS + lane * SPL;
+    float *tile = tiles + (ROWMAJOR ? warp * kPartMaxGroups * TS : 0);
+    const int part = blockIdx.x * (kSpmmThreads / 32) + warp;
+    if (part >= G.nparts) return;  // warp-uniform; the kernel has no block-wide barrier
+    // the part's groups and stored pairs (both pairs of bounds in one round trip, so that the group pointers and
+    // the first token ids can be fetched side by side)
+    const int pp_l = lane < 2 ? G.part_ptr[part + lane] : (lane < 4 ? G.part_ent[part + lane - 2] : 0);
+    const int g0 = __shfl_sync(0xffffffffu, pp_l, 0), ng = __shfl_sync(0xffffffffu, pp_l, 1) - g0;
+    const int e0 = __shfl_sync(0xffffffffu, pp_l, 2), e1 = __shfl_sync(0xffffffffu, pp_l, 3);
+    // this lane's SPL sequences: number sq0 of the chunk, in the 32-sequence batch sq0 / 32 of Dt
+    const int sq0 = blockIdx.y * NS + lane * SPL;
+    const float *col = a.Dt + ((size_t)(sq0 >> 5) * G.V) * 32 + (sq0 & 31);
     const int ptr_l = lane <= ng ? G.group_ptr[g0 + lane] : 0;  // lane i: group_ptr[g0 + i]
-    const int e0 = __shfl_sync(0xffffffffu, ptr_l, 0), e1 = __shfl_sync(0xffffffffu, ptr_l, ng);
     const int nbatch = (e1 - e0 + DEPTH - 1) / DEPTH;
 
     // token ids (and weights) of entries e0 + 32*blk + lane; entries past the end repeat the last one
@@ -1096,21 +1242,26 @@ __global__ void __launch_bounds__(kSpmmThreads) group_spmm_kernel(SpmmArgs a, Gr
 #pragma unroll
         for (int j = 0; j < DEPTH; ++j) {
             const int tok = __shfl_sync(0xffffffffu, src, (off + j) & 31);
-            x[j].load(col + (size_t)tok * a.bpad);  // past the end: a repeat of the last line, never added
+            x[j].load(col + (size_t)tok * 32);  // past the end: a repeat of the last line, never added
         }
     };
-    float acc[SPL];
+    SeqVec<SPL> acc, pos;  // running sums of the open group; sum of the positive parts of the closed ones
 #pragma unroll
-    for (int q = 0; q < SPL; ++q) acc[q] = 0.f;
+    for (int q = 0; q < SPL; ++q) acc.v[q] = pos.v[q] = 0.f;
     int gi = 0;
     int gend = __shfl_sync(0xffffffffu, ptr_l, 1);
     auto close_groups = [&](int k) {  // the entry index reached k: close every group that ends at or before k
         while (gi < ng && gend <= k) {
+            if (ROWMAJOR) {
 #pragma unroll
-            for (int q = 0; q < SPL; ++q) {
-                tile[gi * TS + lane * SPL + q] = acc[q];
-                acc[q] = 0.f;
+                for (int q = 0; q < SPL; ++q) tile[gi * TS + lane * SPL + q] = acc.v[q];
+            } else {
+                acc.store(a.R + (size_t)(g0 + gi) * a.bpad + sq0);
+#pragma unroll
+                for (int q = 0; q < SPL; ++q) pos.v[q] += fmaxf(acc.v[q], 0.f);  // (P - Q)_+ ; NaN counts as 0
             }
+#pragma unroll
+            for (int q = 0; q < SPL; ++q) acc.v[q] = 0.f;
             ++gi;
             gend = __shfl_sync(0xffffffffu, ptr_l, min(gi + 1, 31));
         }
@@ -1125,16 +1276,31 @@ __global__ void __launch_bounds__(kSpmmThreads) group_spmm_kernel(SpmmArgs a, Gr
             load_ids(blk_cur + 1, ids_nxt, w_nxt);
         }
         const int n = min(DEPTH, e1 - e0 - off);
+        if (n == DEPTH && gend > e0 + off + DEPTH) {
+            // a whole batch inside one group (most batches): plain adds, in the same order
+#pragma unroll
+            for (int j = 0; j < DEPTH; ++j) {
+                if (HAS_W) {
+                    const float w = __shfl_sync(0xffffffffu, w_cur, (off + j) & 31);
+#pragma unroll
+                    for (int q = 0; q < SPL; ++q) acc.v[q] += __fmul_rn(x[j].v[q], w);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < SPL; ++q) acc.v[q] += x[j].v[q];
+                }
+            }
+            return;
+        }
 #pragma unroll
         for (int j = 0; j < DEPTH; ++j) {
             if (j < n) {
                 if (HAS_W) {
                     const float w = __shfl_sync(0xffffffffu, w_cur, (off + j) & 31);
 #pragma unroll
-                    for (int q = 0; q < SPL; ++q) acc[q] += __fmul_rn(x[j].v[q], w);
+                    for (int q = 0; q < SPL; ++q) acc.v[q] += __fmul_rn(x[j].v[q], w);
                 } else {
 #pragma unroll
-                    for (int q = 0; q < SPL; ++q) acc[q] += x[j].v[q];
+                    for (int q = 0; q < SPL; ++q) acc.v[q] += x[j].v[q];
                 }
                 close_groups(e0 + off + j + 1);
             }
@@ -1150,54 +1316,40 @@ __global__ void __launch_bounds__(kSpmmThreads) group_spmm_kernel(SpmmArgs a, Gr
         if (i + 1 < nbatch) consume(i + 1, xb);
     }
     close_groups(e1);  // trailing empty groups (gi reaches ng)
-    __syncwarp();
-    const int bbase = a.b0 + blockIdx.y * NS;
-    for (int i = lane; i < NS * GW; i += 32) {  // GW consecutive lanes: the GW groups of one sequence
-        const int sq = i / GW, t = i - sq * GW;
-        if (bbase + sq < a.B && t < ng) a.R[(size_t)(bbase + sq) * G.M + g0 + t] = tile[t * TS + sq];
+    if (ROWMAJOR) {
+        __syncwarp();
+        const int bbase = a.b0 + blockIdx.y * NS;
+        for (int i = lane; i < NS * ng; i += 32) {  // ng consecutive lanes: the part's groups of one sequence
+            const int sq = i / ng, t = i - sq * ng;
+            if (bbase + sq < a.B) a.R[(size_t)(bbase + sq) * G.M + g0 + t] = tile[t * TS + sq];
+        }
+    } else {
+        pos.store(a.Psum + (size_t)part * a.bpad + sq0);
     }
 }
 
-struct DrawArgs {
-    const void *target;
-    const int32_t *draft_tokens;
-    const float *uniforms;
-    int K;
-    float s;
-    const int32_t *labels;
-    const int32_t *term_n;
-    const int32_t *term_flags;
-    const float4 *term_stats;
-    float *R;          // default mode: [B, M] residual sums (clamped in place when the masses are staged in global memory)
-    float *own_rows;   // dense mode with M too large for shared memory: [B, M] staging rows, else null
-    int own_in_smem;   // 1: the M clamped masses of a sequence are staged in shared memory, 0: in global memory
-    const float *Pws;  // dense mode: [B*(K+1), M] target group masses
-    const float *Qws;  // dense mode: [B*K, M] draft group masses
-    int32_t *out_accept_len;
-    int32_t *out_tokens;
-    int32_t *out_groups;  // may be null
-    int32_t *out_flags;   // may be null
-    float *spent;         // scratch no kernel will read again (the transposed operand), or null
-    size_t spent_lines;   // its size in 128-byte lines
-};
-
-__device__ __forceinline__ int own_slot(int j) { return j + (j >> 5); }  // one pad word per 32: chunked reads spread over banks
-
-// Token inside group g by ONE WARP: inverse CDF with u_token over p(t) w_{g,t} in the group's CSR order (the
+// Token inside a group (stored pairs [lo, lo + len)) by ONE WARP: inverse CDF with u_token over p(t) w_{g,t} in the group's CSR order (the
 // target-conditional; the common factor 1/Z cancels, and only ratios inside the group matter, so the terms are
 // taken relative to the group's largest logit).  Sums in double by chunked warp scans.  Returns -1 if no term is
 // positive (non-finite inputs).
 template <typename T>
-__device__ __forceinline__ int warp_token_in_group(const GroupsDev &G, const T *trow, int g, float s, float u_token,
+__device__ __forceinline__ int warp_token_in_range(const GroupsDev &G, const T *trow, int lo, int len, float s, float u_token,
                                                    int lane) {
-    const int lo = G.group_ptr[g], len = G.group_ptr[g + 1] - lo;
-    float mloc = kNegInf;
-    for (int k = lane; k < len; k += 32) mloc = fmaxf(mloc, Elem<T>::widen(trow[G.group_tok[lo + k]]));
+    // this lane's entry of the first 32 (most groups have no more) stays in registers: token, logit, weight
+    const int t0 = lane < len ? G.group_tok[lo + lane] : 0;
+    float l0 = kNegInf, w0 = 0.f;
+    if (lane < len) {
+        l0 = Elem<T>::widen(trow[t0]);
+        w0 = G.pair_w ? G.pair_w[lo + lane] : G.inv_deg[t0];
+    }
+    float mloc = l0;
+    for (int k = lane + 32; k < len; k += 32) mloc = fmaxf(mloc, Elem<T>::widen(trow[G.group_tok[lo + k]]));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, o));
     const float rs = mloc > kNegInf ? mloc * s : 0.f;
     auto omega = [&](int k) -> float {
         if (k >= len) return 0.f;
+        if (k == lane) return __fmul_rn(ex2(__fmaf_rn(l0, s, -rs)), w0);
         const int t = G.group_tok[lo + k];
         const float w = G.pair_w ? G.pair_w[lo + k] : G.inv_deg[t];
         return __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs)), w);
@@ -1225,7 +1377,15 @@ __device__ __forceinline__ int warp_token_in_group(const GroupsDev &G, const T *
         carry += __shfl_sync(0xffffffffu, inc, 31);
     }
     const int ksel = pick >= 0 ? pick : last;  // rounding left no prefix above the target: last token with mass
-    return ksel >= 0 ? G.group_tok[lo + ksel] : -1;
+    if (ksel < 0) return -1;
+    return ksel < 32 ? __shfl_sync(0xffffffffu, t0, ksel) : G.group_tok[lo + ksel];
+}
+
+template <typename T>
+__device__ __forceinline__ int warp_token_in_group(const GroupsDev &G, const T *trow, int g, float s, float u_token,
+                                                   int lane) {
+    const int lo = G.group_ptr[g];
+    return warp_token_in_range<T>(G, trow, lo, G.group_ptr[g + 1] - lo, s, u_token, lane);
 }
 
 // The same from inside a block-wide code path: warp 0 draws, everybody gets the token (ibox: shared ints).
@@ -1269,37 +1429,275 @@ __device__ __forceinline__ void emit_sequence(const GroupsDev &G, int b, int K, 
     }
 }
 
-// One block per sequence.  Shared memory: the M clamped residual masses (padded), then scratch.
-template <typename T, bool DENSE>
+struct PickArgs {
+    const void *target;
+    const int32_t *draft_tokens;
+    const float *uniforms;
+    int K;
+    float s;
+    const int32_t *labels;
+    const int32_t *term_n;
+    const int32_t *term_flags;
+    const float4 *term_stats;
+    const float *Rt;    // [chunks][M, chunk] group sums of every chunk of sequences
+    const float *Psum;  // [chunks][nparts, chunk] per part, the sum of the positive parts of its groups' sums
+    int chunk;          // sequences per chunk
+    int32_t *out_accept_len;
+    int32_t *out_tokens;
+    int32_t *out_groups;  // may be null
+    int32_t *out_flags;   // may be null
+    float *spent;         // scratch no kernel will read again (the transposed operand), or null
+    size_t spent_lines;   // its size in 128-byte lines
+};
+
+// Group draw from the target's own coarse masses, formed straight from the row (nothing stored): the rare path
+// taken when a rejection's residual summed to zero.  Every thread owns a contiguous run of groups; masses are
+// formed twice (for the sums, then by the one thread whose run contains the draw).  Returns the group, or -1 if
+// no group has mass (non-finite inputs).
+template <typename T, int NT>
+__device__ __noinline__ int slow_target_group_draw(const GroupsDev &G, const T *trow, float s, float rs, float u_group,
+                                                   double *dscratch, int *ibox) {
+    const int M = G.M, tid = threadIdx.x;
+    const int per = (M + NT - 1) / NT;
+    const int i0 = min(M, tid * per), i1 = min(M, i0 + per);
+    auto mass = [&](int g) -> float {
+        float acc = 0.f;
+        for (int k = G.group_ptr[g]; k < G.group_ptr[g + 1]; ++k) {
+            const int t = G.group_tok[k];
+            const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
+            acc += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs)), w);
+        }
+        return fmaxf(acc, 0.f);
+    };
+    double my_sum = 0.0;
+    int my_last = -1;
+    for (int g = i0; g < i1; ++g) {
+        const float v = mass(g);
+        my_sum += (double)v;
+        if (v > 0.f) my_last = g;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        ibox[2] = NT;
+        ibox[3] = -1;
+        ibox[4] = -1;
+    }
+    double excl, incl, Ztot;
+    block_scan<NT>(my_sum, dscratch, &excl, &incl, &Ztot);  // (its barriers publish the boxes)
+    if (!(Ztot > 0.0)) return -1;
+    const double target = (double)u_group * Ztot;
+    if (my_last >= 0) atomicMax(&ibox[3], my_last);
+    if (my_sum > 0.0 && incl > target) atomicMin(&ibox[2], tid);
+    __syncthreads();
+    if (ibox[2] == tid) {
+        double loc = 0.0;
+        int pick = my_last;
+        for (int g = i0; g < i1; ++g) {
+            loc += (double)mass(g);
+            if (excl + loc > target) {
+                pick = g;
+                break;
+            }
+        }
+        ibox[4] = pick;
+    }
+    __syncthreads();
+    return ibox[4] >= 0 ? ibox[4] : ibox[3];
+}
+
+// One block per sequence.  The cumulative distribution over the groups is walked in two levels: the parts' sums
+// (a contiguous run of parts per thread, held in registers; prefix sums in double, block scan), then the groups
+// of the one part in which the cumulative mass passes u * Z, by the warp of the thread that owns that part, which
+// goes on to draw the token inside the group.
+template <typename T>
+__global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a, GroupsDev G) {
+    constexpr int NT = kPickThreads, PER = 16;  // PER: part sums a thread keeps in registers
+    __shared__ double dscratch[32];
+    __shared__ int ibox[8];
+    const int M = G.M, V = G.V, K = a.K, NP = G.nparts;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // inputs of the call (not results of the kernels before): fetched before those are waited for
+    const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
+    const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
+    pdl_enter();
+    const int n = a.term_n[b];
+    int flags = a.term_flags[b];
+    const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
+    const bool residual = n < K;  // false: draw from the target's coarse distribution itself (bonus token)
+    const int c = b / a.chunk, colb = b - c * a.chunk;
+    const size_t cs = (size_t)a.chunk;
+    const float *Rt = a.Rt + (size_t)c * M * cs + colb;    // group g of this sequence: Rt[g * chunk]
+    const float *Ps = a.Psum + (size_t)c * NP * cs + colb;  // part p of this sequence: Ps[p * chunk]
+
+    const int per = (NP + NT - 1) / NT;
+    const int p0 = min(NP, tid * per), p1 = min(NP, p0 + per);
+    if (tid == 0) {
+        ibox[2] = NT;  // selected thread (minimum)
+        ibox[3] = -1;  // last part with mass (maximum)
+        ibox[4] = -1;  // drawn group
+        ibox[5] = -1;  // drawn token
+    }
+    float v[PER];  // the first PER part sums of this thread's run (all of it unless there are very many parts)
+#pragma unroll
+    for (int j = 0; j < PER; ++j) v[j] = p0 + j < p1 ? Ps[(size_t)(p0 + j) * cs] : 0.f;
+    double my_sum = 0.0;
+    int my_last = -1;  // last part with mass in this thread's run
+#pragma unroll
+    for (int j = 0; j < PER; ++j) {
+        my_sum += (double)v[j];
+        if (v[j] > 0.f) my_last = p0 + j;
+    }
+    for (int p = p0 + PER; p < p1; ++p) {
+        const float x = Ps[(size_t)p * cs];
+        my_sum += (double)x;
+        if (x > 0.f) my_last = p;
+    }
+    double my_excl, my_incl, Ztot;
+    block_scan<NT>(my_sum, dscratch, &my_excl, &my_incl, &Ztot);  // (its barriers publish the boxes)
+
+    int gsel = -1, z = -1;
+    if (Ztot > 0.0) {
+        // ---- group draw: first group whose inclusive prefix exceeds u * Z ----
+        const double target = (double)u_group * Ztot;
+        if (my_last >= 0) atomicMax(&ibox[3], my_last);
+        if (my_sum > 0.0 && my_incl > target) atomicMin(&ibox[2], tid);
+        __syncthreads();
+        const bool none = ibox[2] == NT;  // rounding left no thread's prefix above the target
+        const int owner = none ? 0 : ibox[2];
+        if (warp == (owner >> 5)) {
+            // the part: the first of the owner's run whose prefix passes the target; if rounding left none, the
+            // last part with mass (of the run, or of all parts)
+            int part = ibox[3];
+            int found = 0;
+            double run = my_excl;
+            if (tid == owner && !none) {
+                part = my_last;
+#pragma unroll
+                for (int j = 0; j < PER; ++j) {
+                    if (!found) {
+                        if (v[j] > 0.f && run + (double)v[j] > target) {
+                            part = p0 + j;
+                            found = 1;
+                        } else {
+                            run += (double)v[j];
+                        }
+                    }
+                }
+                for (int p = p0 + PER; p < p1 && !found; ++p) {
+                    const float x = Ps[(size_t)p * cs];
+                    if (x > 0.f && run + (double)x > target) {
+                        part = p;
+                        found = 1;
+                    } else {
+                        run += (double)x;
+                    }
+                }
+            }
+            part = __shfl_sync(0xffffffffu, part, owner & 31);
+            found = __shfl_sync(0xffffffffu, found, owner & 31);
+            run = __shfl_sync(0xffffffffu, run, owner & 31);
+            if (part >= 0) {
+                // the group inside it (lane j holds group j of the part): the running sum continues from the parts
+                // before; if no prefix passes the target (rounding), the last group with mass
+                const int g0 = G.part_ptr[part], ng = G.part_ptr[part + 1] - g0;  // at most kPartMaxGroups
+                const float r = lane < ng ? fmaxf(Rt[(size_t)(g0 + lane) * cs], 0.f) : 0.f;
+                const int gp = lane <= ng ? G.group_ptr[g0 + lane] : 0;
+                int pick = -1, last = -1;
+                for (int j = 0; j < ng; ++j) {
+                    const float rj = __shfl_sync(0xffffffffu, r, j);
+                    if (rj > 0.f) last = j;
+                    if (found && pick < 0) {
+                        run += (double)rj;
+                        if (rj > 0.f && run > target) pick = j;
+                    }
+                }
+                const int j = pick >= 0 ? pick : last;
+                if (j >= 0) {
+                    const int lo = __shfl_sync(0xffffffffu, gp, j), hi = __shfl_sync(0xffffffffu, gp, j + 1);
+                    const int zt = warp_token_in_range<T>(G, trow, lo, hi - lo, a.s, u_token, lane);
+                    if (lane == 0) {
+                        ibox[4] = g0 + j;
+                        ibox[5] = zt;
+                        ibox[6] = hi > lo ? G.group_tok[lo] : 0;  // stand-in if the group has no token with mass
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        gsel = ibox[4];
+        z = ibox[5];
+        if (gsel >= 0 && z < 0) {  // the drawn group has no token with target mass (non-finite inputs)
+            flags |= PCG_FLAG_NONFINITE;
+            z = ibox[6];
+        }
+    } else if (residual) {
+        // a rejection whose residual vanished (P == Q to rounding): draw from P instead
+        flags |= PCG_FLAG_ZERO_RESIDUAL;
+        gsel = slow_target_group_draw<T, NT>(G, trow, a.s, a.term_stats[b].x, u_group, dscratch, ibox);
+        if (gsel >= 0) z = block_token_in_group<T>(G, trow, gsel, a.s, u_token, ibox, flags);
+    }
+    if (gsel < 0) {  // no mass anywhere (non-finite inputs): emit group 0 / token 0 and flag it
+        gsel = 0;
+        z = 0;
+        flags |= PCG_FLAG_NONFINITE;
+    }
+    emit_sequence<NT>(G, b, K, n, z, gsel, flags, a.draft_tokens, a.labels, a.out_accept_len, a.out_tokens, a.out_groups,
+                      a.out_flags);
+    // The transposed operand has been consumed (workspace contents are of no interest after the call):
+    // dropping its dirty lines from L2 spares the write-back that would otherwise compete with the next call's
+    // streaming reads.  Last, so that it does not delay the draw.
+    if (a.spent)
+        for (size_t l = (size_t)b * NT + tid; l < a.spent_lines; l += (size_t)gridDim.x * NT)
+            asm volatile("discard.global.L2 [%0], 128;" ::"l"(a.spent + l * 32) : "memory");
+}
+
+struct DrawArgs {
+    const void *target;
+    const int32_t *draft_tokens;
+    const float *uniforms;
+    int K;
+    float s;
+    const int32_t *labels;
+    const int32_t *term_n;
+    const int32_t *term_flags;
+    float *own_rows;   // M too large for shared memory: [B, M] staging rows, else null
+    int own_in_smem;   // 1: the M clamped masses of a sequence are staged in shared memory, 0: in global memory
+    const float *Pws;  // [B*(K+1), M] target group masses
+    const float *Qws;  // [B*K, M] draft group masses
+    int32_t *out_accept_len;
+    int32_t *out_tokens;
+    int32_t *out_groups;  // may be null
+    int32_t *out_flags;   // may be null
+};
+
+__device__ __forceinline__ int own_slot(int j) { return j + (j >> 5); }  // one pad word per 32: chunked reads spread over banks
+
+// Dense mode: terminal draw from the stored group masses of every position.  One block per sequence.  Shared
+// memory: the M clamped residual masses (padded), then scratch.
+template <typename T>
 __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a, GroupsDev G) {
     pdl_enter();
     constexpr int NT = kDrawThreads;
     extern __shared__ __align__(16) unsigned char raw[];
     const int M = G.M, V = G.V, K = a.K;
     const int b = blockIdx.x, tid = threadIdx.x;
-    // The M clamped masses of the sequence: in (padded) shared memory when they fit, else in a row of global memory
-    // (the sequence's own row of R, or a staging row in dense mode); `slot` maps a group to its place.
+    // The M clamped masses of the sequence: in (padded) shared memory when they fit, else in a row of global memory;
+    // `slot` maps a group to its place.
     const bool in_smem = a.own_in_smem;
-    float *own = in_smem ? reinterpret_cast<float *>(raw) : (DENSE ? a.own_rows : a.R) + (size_t)b * M;
+    float *own = in_smem ? reinterpret_cast<float *>(raw) : a.own_rows + (size_t)b * M;
     auto slot = [&](int j) { return in_smem ? own_slot(j) : j; };
     unsigned char *tail = raw + (in_smem ? (((size_t)own_slot(M) + 1) * 4 + 15) / 16 * 16 : 0);
     double *dscratch = reinterpret_cast<double *>(tail);      // 32 doubles
     float *scratch = reinterpret_cast<float *>(dscratch + 32);  // 64 floats
     int *ibox = reinterpret_cast<int *>(scratch + 64);          // 8 ints
-    // The transposed operand has been consumed (workspace contents are of no interest after the call):
-    // dropping its dirty lines from L2 spares the write-back that would otherwise compete with the next call's
-    // streaming reads (measured: the next position kernel runs 4 % faster).
-    if (a.spent)
-        for (size_t l = (size_t)b * NT + tid; l < a.spent_lines; l += (size_t)gridDim.x * NT)
-            asm volatile("discard.global.L2 [%0], 128;" ::"l"(a.spent + l * 32) : "memory");
     const int n = a.term_n[b];
     int flags = a.term_flags[b];
     const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
     const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
     const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
     bool residual = n < K;  // false: draw from the target's coarse distribution itself (bonus token)
-    const float *Pn = DENSE ? a.Pws + ((size_t)b * (K + 1) + n) * M : nullptr;
-    const float *Qn = DENSE ? a.Qws + ((size_t)b * K + min(n, K - 1)) * M : nullptr;
+    const float *Pn = a.Pws + ((size_t)b * (K + 1) + n) * M;
+    const float *Qn = a.Qws + ((size_t)b * K + min(n, K - 1)) * M;
 
     const int per = (M + NT - 1) / NT;
     const int i0 = min(M, tid * per), i1 = min(M, i0 + per);
@@ -1311,35 +1709,8 @@ __global__ void __launch_bounds__(kDrawThreads) terminal_draw_kernel(DrawArgs a,
         ibox[4] = -1;  // drawn group
     }
     for (int attempt = 0; attempt < 2; ++attempt) {
-        if (DENSE) {
-            for (int g = tid; g < M; g += NT)
-                own[slot(g)] = fmaxf(residual ? Pn[g] - Qn[g] : Pn[g], 0.f);  // (P - Q)_+ ; NaN becomes 0
-        } else if (attempt == 0) {
-            // R holds sum_t (p - q)/N for a rejection and sum_t p/N for the bonus row
-            const float *Rb = a.R + (size_t)b * M;  // (with global staging this is `own` itself: clamped in place)
-            // sixteen loads in flight per thread before the first is used (one at a time, this loop was 10 of
-            // the kernel's 23 microseconds)
-            for (int g0 = tid; g0 < M; g0 += 16 * NT) {
-                float v[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = g0 + j * NT < M ? Rb[g0 + j * NT] : 0.f;
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    if (g0 + j * NT < M) own[slot(g0 + j * NT)] = fmaxf(v[j], 0.f);
-            }
-        } else {
-            // slow path of the zero-residual fallback: the target masses straight from the row
-            const float rs = a.term_stats[b].x;
-            for (int g = tid; g < M; g += NT) {
-                float acc = 0.f;
-                for (int k = G.group_ptr[g]; k < G.group_ptr[g + 1]; ++k) {
-                    const int t = G.group_tok[k];
-                    const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
-                    acc += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -rs)), w);
-                }
-                own[slot(g)] = fmaxf(acc, 0.f);
-            }
-        }
+        for (int g = tid; g < M; g += NT)
+            own[slot(g)] = fmaxf(residual ? Pn[g] - Qn[g] : Pn[g], 0.f);  // (P - Q)_+ ; NaN becomes 0
         __syncthreads();
         // ---- prefix sums over the groups (double): a contiguous chunk per thread, then a block scan ----
         my_sum = 0.0;
@@ -1486,10 +1857,7 @@ static cudaError_t launch_cluster(Kern kern, int blocks, int cluster, size_t sme
     return cudaLaunchKernelEx(&cfg, kern, args, G);
 }
 
-#ifndef PCG_DT_BUDGET_MB
-#define PCG_DT_BUDGET_MB 64
-#endif
-constexpr size_t kDtBudgetBytes = (size_t)PCG_DT_BUDGET_MB << 20;  // Dt of one chunk of sequences must stay inside the L2
+constexpr size_t kDtBudgetBytes = (size_t)64 << 20;  // Dt of one chunk of sequences must stay inside the L2
 
 // Sequences per lane of the sparse product: 8 (one 256-bit load per token and lane) from 256 sequences on if
 // that many fit the budget of the transposed operand, kSpmmWide (4) from 128 on, else 1.
@@ -1505,17 +1873,17 @@ static int terminal_chunk(int B, int V) {
     const int64_t bpad = ((int64_t)B + unit - 1) / unit * unit;
     int64_t fit = (int64_t)(kDtBudgetBytes / ((size_t)V * 4)) / unit * unit;
     if (fit < unit) fit = unit;
-    return (int)(fit < bpad ? fit : bpad);
+    return (int)std::max<int64_t>(unit, fit < bpad ? fit : bpad);
 }
 
 static size_t draw_smem_bytes(int M) { return (((size_t)M + (size_t)(M >> 5) + 1) * 4 + 15) / 16 * 16 + 32 * 8 + 64 * 4 + 8 * 4; }
 
 struct VerifyWorkspace {
-    int32_t *accept, *labels, *posflags, *term_n, *term_flags;
-    float4 *stats, *term_stats;
-    float *Dt, *R;     // default mode
-    float *Pws, *Qws;  // dense mode
-    float *own_rows;   // dense mode, M beyond the draw kernel's shared memory
+    int32_t *accept, *labels, *posflags, *term_n, *term_flags, *bonus_flags;
+    float4 *stats, *term_stats, *bonus_stats;
+    float *Dt, *Rt, *Psum;  // default mode
+    float *Pws, *Qws;       // dense mode
+    float *own_rows;        // dense mode, M beyond the draw kernel's shared memory
     size_t bytes;
 };
 
@@ -1541,66 +1909,41 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
         w.Qws = (float *)(p + take((size_t)(B * K * M) * 4));
         if (draw_smem_bytes((int)M) > kMaxDynSmem) w.own_rows = (float *)(p + take((size_t)(B * M) * 4));
     } else if (mode != PCG_VERIFY_CLUSTER_TERMINAL) {
-        w.Dt = (float *)(p + take((size_t)V * (size_t)terminal_chunk((int)B, (int)V) * 4));
-        w.R = (float *)(p + take((size_t)(B * M) * 4));
+        const int64_t chunk = terminal_chunk((int)B, (int)V);
+        const int64_t chunks = (B + chunk - 1) / chunk;
+        w.bonus_stats = (float4 *)(p + take((size_t)B * 16));
+        w.bonus_flags = (int32_t *)(p + take((size_t)B * 4));
+        w.Dt = (float *)(p + take((size_t)V * (size_t)chunk * 4));
+        w.Rt = (float *)(p + take((size_t)(chunks * chunk * M) * 4));
+        w.Psum = (float *)(p + take((size_t)(chunks * chunk * M) * 4));  // (a part holds at least one group)
     }
     w.bytes = off ? off : 256;
     return w;
 }
 
-// Groups per warp for a launch of `warps_y` warp rows over M groups.  All warps take about the same time, so a
-// launch of 1.7 waves costs two: with few waves the groups per warp are chosen to fill whole waves (C5: 7 groups
-// per warp = 586 blocks on 592 resident ones, instead of 4 = 1024 blocks = 1.73 waves); with many waves the
-// measured best, kSpmmGroupsPerWarp.
-static int spmm_groups_per_warp(int M, int64_t warps_y, int64_t resident_blocks) {
-    const int wpb = kSpmmThreads / 32;
-    auto waves = [&](int gw) {
-        const int64_t blocks = ((M + gw - 1) / gw + wpb - 1) / wpb * warps_y;
-        return (blocks + resident_blocks - 1) / resident_blocks;
-    };
-    if (waves(kSpmmGroupsPerWarp) > 4) return kSpmmGroupsPerWarp;  // many waves: the tail no longer matters
-    int best = kSpmmGroupsPerWarp;
-    int64_t best_cost = waves(best) * best;  // time ~ waves x work per warp
-    for (int gw = kSpmmMaxGroupsPerWarp; gw >= 2; --gw)
-        if (waves(gw) * gw < best_cost) {
-            best = gw;
-            best_cost = waves(gw) * gw;
-        }
-    return best;
+// The transposed-operand kernel over nb batches of 32 sequences: about three resident blocks per SM, shared out
+// over the batches, each walking a run of its batch's rows.
+template <typename T>
+static cudaError_t launch_transpose(const TransposeArgs &tr, int nb, const GroupsDev &G, int sm_count, cudaStream_t cs) {
+    constexpr int ch = 32 / (int)sizeof(T);  // tokens per step of a lane
+    const int nsteps = (G.V + ch - 1) / ch;
+    // a block's run: at least 8 steps per warp, so that finding the terminal positions is paid for
+    const int per_batch = std::max(1, std::min((nsteps + 63) / 64, 3 * sm_count / std::max(nb, 1)));
+    const dim3 grid((unsigned)per_batch, (unsigned)nb);
+    return launch_after(residual_transpose_kernel<T>, grid, dim3(kTrThreads), 0, cs, tr, G);
 }
 
-// The sparse product over nb blocks of 32 sequences (nb a multiple of `lanes`, the sequences per lane: 8, 4 or 1).
-static void launch_spmm(SpmmArgs sp, int nb, int lanes, const GroupsDev &G, int sm_count, cudaStream_t cs) {
+// The sparse product over nb batches of 32 sequences (nb a multiple of `lanes`, the sequences per lane: 8, 4 or 1).
+template <bool ROWMAJOR>
+static cudaError_t launch_spmm(const SpmmArgs &sp, int nb, int lanes, const GroupsDev &G, cudaStream_t cs) {
     const bool has_w = G.pair_w != nullptr;
-    auto go = [&](auto kern, int slot) {
-        static std::atomic<int> occupancy[6];  // resident blocks per SM of each variant (0 = not asked yet)
-        int occ = occupancy[slot].load(std::memory_order_relaxed);
-        if (occ == 0) {
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kSpmmThreads, 0) != cudaSuccess || occ < 1) occ = 4;
-            occupancy[slot].store(occ, std::memory_order_relaxed);
-        }
-        const int64_t wy = nb / lanes;
-        sp.gw = spmm_groups_per_warp(G.M, wy, (int64_t)occ * sm_count);
-        const int gpb = sp.gw * (kSpmmThreads / 32);  // groups per block
-        const dim3 grid((unsigned)((G.M + gpb - 1) / gpb), (unsigned)wy);
-        launch_after(kern, grid, dim3(kSpmmThreads), 0, cs, sp, G);
-    };
-    if (lanes == 8) {
-        if (has_w)
-            go(group_spmm_kernel<8, 4, true>, 0);
-        else
-            go(group_spmm_kernel<8, 4, false>, 1);
-    } else if (lanes == kSpmmWide) {
-        if (has_w)
-            go(group_spmm_kernel<kSpmmWide, kSpmmDepth, true>, 2);
-        else
-            go(group_spmm_kernel<kSpmmWide, kSpmmDepth, false>, 3);
-    } else {
-        if (has_w)
-            go(group_spmm_kernel<1, 16, true>, 4);
-        else
-            go(group_spmm_kernel<1, 16, false>, 5);
-    }
+    const dim3 grid((unsigned)((G.nparts + kSpmmThreads / 32 - 1) / (kSpmmThreads / 32)), (unsigned)(nb / lanes));
+    auto go = [&](auto kern) { return launch_after(kern, grid, dim3(kSpmmThreads), 0, cs, sp, G); };
+    if (lanes == 8) return has_w ? go(group_spmm_kernel<8, 4, true, ROWMAJOR>) : go(group_spmm_kernel<8, 4, false, ROWMAJOR>);
+    if (lanes == kSpmmWide)
+        return has_w ? go(group_spmm_kernel<kSpmmWide, kSpmmDepth, true, ROWMAJOR>)
+                     : go(group_spmm_kernel<kSpmmWide, kSpmmDepth, false, ROWMAJOR>);
+    return has_w ? go(group_spmm_kernel<1, 16, true, ROWMAJOR>) : go(group_spmm_kernel<1, 16, false, ROWMAJOR>);
 }
 
 #include "pcg_thinning.cuh"
@@ -1630,19 +1973,25 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
         // many rows: the same transposed-operand / sparse-product kernels as the per-sequence stage of pcg_verify,
         // a chunk of rows at a time through the handle's scratch (row statistics, then p(t) w in place of p - q)
         const int chunk = groups->probs_chunk;  // a multiple of 128
-        const int tt = 32 * (int)(16 / dtype_bytes(dtype));
         for (int64_t r0 = 0; r0 < rows; r0 += chunk) {
             const int nr = (int)std::min<int64_t>(chunk, rows - r0);
             const char *base = (const char *)logits + (size_t)r0 * G.V * dtype_bytes(dtype);
             PCG_DISPATCH_DTYPE(dtype, launch_after(row_stats_kernel<LogitT>, dim3((unsigned)nr), dim3(kPrepThreads), 0, cs,
                                                    (const void *)base, s, groups->probs_stats, G));
             const int lanes = (chunk % 256 == 0 && nr >= 256) ? 8 : kSpmmWide;      // rows per lane of the sparse product
-            const int nb = (nr + 32 * lanes - 1) / (32 * lanes) * lanes;          // blocks of 32 rows, whole warps of it
+            const int nb = (nr + 32 * lanes - 1) / (32 * lanes) * lanes;          // batches of 32 rows, whole warps of it
             // every row is "a sequence whose only row is accepted": K = 0 makes the kernel form p alone
-            TransposeArgs tr{base, base, nr, 0, 0, chunk, s, groups->probs_zero, groups->probs_stats, groups->probs_dt};
-            const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
-            PCG_DISPATCH_DTYPE(dtype, launch_after(residual_transpose_kernel<LogitT>, tgrid, dim3(kTrThreads), 0, cs, tr, G));
-            launch_spmm(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M, 0}, nb, lanes, G, groups->sm_count, cs);
+            TransposeArgs tr{};
+            tr.target = tr.draft = base;
+            tr.B = nr;
+            tr.s = s;
+            tr.term_n = groups->probs_zero;
+            tr.term_stats = groups->probs_stats;
+            tr.Dt = groups->probs_dt;
+            PCG_DISPATCH_DTYPE(dtype, e = launch_transpose<LogitT>(tr, nb, G, groups->sm_count, cs));
+            if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
+            e = launch_spmm<true>(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M, nullptr}, nb, lanes, G, cs);
+            if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
         }
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching the batched group-probability kernels");
@@ -1735,8 +2084,10 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching dense_accept_kernel");
     } else {
+        // (the batched per-sequence stage takes the bonus row's statistics from this kernel)
         PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
-                        w.accept,      w.labels,     w.posflags,   w.stats,  nullptr};
+                        w.accept,      w.labels,     w.posflags,   w.stats,  nullptr,
+                        cluster_terminal ? nullptr : w.bonus_stats, cluster_terminal ? nullptr : w.bonus_flags};
         PCG_DISPATCH_DTYPE(dtype, position_kernel<LogitT><<<B * K, kPosThreads, 0, cs>>>(pa, G));
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
@@ -1753,42 +2104,42 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         PCG_DISPATCH_DTYPE(dtype, e = launch_cluster(terminal_kernel<LogitT>, B * G.slices, G.slices,
                                                      groups->agg_smem_bytes, cs, ta, G));
         if (e != cudaSuccess) return cuda_fail(e, "launching terminal_kernel");
-    } else {
-        PrepareArgs pr{target_logits, K, s, dense ? 0 : 1, w.accept, w.posflags, w.stats, w.term_n, w.term_flags, w.term_stats};
+    } else if (dense) {
+        PrepareArgs pr{target_logits, K, s, 0, w.accept, w.posflags, w.stats, w.term_n, w.term_flags, w.term_stats};
         PCG_DISPATCH_DTYPE(dtype, launch_after(terminal_prepare_kernel<LogitT>, dim3((unsigned)B), dim3(kPrepThreads), 0, cs, pr, G));
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching terminal_prepare_kernel");
-        if (!dense) {
-            const int chunk = terminal_chunk(B, G.V);
-            const int tt = 32 * (int)(16 / dtype_bytes(dtype));
-            const int lanes = spmm_lanes(B, G.V);  // sequences per lane in the sparse product
-            for (int b0 = 0; b0 < B; b0 += chunk) {
-                // blocks of 32 sequences in this chunk, rounded up to what one warp of the sparse product reads
-                const int unit = 32 * lanes;
-                const int nb = (std::min(B - b0, chunk) + unit - 1) / unit * (unit / 32);
-                TransposeArgs tr{target_logits, draft_logits, B, K, b0, chunk, s, w.term_n, w.term_stats, w.Dt};
-                const dim3 tgrid((unsigned)((G.V + tt - 1) / tt), (unsigned)nb);
-                PCG_DISPATCH_DTYPE(dtype, launch_after(residual_transpose_kernel<LogitT>, tgrid, dim3(kTrThreads), 0, cs, tr, G));
-                e = cudaGetLastError();
-                if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
-                launch_spmm(SpmmArgs{w.Dt, B, b0, chunk, w.R, 0}, nb, lanes, G, groups->sm_count, cs);
-                e = cudaGetLastError();
-                if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
-            }
-        }
-        DrawArgs dr{target_logits, draft_tokens, uniforms, K,     s,     w.labels,       w.term_n,   w.term_flags,
-                    w.term_stats,  w.R,          w.own_rows, own_in_smem ? 1 : 0, w.Pws, w.Qws, out_accept_len, out_tokens,
-                    out_groups,    out_flags,
-                    dense ? nullptr : w.Dt,
-                    dense ? 0 : (size_t)G.V * (size_t)terminal_chunk(B, G.V) * 4 / 128};
+        DrawArgs dr{target_logits, draft_tokens, uniforms, K, s, w.labels, w.term_n, w.term_flags, w.own_rows,
+                    own_in_smem ? 1 : 0, w.Pws, w.Qws, out_accept_len, out_tokens, out_groups, out_flags};
         auto launch_draw = [&](auto kern) -> cudaError_t {
             cudaError_t le = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)draw_smem);
             if (le != cudaSuccess) return le;
             return launch_after(kern, dim3((unsigned)B), dim3(kDrawThreads), draw_smem, cs, dr, G);
         };
-        PCG_DISPATCH_DTYPE(dtype, e = dense ? launch_draw(terminal_draw_kernel<LogitT, true>)
-                                            : launch_draw(terminal_draw_kernel<LogitT, false>));
+        PCG_DISPATCH_DTYPE(dtype, e = launch_draw(terminal_draw_kernel<LogitT>));
         if (e != cudaSuccess) return cuda_fail(e, "launching terminal_draw_kernel");
+    } else {
+        const int chunk = terminal_chunk(B, G.V);
+        const int lanes = spmm_lanes(B, G.V);  // sequences per lane in the sparse product
+        for (int b0 = 0, ci = 0; b0 < B; b0 += chunk, ++ci) {
+            // batches of 32 sequences in this chunk, rounded up to what one warp of the sparse product reads
+            const int unit = 32 * lanes;
+            const int nb = (std::min(B - b0, chunk) + unit - 1) / unit * (unit / 32);
+            TransposeArgs tr{target_logits, draft_logits, B,        K,         b0,          s,           1,
+                             w.accept,      w.posflags,   w.stats,  w.bonus_stats, w.bonus_flags, w.term_n, w.term_flags,
+                             w.term_stats,  w.Dt};
+            PCG_DISPATCH_DTYPE(dtype, e = launch_transpose<LogitT>(tr, nb, G, groups->sm_count, cs));
+            if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
+            e = launch_spmm<false>(SpmmArgs{w.Dt, B, b0, chunk, w.Rt + (size_t)ci * G.M * chunk,
+                                            w.Psum + (size_t)ci * G.nparts * chunk},
+                                   nb, lanes, G, cs);
+            if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
+        }
+        PickArgs pk{target_logits, draft_tokens, uniforms,   K,          s,         w.labels, w.term_n, w.term_flags, w.term_stats,
+                    w.Rt,          w.Psum,       chunk,      out_accept_len, out_tokens, out_groups, out_flags,
+                    w.Dt,          (size_t)G.V * (size_t)chunk * 4 / 128};
+        PCG_DISPATCH_DTYPE(dtype, e = launch_after(terminal_pick_kernel<LogitT>, dim3((unsigned)B), dim3(kPickThreads), 0, cs, pk, G));
+        if (e != cudaSuccess) return cuda_fail(e, "launching terminal_pick_kernel");
     }
     if (stage_events) {
         e = cudaEventRecord((cudaEvent_t)stage_events[2], cs);
@@ -1821,7 +2172,7 @@ static ThinWorkspace carve_thin_workspace(void *base, int64_t B, int64_t K, int6
     w.labels = (int32_t *)(p + take((size_t)(B * K) * 4));
     w.posflags = (int32_t *)(p + take((size_t)(B * K) * 4));
     w.fallback_rows = (float *)(p + take((size_t)(B * M) * 4));
-    w.strata = (float2 *)(p + take((size_t)(B * K) * kHalf * 8));
+    w.strata = (float2 *)(p + take((size_t)(B * K) * kPosThreads * 8));
     w.bytes = off ? off : 256;
     return w;
 }
@@ -1882,7 +2233,7 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
     // (t div W) mod 128), so the thinning kernel needs no pass of its own over the row.
     const bool strata = ((uintptr_t)target_logits & 15u) == 0 && ((size_t)G.V * esz) % 16 == 0;
     PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
-                    w.accept,      w.labels,     w.posflags,   w.stats,  strata ? w.strata : nullptr};
+                    w.accept,      w.labels,     w.posflags,   w.stats,  strata ? w.strata : nullptr, nullptr, nullptr};
     PCG_DISPATCH_DTYPE(dtype, position_kernel<LogitT><<<B * K, kPosThreads, 0, cs>>>(pa, G));
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
