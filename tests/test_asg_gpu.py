@@ -127,3 +127,30 @@ def test_argument_errors():
     with pytest.raises(binding.PcgError) as err:
         binding.Asg(emb, float("nan"))
     assert err.value.status == 1
+
+
+def _clear_threshold_chunked(emb, lo, hi, chunk=1024):
+    """As _clear_threshold for tables too large to hold all cosines: only those inside (lo, hi) are collected."""
+    from oracle import asg_oracle as A
+
+    E = A.widen(emb)
+    n = np.sqrt((E * E).sum(1))
+    En = E / np.maximum(n, 1e-300)[:, None]
+    near = [np.array([lo, hi])]
+    for r0 in range(0, E.shape[0], chunk):
+        cos = En[r0:r0 + chunk] @ En.T
+        near.append(cos[(cos > lo) & (cos < hi)])
+    c = np.sort(np.concatenate(near))
+    k = int(np.argmax(np.diff(c)))
+    assert c[k + 1] - c[k] > 10 * BAND
+    return float(np.float32(0.5 * (c[k] + c[k + 1])))
+
+
+def test_large_table_of_sixteen_thousand_tokens():
+    """V = 16,384 (128 x 64 tiles of the tensor-core kernel, several waves of its persistent blocks), both tensor
+    paths: clusters with duplicated rows and bridge tokens, the threshold in the widest gap of the cosines near 0.6."""
+    rng = np.random.default_rng(16)
+    emb = _clustered(rng, 16384, 96, 700, noise=0.03, bridges=300)
+    emb[5000:5040] = emb[100:140]  # duplicated embeddings: identical neighbourhoods must merge
+    asg, want = _check(emb, _clear_threshold_chunked(emb, 0.58, 0.62))
+    assert want.M < 16384 and want.tok_degree.max() >= 2

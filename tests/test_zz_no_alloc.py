@@ -5,7 +5,8 @@ with its own memory pool, a plug-in inside another application) and cudaMalloc i
 cannot provide the workspace pcg_verify asks for.  pcg_verify_static keeps its scratch inside the library image
 instead.  This test calls it through the C ABI twice in a row, on different inputs, and checks that it returns
 exactly what pcg_verify returns in the same mode -- the second call runs on top of whatever the first left in the
-shared scratch -- and that calls too large for the built-in scratch are refused before anything is launched.
+shared scratch --, that both calls agree with the CPU oracle decision by decision, and that calls too large for
+the built-in scratch are refused before anything is launched.
 This file sorts last so that a failure here cannot hide the result of any other test.
 """
 import numpy as np
@@ -24,8 +25,9 @@ def _device_inputs(bt):
             torch.from_numpy(bt.draft_tokens).cuda(), torch.from_numpy(bt.uniforms).cuda())
 
 
-def test_static_scratch_entry_point_matches_pcg_verify_on_two_calls_in_a_row():
-    from gpu_util import make_handle
+def test_static_scratch_entry_point_matches_pcg_verify_on_two_calls_in_a_row(oracle):
+    from gpu_util import make_handle, run_oracle
+    from oracle.compare import compare_verify
     from paper_2511_13732_b200 import binding
 
     cfg = W.scaled(W.CONFIGS["C3"], B=40, K=6, V=4000, M=900)
@@ -48,6 +50,10 @@ def test_static_scratch_entry_point_matches_pcg_verify_on_two_calls_in_a_row():
         torch.cuda.synchronize()
         for got, ref in zip(out, want):
             assert np.array_equal(got.cpu().numpy(), ref.cpu().numpy())  # integer outputs: bit-exact
+        # and against the oracle itself, not only against the library's other entry point
+        cmp = compare_verify(out[0].cpu().numpy(), out[1].cpu().numpy(), out[2].cpu().numpy(), run_oracle(oracle, bt, groups),
+                             band=1e-6)
+        assert cmp.hard == 0 and cmp.excused == 0, cmp.details[:3]
         assert out[0].min().item() >= 0 and out[0].max().item() <= cfg.K
     assert out[0].max().item() == cfg.K  # the second call did reach bonus-token rows
 
