@@ -32,9 +32,37 @@ from paper_2511_13732_b200 import workloads as W  # noqa: E402
 METRIC = "verified draft positions/sec"
 UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0  # used only when MEASURED_PEAKS.json is absent
-# dram__bytes_read.sum + dram__bytes_write.sum of one position_kernel launch, from the ncu capture summarised in
-# profiles/ (null until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {"C5": 1076131840 + 12466432}
+KERNEL_SOURCES = ("paper_2511_13732_b200/csrc/pcg_kernels.cu", "paper_2511_13732_b200/csrc/pcg_common.cuh")
+
+
+def kernel_source_hash():
+    """sha256 (first 16 hex digits) of the sources of the verification kernels: ties an ncu record to a kernel version."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic_bytes(workload):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one position_kernel launch, from the ncu record kept under
+    profiles/ (lines `workload:`, `kernel_source_hash:`, `dram_bytes_read_per_launch:`, `dram_bytes_write_per_launch:`).
+    None when there is no record for the workload or the kernels have been edited since it was taken."""
+    path = os.path.join(ROOT, "profiles", f"position_kernel_{workload.lower()}_dram_traffic.md")
+    try:
+        fields = {}
+        with open(path) as f:
+            for ln in f:
+                if ":" in ln and not ln.startswith(" "):
+                    k, v = ln.split(":", 1)
+                    fields[k.strip().strip("`")] = v.strip().strip("`")
+        if fields.get("kernel_source_hash") != kernel_source_hash():
+            return None
+        return int(fields["dram_bytes_read_per_launch"]) + int(fields["dram_bytes_write_per_launch"])
+    except (OSError, KeyError, ValueError):
+        return None
 
 
 def hbm_peak():
@@ -134,10 +162,22 @@ def oracle_leg(cfg, groups, batch, min_seconds=2.0, max_passes=200, timed_output
     while passes < max_passes and (spent < min_seconds or passes < 2):
         spent += one_pass(nseq)
         passes += 1
+    evaluated = int((np.minimum(last["ref"].accept_len, cfg.K - 1) + 1).sum())  # positions the oracle really formed
     out = {"value": nseq * cfg.K * passes / spent, "unit": UNIT, "cores": cores, "kind": "oracle",
            "sample": f"first {nseq} of {B} sequences of {cfg.name} ({nseq * cfg.K} drafted positions), {passes} "
                      f"passes, {spent:.3f} s wall on {cores} threads (OpenMP over sequences; the oracle stops a "
-                     f"sequence at its first rejection, as Algorithm 1 does)"}
+                     f"sequence at its first rejection, as Algorithm 1 does: it evaluates {evaluated} of the "
+                     f"{nseq * cfg.K} positions it is credited with here, so the figure flatters the CPU)",
+           "positions_evaluated_per_pass": evaluated,
+           "value_counting_evaluated_positions_only": evaluated * passes / spent}
+    # the same oracle on ONE thread, on a smaller sample (about a quarter of the time budget)
+    n1 = int(max(1, min(nseq, round(nseq * 0.25 * min_seconds / max(spent / passes, 1e-9) / max(cores, 1)))))
+    t0 = time.perf_counter()
+    oracle.verify(batch.target_logits[:n1], batch.draft_logits[:n1], batch.draft_tokens[:n1], groups.group_ptr,
+                  groups.group_tok, groups.tok_degree, batch.uniforms[:n1], batch.temperature, threads=1)
+    t1 = time.perf_counter() - t0
+    out["single_thread"] = {"value": n1 * cfg.K / t1, "unit": UNIT, "cores": 1,
+                            "sample": f"first {n1} sequences, one pass, {t1:.3f} s wall on one thread"}
     if timed_outputs is not None:
         # the oracle's results on that sample against what the timed GPU steps produced, decision by decision
         from oracle.compare import compare_verify
@@ -183,6 +223,73 @@ def run_reference(args, cfg, rank):
     print(json.dumps(line), flush=True)
 
 
+def quick_workload(binding, torch, wcfg, peak, steps=300):
+    """ms per pcg_verify call (default mode, rotating input copies) and pcg_verify_thinning call of a small workload."""
+    groups = W.make_groups(wcfg)
+    batch = W.make_batch(wcfg)
+    handle = binding.Groups(groups.V, groups.group_ptr, groups.group_tok, groups.tok_degree)
+
+    def dev(a):
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(a).cuda()
+
+    base = (dev(batch.target_logits), dev(batch.draft_logits), dev(batch.draft_tokens), dev(batch.uniforms))
+    rotation = [base] + [tuple(t.clone() for t in base) for _ in range(input_copies(wcfg) - 1)]
+    B, K, V, M = wcfg.B, wcfg.K, wcfg.V, groups.M
+    dt_code = binding.PCG_BF16 if wcfg.dtype == "bf16" else binding.PCG_F32
+    esz = 2 if wcfg.dtype == "bf16" else 4
+    ws = torch.empty(binding.pcg_verify_workspace_bytes(B, K, V, M, dt_code, 0), dtype=torch.uint8, device="cuda")
+    out = (torch.empty(B, dtype=torch.int32, device="cuda"), torch.empty((B, K + 1), dtype=torch.int32, device="cuda"),
+           torch.empty((B, K + 1), dtype=torch.int32, device="cuda"), torch.empty(B, dtype=torch.int32, device="cuda"))
+    thin_u = torch.from_numpy(W.make_thin_uniforms(wcfg, 32)).cuda()
+    thin_ws = torch.empty(binding.pcg_verify_thinning_workspace_bytes(B, K, V, M, dt_code), dtype=torch.uint8, device="cuda")
+    thin_out = out + (torch.empty(B, dtype=torch.int32, device="cuda"),)
+    res = {"config": workload_config(wcfg)}
+    for key in ("verify", "verify_thinning"):
+        def one(i):
+            a_tl, a_dl, a_x, a_u = rotation[i % len(rotation)]
+            if key == "verify":
+                binding.pcg_verify(a_tl, a_dl, a_x, handle, a_u, wcfg.temperature, workspace=ws, out=out)
+            else:
+                binding.pcg_verify_thinning(a_tl, a_dl, a_x, handle, a_u, thin_u, wcfg.temperature, workspace=thin_ws,
+                                            out=thin_out)
+        for i in range(10):
+            one(i)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(steps):
+            one(i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        gbs = B * (2 * K + 1) * V * esz / (ms * 1e-3) / 1e9
+        res[key] = {"ms_per_step": ms, "steps": steps, "value": B * K / (ms * 1e-3), "unit": UNIT,
+                    "whole_step_gbs": gbs, "whole_step_frac_of_measured_peak": gbs / peak}
+    handle.close()
+    return res
+
+
+def group_construction_leg(binding, torch, V, reps=2):
+    """The one-time group construction (Sec. 2.1) on a seeded clustered table of vocabulary size V, both tensor paths."""
+    d_emb = 512 if V >= 32768 else 128
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(2511)
+    centres = torch.randn((max(1, V // 24), d_emb), device="cuda", generator=gen)
+    which = torch.randint(0, max(1, V // 24), (V,), device="cuda", generator=gen)
+    table = (centres[which] + 0.35 * torch.randn((V, d_emb), device="cuda", generator=gen)).to(torch.bfloat16)
+    res = {"V": V, "d": d_emb, "theta": 0.42}
+    for flag, key in ((False, "tcgen05"), (True, "mma_sync")):
+        for _ in range(reps):  # the last repetition is reported
+            asg = binding.Asg(table, 0.42, mma_sync=flag)
+            info = {"similarity_ms": asg.info.similarity_ms, "total_ms": asg.info.total_ms, "groups": asg.info.M,
+                    "tflops": 2.0 * V * V * d_emb / (asg.info.similarity_ms * 1e-3) / 1e12}
+            asg.close()
+        res[key] = info
+    return res
+
+
 L2_BYTES = 126 << 20
 
 
@@ -225,6 +332,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-modes", action="store_true", help="skip the brief timing of the other pcg_verify modes")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the brief timing of the smaller workloads C1-C4")
+    ap.add_argument("--only-group-construction", action="store_true",
+                    help="run nothing but the one-time group construction (pcg_asg_create) on a seeded clustered table "
+                         "of the workload's vocabulary size and print its timing (used for profiling that kernel)")
     args = ap.parse_args()
     cfg = W.CONFIGS[args.workload]
     if args.batch > 0:
@@ -254,6 +365,10 @@ def main():
 
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     binding.load()
+    if args.only_group_construction:
+        if rank == 0:
+            print(json.dumps({"group_construction": group_construction_leg(binding, torch, cfg.V, reps=3)}), flush=True)
+        return
 
     # ---- inputs: this rank's own batch (sequences rank*B .. rank*B+B-1 of the workload's stream) ----
     groups = W.make_groups(cfg)
@@ -312,24 +427,28 @@ def main():
 
     for _ in range(max(args.warmup, 3)):
         step()
-    # stage events on every 8th timed step (recorded once here so that their handles exist): an event between two
-    # kernels costs a drain of the first one, 7 us per call at C5 when every step carries them
-    STAGE_EVERY = 8
-    stage = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(-(-args.steps // STAGE_EVERY))]
-    for evs in stage:
-        for e in evs:
-            e.record()
     barrier()
-    sampler = ClockSampler(physical_gpu_index(local_rank)).start()
+    sampler = ClockSampler(physical_gpu_index(local_rank), period_s=0.002).start()
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_begin.record()
     for i in range(args.steps):
-        step(stage[i // STAGE_EVERY] if i % STAGE_EVERY == 0 else None)
+        step()
     t_end.record()
     barrier()
-    clocks = sampler.stop()
     ms_total = max_over_ranks(t_begin.elapsed_time(t_end), dist)
     ms_step = ms_total / args.steps
+    # Stage times: a second, short loop after the timed region, every step carrying the library's three stage events
+    # (an event between two kernels costs a drain of the first one, which is why the timed steps carry none).
+    STAGE_STEPS = 16
+    stage = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(STAGE_STEPS)]
+    for evs in stage:
+        for e in evs:
+            e.record()
+    torch.cuda.synchronize()
+    for evs in stage:
+        step(evs)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
     pos_ms = statistics.fmean(e[0].elapsed_time(e[1]) for e in stage)
     term_ms = statistics.fmean(e[1].elapsed_time(e[2]) for e in stage)
     accept_len = (thin_out if thinning else out)[0].cpu().numpy()
@@ -359,11 +478,11 @@ def main():
     info = handle.info
     chunk_unit = 256 if (B >= 256 and (64 << 20) // (V * 4) >= 256) else 128 if B >= 128 else 32
     chunk = min(-(-B // chunk_unit) * chunk_unit, max(chunk_unit, ((64 << 20) // (V * 4)) // chunk_unit * chunk_unit))
-    batched = 1 + 1 + 2 * (-(-B // chunk)) + 1  # position, prepare, (transpose, sparse product) per chunk, draw
+    batched = 1 + 2 * (-(-B // chunk)) + 1  # position, (transposed operand, sparse product) per chunk, pick
     sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
     default_is_cluster = B * info.slices <= 2 * sm_count  # the library's rule for PCG_VERIFY_DEFAULT
     launches_per_step = {"default": 2 if default_is_cluster else batched, "cluster": 2, "batched": batched,
-                         "dense": 2 + 1 + 1 + 1, "thinning": 2}[args.mode]
+                         "dense": 2 * 3 + 1 + 1 + 1, "thinning": 2}[args.mode]
 
     # the other modes, briefly (same inputs, same outputs): context for the headline mode
     other_modes = {}
@@ -411,6 +530,13 @@ def main():
         c1.record()
         torch.cuda.synchronize()
         other_modes["cuda_graph_replay_of_timed_mode"] = {"ms_per_step": c0.elapsed_time(c1) / reps, "steps": reps}
+
+    # the smaller workloads C1-C4, briefly, in the default mode (they are parity-test cases, not the headline; their
+    # times are launch-latency bound, see config.l2 of each)
+    other_workloads = {}
+    if world == 1 and not args.no_other_workloads and not args.no_other_modes and cfg.name == "C5":
+        for name in ("C1", "C2", "C3", "C4"):
+            other_workloads[name] = quick_workload(binding, torch, W.CONFIGS[name], hbm_peak()[0])
 
     # the other two entry points of the boundary, briefly: pcg_group_probs on a slice of the target rows, and the
     # one-time group construction on a seeded clustered table of the workload's vocabulary size
@@ -467,21 +593,7 @@ def main():
             "positions_sampled": ns,
             "group_overlap_sum_min_PQ": float(torch.minimum(Pg, Qg).sum(dim=1).mean()),
             "token_overlap_sum_min_pq": float(torch.minimum(pt, qt).sum(dim=1).mean())}
-        d_emb = 512 if V >= 32768 else 128
-        gen = torch.Generator(device="cuda")
-        gen.manual_seed(2511)
-        centres = torch.randn((max(1, V // 24), d_emb), device="cuda", generator=gen)
-        which = torch.randint(0, max(1, V // 24), (V,), device="cuda", generator=gen)
-        table = (centres[which] + 0.35 * torch.randn((V, d_emb), device="cuda", generator=gen)).to(torch.bfloat16)
-        for flag, key in ((False, "tcgen05"), (True, "mma_sync")):
-            asg = binding.Asg(table, 0.42, mma_sync=flag)
-            asg.close()
-            asg = binding.Asg(table, 0.42, mma_sync=flag)
-            extras.setdefault("group_construction", {"V": V, "d": d_emb, "theta": 0.42})[key] = {
-                "similarity_ms": asg.info.similarity_ms, "total_ms": asg.info.total_ms, "groups": asg.info.M,
-                "tflops": 2.0 * V * V * d_emb / (asg.info.similarity_ms * 1e-3) / 1e12}
-            asg.close()
-        del table, centres, which
+        extras["group_construction"] = group_construction_leg(binding, torch, V)
     if rank == 0:
         peak, peak_src = hbm_peak()
         alg_bytes = B * K * 2 * V * esz  # per drafted position: one target and one draft row, read once
@@ -496,15 +608,22 @@ def main():
                     "whole_step_frac_of_measured_peak": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9 / peak,
                     "whole_step_frac_of_8tbs": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9 / 8000.0},
             "roofline": {"bound": "hbm", "kernel": "position_kernel", "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                         "unit": "GB/s", "frac": achieved / peak, "traffic": ncu_traffic_bytes(cfg.name),
+                         "traffic_source": f"profiles/position_kernel_{cfg.name.lower()}_dram_traffic.md (null if the "
+                                           "kernels were edited after that capture)",
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": alg_bytes,
-                         "avg_launch_ms": pos_ms},
+                         "avg_launch_ms": pos_ms,
+                         # the figure the target is stated on: ALL kernels of the call, counted logits bytes / step time
+                         "whole_call": {"achieved": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9,
+                                        "frac": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9 / peak,
+                                        "counted_bytes_per_step": B * (2 * K + 1) * V * esz, "ms_per_step": ms_step}},
             "stages_ms": {"per_position_stage": pos_ms, "per_sequence_stage": term_ms,
-                          "sampled_on_every_nth_timed_step": STAGE_EVERY},
+                          "samples": STAGE_STEPS, "sampled": "on a separate loop of steps after the timed region"},
             "mode": args.mode + (" (per-sequence stage: " + ("cluster" if default_is_cluster else "batched") + ")"
                                  if args.mode == "default" else
                                  f" (pcg_verify_thinning, {args.thin_trials} trials supplied)" if thinning else ""),
             "other_modes": other_modes,
+            "other_workloads": other_workloads,
             "other_entry_points": extras,
             "e2e": {"value": world * B * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,

@@ -189,6 +189,35 @@ def pcg_group_probs(logits, groups: Groups, temperature: float = 1.0, out=None, 
     return out
 
 
+def _check_verify_tensors(target_logits, draft_logits, draft_tokens, groups, uniforms, out=None, extra=(), cuda=True):
+    """Shapes, types, contiguity and placement of the tensors of a verification call (the library itself only sees
+    raw pointers).  ``extra`` lists further (tensor, shape, dtype) triples; ``out`` is the tuple of output tensors
+    (accept_len [B], tokens [B, K+1], groups [B, K+1] or None, flags [B] or None, then [B] tensors or None)."""
+    import torch
+
+    if target_logits.dim() != 3:
+        raise ValueError("target_logits must be [B, K+1, V]")
+    B, K1, V = target_logits.shape
+    K = K1 - 1
+    if V != groups.V:
+        raise ValueError(f"the logits have V={V} but the group handle was built for V={groups.V}")
+    dev = target_logits.device
+    if target_logits.is_cuda != cuda:
+        raise ValueError("the tensors of this call must live in %s memory" % ("CUDA" if cuda else "host"))
+    checks = [(target_logits, (B, K1, V), target_logits.dtype), (draft_logits, (B, K, V), target_logits.dtype),
+              (draft_tokens, (B, K), torch.int32), (uniforms, (B, K + 1, 2), torch.float32)] + list(extra)
+    if out is not None:
+        shapes = [(B,), (B, K + 1), (B, K + 1), (B,)] + [(B,)] * (len(out) - 4)
+        checks += [(t, sh, torch.int32) for t, sh in zip(out, shapes) if t is not None]
+        if out[0] is None or out[1] is None:
+            raise ValueError("the accept-length and token outputs are required")
+    for t, shape, dtype in checks:
+        if tuple(t.shape) != tuple(shape) or not t.is_contiguous() or t.device != dev or t.dtype != dtype:
+            raise ValueError(f"expected a contiguous {dtype} tensor of shape {tuple(shape)} on {dev}, got "
+                             f"{t.dtype} {tuple(t.shape)} on {t.device}")
+    return B, K, V
+
+
 def pcg_verify_workspace_bytes(B: int, K: int, V: int, M: int, dtype: int, mode: int = 0) -> int:
     return int(load().pcg_verify_workspace_bytes(B, K, V, M, dtype, mode))
 
@@ -204,16 +233,8 @@ def pcg_verify(target_logits, draft_logits, draft_tokens, groups: Groups, unifor
     """
     import torch
 
-    B, K1, V = target_logits.shape
-    K = K1 - 1
+    B, K, V = _check_verify_tensors(target_logits, draft_logits, draft_tokens, groups, uniforms, out)
     dev = target_logits.device
-    for t, shape in ((draft_logits, (B, K, V)), (draft_tokens, (B, K)), (uniforms, (B, K + 1, 2))):
-        if tuple(t.shape) != shape or not t.is_contiguous() or t.device != dev:
-            raise ValueError(f"expected a contiguous tensor of shape {shape} on {dev}")
-    if not target_logits.is_contiguous() or draft_logits.dtype != target_logits.dtype:
-        raise ValueError("target and draft logits must be contiguous and share a dtype")
-    if draft_tokens.dtype != torch.int32 or uniforms.dtype != torch.float32:
-        raise TypeError("draft_tokens must be int32 and uniforms float32")
     dt = dtype_code(target_logits)
     need = pcg_verify_workspace_bytes(B, K, V, groups.M, dt, mode)
     if workspace is None:
@@ -243,8 +264,9 @@ def pcg_verify_host(target_logits, draft_logits, draft_tokens, groups: Groups, u
                     arena, out, mode: int = 0, stream=None):
     """``pcg_verify_host``: inputs and the four ``out`` tensors are HOST torch tensors (pinned for speed);
     ``arena`` is a uint8 CUDA tensor of at least ``pcg_verify_host_arena_bytes`` bytes.  Synchronises."""
-    B, K1, V = target_logits.shape
-    K = K1 - 1
+    B, K, V = _check_verify_tensors(target_logits, draft_logits, draft_tokens, groups, uniforms, out, cuda=False)
+    if not arena.is_cuda or arena.element_size() != 1 or not arena.is_contiguous():
+        raise ValueError("arena must be a contiguous one-byte-per-element CUDA tensor")
     accept_len, tokens, grp, flags = out
     _check(load().pcg_verify_host(_dev_ptr(target_logits), _dev_ptr(draft_logits), dtype_code(target_logits), B, K,
                                   _dev_ptr(draft_tokens), groups.handle, _dev_ptr(uniforms), float(temperature),
@@ -257,10 +279,10 @@ def pcg_verify_static(target_logits, draft_logits, draft_tokens, groups: Groups,
                       out, stream=None):
     """``pcg_verify_static``: verification with the library's built-in scratch.  Every tensor, the four outputs
     in ``out`` included (groups and flags may be None), is supplied by the caller; nothing is allocated here."""
-    B, K1, V = target_logits.shape
+    B, K, V = _check_verify_tensors(target_logits, draft_logits, draft_tokens, groups, uniforms, out)
     accept_len, tokens, grp, flags = out
     _check(load().pcg_verify_static(_dev_ptr(target_logits), _dev_ptr(draft_logits), dtype_code(target_logits), B,
-                                    K1 - 1, _dev_ptr(draft_tokens), groups.handle, _dev_ptr(uniforms),
+                                    K, _dev_ptr(draft_tokens), groups.handle, _dev_ptr(uniforms),
                                     float(temperature), _dev_ptr(accept_len), _dev_ptr(tokens), _dev_ptr(grp),
                                     _dev_ptr(flags), _stream_ptr(stream)))
     return out
@@ -279,20 +301,12 @@ def pcg_verify_thinning(target_logits, draft_logits, draft_tokens, groups: Group
     """
     import torch
 
-    B, K1, V = target_logits.shape
-    K = K1 - 1
-    dev = target_logits.device
-    if thin_uniforms.dim() != 3 or thin_uniforms.shape[0] != B or thin_uniforms.shape[2] != 3:
+    if thin_uniforms.dim() != 3 or thin_uniforms.shape[2] != 3:
         raise ValueError("thin_uniforms must be [B, n_trials, 3]")
     n_trials = int(thin_uniforms.shape[1])
-    for t, shape in ((draft_logits, (B, K, V)), (draft_tokens, (B, K)), (uniforms, (B, K + 1, 2)),
-                     (thin_uniforms, (B, n_trials, 3))):
-        if tuple(t.shape) != shape or not t.is_contiguous() or t.device != dev:
-            raise ValueError(f"expected a contiguous tensor of shape {shape} on {dev}")
-    if not target_logits.is_contiguous() or draft_logits.dtype != target_logits.dtype:
-        raise ValueError("target and draft logits must be contiguous and share a dtype")
-    if draft_tokens.dtype != torch.int32 or uniforms.dtype != torch.float32 or thin_uniforms.dtype != torch.float32:
-        raise TypeError("draft_tokens must be int32 and the uniforms float32")
+    B, K, V = _check_verify_tensors(target_logits, draft_logits, draft_tokens, groups, uniforms, out,
+                                    extra=[(thin_uniforms, (target_logits.shape[0], n_trials, 3), torch.float32)])
+    dev = target_logits.device
     dt = dtype_code(target_logits)
     if workspace is None:
         workspace = torch.empty(pcg_verify_thinning_workspace_bytes(B, K, V, groups.M, dt), dtype=torch.uint8, device=dev)

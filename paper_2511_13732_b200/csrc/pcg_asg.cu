@@ -255,7 +255,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const 
                                                                          int *error) {
     constexpr int S = kTcStages, BK = kTcBK;
     extern __shared__ unsigned char tc_smem_raw[];  // [S][A 128 rows | B 256 rows][128 bytes per row], 1024-aligned below
-    __shared__ __align__(8) uint64_t bars[2 * S + 4];          // full[S], empty[S], acc_full[2], acc_empty[2]
+    __shared__ __align__(8) uint64_t bars[2 * S + 5];          // full[S], empty[S], acc_full[2], acc_empty[2], drain
     __shared__ uint32_t tmem_slot;
     __shared__ int failed_flag;
     volatile int *failed = &failed_flag;
@@ -266,6 +266,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const 
     auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
     auto acc_full_bar = [&](int b) { return bar0 + 8u * (2 * S + b); };
     auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * S + 2 + b); };
+    const uint32_t drain_bar = bar0 + 8u * (2 * S + 4);  // failure path only: all issued MMAs have retired
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_bar(s)));
@@ -275,6 +276,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const 
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(acc_full_bar(b)));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(acc_empty_bar(b)), "r"(32 * kTcEpilogueWarps));
         }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(drain_bar));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         failed_flag = 0;
     }
@@ -389,6 +391,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const 
                     tma_box(b + kTcABytes, j0 + 128);
                 }
             }
+            if (*failed) {
+                // Giving up: copies already requested may still be landing in shared memory.  Wait (bounded, and no
+                // longer cut short by the failure flag) for the last S armed stages before the block may end.
+                for (int back = 1; back <= S && back <= it; ++back) {
+                    const int j = it - back, s = j % S;
+                    for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin) {
+                        uint32_t done;
+                        asm volatile(
+                            "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                            : "=r"(done)
+                            : "r"(full_bar(s)), "r"((uint32_t)((j / S) & 1))
+                            : "memory");
+                        if (done) break;
+                        __nanosleep(20);
+                    }
+                }
+            }
         }
     } else if (warp == kTcEpilogueWarps + kTcProducerWarps && lane == 0) {
         // ------------------------------------------------------------------ MMA issuer (one thread)
@@ -429,6 +448,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const 
                                  acc_full_bar(buf))
                              : "memory");
             ++tcount;
+        }
+        if (*failed) {
+            // Giving up: MMAs already issued may still be writing tensor memory.  One more commit arrives on a
+            // barrier of its own when all of them have retired; wait for it (bounded) before the memory is freed.
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(drain_bar)
+                         : "memory");
+            for (uint32_t spin = 0; spin < kTcSpinLimit; ++spin) {
+                uint32_t done;
+                asm volatile(
+                    "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                    : "=r"(done)
+                    : "r"(drain_bar), "r"(0u)
+                    : "memory");
+                if (done) break;
+                __nanosleep(20);
+            }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

@@ -1,4 +1,6 @@
 // pcg_verify_host: the same verification for callers whose tensors live in host memory.
+#include <cmath>
+
 #include "pcg_common.cuh"
 
 namespace {
@@ -64,11 +66,36 @@ extern "C" pcg_status pcg_verify_host(const void *target_logits, const void *dra
         set_error("pcg_verify_host: need B >= 0 and K >= 1 (B=%d K=%d)", B, K);
         return PCG_ERR_INVALID_ARG;
     }
+    if (K > 1024) {
+        set_error("pcg_verify_host: K=%d exceeds the supported 1024 drafted positions per sequence", K);
+        return PCG_ERR_UNSUPPORTED;
+    }
+    if (mode != PCG_VERIFY_DEFAULT && mode != PCG_VERIFY_DENSE && mode != PCG_VERIFY_CLUSTER_TERMINAL &&
+        mode != PCG_VERIFY_BATCHED_TERMINAL) {
+        set_error("pcg_verify_host: unknown or contradictory mode bits 0x%x", mode);
+        return PCG_ERR_INVALID_ARG;
+    }
+    if (!(temperature >= 1e-6f) || !std::isfinite(temperature)) {
+        set_error("pcg_verify_host: temperature must be finite and at least 1e-6");
+        return PCG_ERR_INVALID_ARG;
+    }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev != groups->device) {
+        set_error("pcg_verify_host: the handle lives on device %d but device %d is current", groups->device, dev);
+        return PCG_ERR_INVALID_ARG;
+    }
+    if (mode == PCG_VERIFY_CLUSTER_TERMINAL && !groups->has_sweep) {
+        set_error("pcg_verify_host: this handle has no sweep layout, so the cluster terminal is unavailable");
+        return PCG_ERR_UNSUPPORTED;
+    }
     if (B == 0) return PCG_OK;
     if (!target_logits || !draft_logits || !draft_tokens || !uniforms || !out_accept_len || !out_tokens) {
         set_error("pcg_verify_host: null pointer");
         return PCG_ERR_INVALID_ARG;
     }
+    // everything the host can refuse has been refused above: no copy is enqueued for a call that cannot run
     const Arena a = layout(B, K, groups->dev.V, groups->dev.M, dtype, mode);
     if (!device_arena || ((uintptr_t)device_arena & 255u) || device_arena_bytes < a.total) {
         set_error("pcg_verify_host: device arena must be 256-byte aligned and hold %zu bytes (got %zu)", a.total,
@@ -77,23 +104,30 @@ extern "C" pcg_status pcg_verify_host(const void *target_logits, const void *dra
     }
     char *d = (char *)device_arena;
     cudaStream_t cs = (cudaStream_t)stream;
-    cudaError_t e = cudaMemcpyAsync(d + a.target, target_logits, a.target_bytes, cudaMemcpyHostToDevice, cs);
+    // From the first enqueued copy on, no return before the stream has drained: the caller may free or overwrite
+    // its buffers as soon as this call is back, also after an error.
+    auto fail_after_enqueue = [&](pcg_status st) {
+        (void)cudaStreamSynchronize(cs);
+        return st;
+    };
+    e = cudaMemcpyAsync(d + a.target, target_logits, a.target_bytes, cudaMemcpyHostToDevice, cs);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d + a.draft, draft_logits, a.draft_bytes, cudaMemcpyHostToDevice, cs);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d + a.tokens, draft_tokens, a.tokens_bytes, cudaMemcpyHostToDevice, cs);
     if (e == cudaSuccess) e = cudaMemcpyAsync(d + a.uniforms, uniforms, a.uniforms_bytes, cudaMemcpyHostToDevice, cs);
-    if (e != cudaSuccess) return cuda_fail(e, "copying inputs to the device");
+    if (e != cudaSuccess) return fail_after_enqueue(cuda_fail(e, "copying inputs to the device"));
     pcg_status st = pcg_verify(d + a.target, d + a.draft, dtype, B, K, (const int32_t *)(d + a.tokens), groups,
                                (const float *)(d + a.uniforms), temperature, (int32_t *)(d + a.accept_len),
                                (int32_t *)(d + a.out_tokens), (int32_t *)(d + a.out_groups),
                                (int32_t *)(d + a.out_flags), d + a.workspace, a.ws_bytes, mode, stream, nullptr);
-    if (st != PCG_OK) return st;
+    if (st != PCG_OK) return fail_after_enqueue(st);
     e = cudaMemcpyAsync(out_accept_len, d + a.accept_len, a.len_bytes, cudaMemcpyDeviceToHost, cs);
     if (e == cudaSuccess) e = cudaMemcpyAsync(out_tokens, d + a.out_tokens, a.outtok_bytes, cudaMemcpyDeviceToHost, cs);
     if (e == cudaSuccess && out_groups)
         e = cudaMemcpyAsync(out_groups, d + a.out_groups, a.outtok_bytes, cudaMemcpyDeviceToHost, cs);
     if (e == cudaSuccess && out_flags)
         e = cudaMemcpyAsync(out_flags, d + a.out_flags, a.len_bytes, cudaMemcpyDeviceToHost, cs);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
-    if (e != cudaSuccess) return cuda_fail(e, "copying outputs to the host");
+    if (e != cudaSuccess) return fail_after_enqueue(cuda_fail(e, "copying outputs to the host"));
+    e = cudaStreamSynchronize(cs);
+    if (e != cudaSuccess) return cuda_fail(e, "waiting for the verification to finish");
     return PCG_OK;
 }
