@@ -1005,20 +1005,22 @@ __device__ __forceinline__ void ld_stream_32(const void *p, uint32_t (&w)[8]) {
 }
 
 // Grid (blocks per batch, batches of 32 sequences); block = 8 warps.  LANE = SEQUENCE throughout: a lane reads
-// 32 bytes of its own sequence's two rows per step (whole sectors; the eight warps of a block take neighbouring
-// steps, so a row is fetched in 256-byte stretches), forms D = (p - q) w for those tokens in registers, and the
+// 64 bytes of its own sequence's two rows per step (two whole sectors, one DRAM access: with 32 bytes per step a
+// third more bytes than needed came from DRAM; the eight warps of a block take neighbouring steps, so a row is
+// fetched in 512-byte stretches), forms D = (p - q) w for those tokens in registers, and the
 // warp writes one 128-byte line of Dt per token -- [token][32 sequences] needs no transposition this way.
 //   0. once per block, by warp 0: every lane finds its sequence's first rejection from the accept bits (its
 //      loads all in flight) and fetches the softmax statistics of that position;
-//   1. the block's run of the row is walked with the next step's 64 bytes in flight while the current step's
+//   1. the block's run of the row is walked with the next step's 128 bytes in flight while the current step's
 //      tokens are computed and stored.
 // Lanes that have nothing to read (sequences past the batch, the draft row of a bonus position, tokens past the
 // end of a row) use -inf logits, which contribute exact zeros.
 template <typename T>
-__global__ void __launch_bounds__(kTrThreads, 3) residual_transpose_kernel(TransposeArgs a, GroupsDev G) {
+__global__ void __launch_bounds__(kTrThreads, 2) residual_transpose_kernel(TransposeArgs a, GroupsDev G) {
     pdl_enter();
     constexpr int PW = WordElems<T>::kPerWord;  // logits per 32-bit word
-    constexpr int CH = 8 * PW;                  // tokens per step: 32 bytes of a row
+    constexpr int WPS = 16;                     // 32-bit words per step: 64 bytes of a row
+    constexpr int CH = WPS * PW;                // tokens per step
     constexpr int NWARP = kTrThreads / 32;
     __shared__ int s_n[32];
     __shared__ float4 s_st[32];
@@ -1080,26 +1082,32 @@ __global__ void __launch_bounds__(kTrThreads, 3) residual_transpose_kernel(Trans
     const int b = bbase + lane, nn = max(n, 0);
     const T *tp = reinterpret_cast<const T *>(a.target) + ((int64_t)(live ? b : 0) * (K + 1) + nn) * V;
     const T *qp = K > 0 ? reinterpret_cast<const T *>(a.draft) + ((int64_t)(live ? b : 0) * K + min(nn, K - 1)) * V : tp;
-    // whole 32-byte pieces can be loaded as such if every live lane's rows start on 32-byte boundaries
-    const bool lane_al = !live || ((((uintptr_t)tp | (resid ? (uintptr_t)qp : 0)) & 31u) == 0);
-    const bool aligned = __all_sync(0xffffffffu, lane_al) && ((size_t)V * sizeof(T)) % 32 == 0;
+    // whole 64-byte pieces can be loaded as such if every live lane's rows start on 64-byte boundaries
+    const bool lane_al = !live || ((((uintptr_t)tp | (resid ? (uintptr_t)qp : 0)) & 63u) == 0);
+    const bool aligned = __all_sync(0xffffffffu, lane_al) && ((size_t)V * sizeof(T)) % 64 == 0;
     const int nsteps = (V + CH - 1) / CH;
     const int step_lo = (int)(((int64_t)nsteps * blockIdx.x) / gridDim.x);
     const int step_hi = (int)(((int64_t)nsteps * (blockIdx.x + 1)) / gridDim.x);
     float *dst = a.Dt + ((size_t)blockIdx.y * V) * 32 + lane;
 
-    auto fetch = [&](int step, uint32_t(&wp)[8], uint32_t(&wq)[8]) {
+    auto fetch = [&](int step, uint32_t(&wp)[WPS], uint32_t(&wq)[WPS]) {
         const int t = step * CH;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) wp[j] = wq[j] = NegInfBits<T>::word;
+        for (int j = 0; j < WPS; ++j) wp[j] = wq[j] = NegInfBits<T>::word;
         if (step >= step_hi) return;
         if (aligned && t + CH <= V) {
-            if (live) ld_stream_32(tp + t, wp);
-            if (resid) ld_stream_32(qp + t, wq);
-        } else {  // ragged end of the row, or rows that are not 32-byte aligned: element by element
+            if (live) {
+                ld_stream_32(tp + t, *reinterpret_cast<uint32_t(*)[8]>(&wp[0]));
+                ld_stream_32(tp + t + CH / 2, *reinterpret_cast<uint32_t(*)[8]>(&wp[8]));
+            }
+            if (resid) {
+                ld_stream_32(qp + t, *reinterpret_cast<uint32_t(*)[8]>(&wq[0]));
+                ld_stream_32(qp + t + CH / 2, *reinterpret_cast<uint32_t(*)[8]>(&wq[8]));
+            }
+        } else {  // ragged end of the row, or rows that are not 64-byte aligned: element by element
             T ep[CH], eq[CH];
-            memcpy(ep, wp, 32);
-            memcpy(eq, wq, 32);
+            memcpy(ep, wp, 4 * WPS);
+            memcpy(eq, wq, 4 * WPS);
 #pragma unroll
             for (int e = 0; e < CH; ++e) {
                 if (t + e < V) {
@@ -1107,11 +1115,11 @@ __global__ void __launch_bounds__(kTrThreads, 3) residual_transpose_kernel(Trans
                     if (resid) eq[e] = qp[t + e];
                 }
             }
-            memcpy(wp, ep, 32);
-            memcpy(wq, eq, 32);
+            memcpy(wp, ep, 4 * WPS);
+            memcpy(wq, eq, 4 * WPS);
         }
     };
-    auto emit = [&](int step, const uint32_t(&wp)[8], const uint32_t(&wq)[8]) {
+    auto emit = [&](int step, const uint32_t(&wp)[WPS], const uint32_t(&wq)[WPS]) {
         const int t = step * CH;
         float inv[CH];
         if (!G.ent_w && t + CH <= V) {
@@ -1125,7 +1133,7 @@ __global__ void __launch_bounds__(kTrThreads, 3) residual_transpose_kernel(Trans
             for (int e = 0; e < CH; ++e) inv[e] = (!G.ent_w && t + e < V) ? G.inv_deg[t + e] : 1.f;
         }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < WPS; ++j) {
             float lp[PW], lq[PW];
             WordElems<T>::unpack(wp[j], lp);
             WordElems<T>::unpack(wq[j], lq);
@@ -1138,7 +1146,7 @@ __global__ void __launch_bounds__(kTrThreads, 3) residual_transpose_kernel(Trans
             }
         }
     };
-    uint32_t ap[8], aq[8], bp[8], bq[8];
+    uint32_t ap[WPS], aq[WPS], bp[WPS], bq[WPS];
     int step = step_lo + warp;
     fetch(step, ap, aq);
     for (; step < step_hi; step += 2 * NWARP) {
@@ -1921,14 +1929,14 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
     return w;
 }
 
-// The transposed-operand kernel over nb batches of 32 sequences: about three resident blocks per SM, shared out
+// The transposed-operand kernel over nb batches of 32 sequences: two resident blocks per SM, shared out
 // over the batches, each walking a run of its batch's rows.
 template <typename T>
 static cudaError_t launch_transpose(const TransposeArgs &tr, int nb, const GroupsDev &G, int sm_count, cudaStream_t cs) {
-    constexpr int ch = 32 / (int)sizeof(T);  // tokens per step of a lane
+    constexpr int ch = 64 / (int)sizeof(T);  // tokens per step of a lane
     const int nsteps = (G.V + ch - 1) / ch;
     // a block's run: at least 8 steps per warp, so that finding the terminal positions is paid for
-    const int per_batch = std::max(1, std::min((nsteps + 63) / 64, 3 * sm_count / std::max(nb, 1)));
+    const int per_batch = std::max(1, std::min((nsteps + 63) / 64, 2 * sm_count / std::max(nb, 1)));
     const dim3 grid((unsigned)per_batch, (unsigned)nb);
     return launch_after(residual_transpose_kernel<T>, grid, dim3(kTrThreads), 0, cs, tr, G);
 }
