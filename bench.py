@@ -284,7 +284,9 @@ def group_construction_leg(binding, torch, V, reps=2):
         for _ in range(reps):  # the last repetition is reported
             asg = binding.Asg(table, 0.42, mma_sync=flag)
             info = {"similarity_ms": asg.info.similarity_ms, "total_ms": asg.info.total_ms, "groups": asg.info.M,
-                    "tflops": 2.0 * V * V * d_emb / (asg.info.similarity_ms * 1e-3) / 1e12}
+                    # the full V x V product at 2 flops per multiply-add; the tensor-core form executes about half of it
+                    # (the cosine is symmetric: tiles below the diagonal blocks are mirrored, not computed)
+                    "tflops_full_matrix_equivalent": 2.0 * V * V * d_emb / (asg.info.similarity_ms * 1e-3) / 1e12}
             asg.close()
         res[key] = info
     return res

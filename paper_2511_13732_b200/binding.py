@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "PCG_OK", 1: "PCG_ERR_INVALID_ARG", 2: "PCG_ERR_INVALID_GROUP
 EXPORTS = [
     "pcg_status_string", "pcg_last_error", "pcg_groups_create", "pcg_groups_destroy", "pcg_groups_info",
     "pcg_groups_set_accept_bias",
-    "pcg_group_probs", "pcg_verify_workspace_bytes", "pcg_verify", "pcg_verify_host_arena_bytes", "pcg_verify_host",
+    "pcg_group_probs", "pcg_group_probs_workspace_bytes", "pcg_group_probs_ws", "pcg_verify_workspace_bytes", "pcg_verify", "pcg_verify_host_arena_bytes", "pcg_verify_host",
     "pcg_verify_static", "pcg_verify_thinning_workspace_bytes", "pcg_verify_thinning", "pcg_asg_create", "pcg_asg_info", "pcg_asg_csr", "pcg_asg_destroy",
 ]
 
@@ -85,6 +85,9 @@ def load(build_if_missing: bool = True):
     lib.pcg_groups_set_accept_bias.argtypes, lib.pcg_groups_set_accept_bias.restype = [vp, f32], ctypes.c_int
     lib.pcg_group_probs.argtypes = [vp, ctypes.c_int, i64, f32, vp, vp, vp]
     lib.pcg_group_probs.restype = ctypes.c_int
+    lib.pcg_group_probs_workspace_bytes.argtypes, lib.pcg_group_probs_workspace_bytes.restype = [i32], sz
+    lib.pcg_group_probs_ws.argtypes = [vp, ctypes.c_int, i64, f32, vp, vp, vp, sz, vp]
+    lib.pcg_group_probs_ws.restype = ctypes.c_int
     lib.pcg_verify_workspace_bytes.argtypes = [i32, i32, i32, i32, ctypes.c_int, u32]
     lib.pcg_verify_workspace_bytes.restype = sz
     lib.pcg_verify.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, vp, f32, vp, vp, vp, vp, vp, sz, u32, vp, vp]
@@ -175,8 +178,16 @@ class Groups:
             pass
 
 
-def pcg_group_probs(logits, groups: Groups, temperature: float = 1.0, out=None, stream=None):
-    """``pcg_group_probs``: logits [rows, V] (CUDA, float32 or bfloat16) -> float32 [rows, M]."""
+def pcg_group_probs_workspace_bytes(V: int) -> int:
+    return int(load().pcg_group_probs_workspace_bytes(int(V)))
+
+
+def pcg_group_probs(logits, groups: Groups, temperature: float = 1.0, out=None, stream=None, workspace=None):
+    """``pcg_group_probs``: logits [rows, V] (CUDA, float32, bfloat16 or float16) -> float32 [rows, M].
+
+    With ``workspace`` (a uint8 CUDA tensor of at least ``pcg_group_probs_workspace_bytes(V)`` bytes) the call goes
+    through ``pcg_group_probs_ws`` and touches no scratch of the handle, so calls with separate workspaces may run
+    side by side on different streams."""
     import torch
 
     if logits.dim() != 2 or logits.shape[1] != groups.V or not logits.is_contiguous() or not logits.is_cuda:
@@ -184,8 +195,15 @@ def pcg_group_probs(logits, groups: Groups, temperature: float = 1.0, out=None, 
     rows = logits.shape[0]
     if out is None:
         out = torch.empty((rows, groups.M), dtype=torch.float32, device=logits.device)
-    _check(load().pcg_group_probs(_dev_ptr(logits), dtype_code(logits), rows, float(temperature), groups.handle,
-                                  _dev_ptr(out), _stream_ptr(stream)))
+    elif tuple(out.shape) != (rows, groups.M) or out.dtype != torch.float32 or not out.is_contiguous() or out.device != logits.device:
+        raise ValueError("out must be a contiguous float32 tensor [rows, M] on the logits' device")
+    if workspace is None:
+        _check(load().pcg_group_probs(_dev_ptr(logits), dtype_code(logits), rows, float(temperature), groups.handle,
+                                      _dev_ptr(out), _stream_ptr(stream)))
+    else:
+        _check(load().pcg_group_probs_ws(_dev_ptr(logits), dtype_code(logits), rows, float(temperature), groups.handle,
+                                         _dev_ptr(out), _dev_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                         _stream_ptr(stream)))
     return out
 
 

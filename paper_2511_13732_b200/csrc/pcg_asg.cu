@@ -5,7 +5,9 @@
 //   asg_prepare_kernel      rows to bfloat16 (zero-padded to a multiple of 32 columns and 128 rows), 1/|row| in fp32
 //   asg_similarity_tc_kernel  E * E^T on the tensor cores (tcgen05, TMA; asg_similarity_kernel is the mma.sync form);
 //                           the epilogue turns each dot product into cos = dot * rn_i * rn_j, compares with theta
-//                           and packs the decisions into a V x V BIT matrix (the similarities are never stored)
+//                           and packs the decisions into a V x V BIT matrix (the similarities are never stored);
+//                           the tensor-core form computes only the tiles on or right of the diagonal blocks
+//   asg_mirror_kernel       (tensor-core form) the lower triangle of the bit matrix as the transpose of the upper
 //   asg_row_kernel          per row: population count and a position-aware 64-bit hash of its bit row
 //   asg_representative_kernel  rep(t) = smallest t' with G(t') == G(t).  Such a t' is itself a member of G(t)
 //                           (t' is in G(t') = G(t)), so only the set bits below t are candidates: hash, then
@@ -302,7 +304,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const 
         const int tj = (sb % sbJ) * kTcRasterCols + local / kTcRasterRows;
         i0 = ti * kTcRows;
         j0 = tj * kTcTile;
-        return ti < nI && tj < nJ;
+        // The cosine is symmetric: only tiles that reach the diagonal block of 256 columns of their rows, or lie to
+        // its right, are computed (column block tj >= row block ti / 2); asg_mirror_kernel fills in the rest.
+        return ti < nI && tj < nJ && tj >= ti * kTcRows / kTcTile;
     };
 
     if (warp < kTcEpilogueWarps) {
@@ -470,6 +474,52 @@ __global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const 
     __syncthreads();
     if (tid == 0 && failed_flag) atomicMax(error, 1);
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
+}
+
+// The lower triangle of the bit matrix from the upper one (cos is symmetric, so t' in G(t) iff t in G(t')): the
+// block of 256 rows x 256 columns at (TR, TC), TC < TR, is the transpose of the block at (TC, TR).  One thread block
+// per such pair: 256 rows x 32 bytes in (whole sectors), the 256 x 256 bits turned with warp ballots (lane = input
+// row; one ballot per bit position gives a word of the output row of that position), 256 rows x 32 bytes out.
+constexpr int kMirrorBits = 256;
+static_assert(kMirrorBits == kTcTile, "the tensor-core kernel computes whole diagonal blocks of this size");
+__global__ void __launch_bounds__(kMirrorBits) asg_mirror_kernel(uint32_t *bits, int V, int W) {
+    const int TR = blockIdx.y, TC = blockIdx.x;
+    if (TC >= TR) return;
+    constexpr int WB = kMirrorBits / 32;  // words per block row
+    __shared__ uint32_t win[kMirrorBits][WB + 1], wout[kMirrorBits][WB + 1];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    {
+        const int row = TC * kMirrorBits + tid;
+        uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+        if (row < V) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(bits + (size_t)row * W + (size_t)TR * WB);
+            a = src[0];
+            b = src[1];
+        }
+        win[tid][0] = a.x, win[tid][1] = a.y, win[tid][2] = a.z, win[tid][3] = a.w;
+        win[tid][4] = b.x, win[tid][5] = b.y, win[tid][6] = b.z, win[tid][7] = b.w;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < WB; ++k) {
+        const uint32_t word = win[32 * warp + lane][k];  // input row 32 warp + lane, columns 32 k .. 32 k + 31
+        uint32_t mine = 0;
+#pragma unroll
+        for (int bpos = 0; bpos < 32; ++bpos) {
+            const uint32_t col = __ballot_sync(0xffffffffu, (word >> bpos) & 1u);  // column 32 k + bpos of the 32 rows
+            if (lane == bpos) mine = col;
+        }
+        wout[32 * k + lane][warp] = mine;  // output row 32 k + lane, columns 32 warp .. 32 warp + 31
+    }
+    __syncthreads();
+    {
+        const int row = TR * kMirrorBits + tid;
+        if (row < V) {
+            uint4 *dst = reinterpret_cast<uint4 *>(bits + (size_t)row * W + (size_t)TC * WB);
+            dst[0] = make_uint4(wout[tid][0], wout[tid][1], wout[tid][2], wout[tid][3]);
+            dst[1] = make_uint4(wout[tid][4], wout[tid][5], wout[tid][6], wout[tid][7]);
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------- rows
@@ -740,6 +790,8 @@ extern "C" pcg_status pcg_asg_create(const void *emb, pcg_dtype dtype, int32_t V
         const int ntiles = (Vp / kTcRows) * (Vp / kTcTile);
         asg_similarity_tc_kernel<<<std::min(sms, std::max(1, ntiles)), kTcThreads, smem>>>(tmap, rnorm, V, Vp, dp, theta, W,
                                                                                           bits, maxes + 2);
+        const int nT = Vp / kMirrorBits;
+        if (nT > 1) asg_mirror_kernel<<<dim3(nT, nT), kMirrorBits>>>(bits, V, W);
     }
     cudaEventRecord(ev[2], 0);
     {

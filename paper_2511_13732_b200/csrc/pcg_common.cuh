@@ -63,11 +63,10 @@ struct pcg_groups {
     float accept_bias;      // constant added to the acceptance ratio (0 = PCG)
     bool has_sweep;         // the token-sliced sweep layout exists (M <= 65534 and it fits in shared memory)
     // scratch of the batched route of pcg_group_probs (inside `allocation`): rows are processed in chunks of
-    // probs_chunk; the transposed operand Dt[V, probs_chunk], per-row statistics and a row of zeros
+    // probs_chunk; the transposed operand Dt[V, probs_chunk] and per-row statistics
     int probs_chunk;
     float *probs_dt;
     float4 *probs_stats;
-    int32_t *probs_zero;
 };
 
 namespace pcg {
@@ -77,6 +76,13 @@ pcg_status cuda_fail(cudaError_t e, const char *what);
 
 inline bool valid_dtype(pcg_dtype d) { return d == PCG_F32 || d == PCG_BF16 || d == PCG_F16; }
 inline size_t dtype_bytes(pcg_dtype d) { return d == PCG_F32 ? 4 : 2; }
+
+// Rows per chunk of the batched route of pcg_group_probs: 128, or 256 while the transposed operand of a chunk
+// (4 * V bytes per row) stays within 64 MB, so that it remains L2-resident.
+inline int probs_chunk_rows(int V) {
+    const int64_t fit = ((int64_t)64 << 20) / ((int64_t)V * 4) / 128 * 128;
+    return (int)(fit < 128 ? 128 : (fit > 256 ? 256 : fit));
+}
 
 // Runs `...` with LogitT bound to the element type of `dtype` (float, uint16_t for bfloat16 bit patterns, f16_t).
 #define PCG_DISPATCH_DTYPE(dtype, ...)        \

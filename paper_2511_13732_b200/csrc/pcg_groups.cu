@@ -312,9 +312,8 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     for (size_t k = 0; k < part_ptr.size(); ++k) part_ent[k] = gptr[part_ptr[k]];
     const size_t o_part = cv.take(part_ptr.size() * 4), o_pent = cv.take(part_ent.size() * 4);
     // scratch of the batched route of pcg_group_probs: 128 rows per chunk, more while Dt stays within 64 MB
-    int probs_chunk = (int)std::min<int64_t>(256, std::max<int64_t>(128, ((int64_t)64 << 20) / ((int64_t)V * 4) / 128 * 128));
+    const int probs_chunk = probs_chunk_rows(V);
     const size_t o_pdt = cv.take((size_t)V * probs_chunk * 4), o_pst = cv.take((size_t)probs_chunk * 16);
-    const size_t o_pz = cv.take((size_t)probs_chunk * 4);
     const size_t total = cv.off ? cv.off : 256;
     void *mem = nullptr;
     if (!have_device) {
@@ -336,7 +335,6 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     if (e == cudaSuccess) e = upload(base, o_rw, rw);
     if (e == cudaSuccess) e = upload(base, o_part, part_ptr);
     if (e == cudaSuccess) e = upload(base, o_pent, part_ent);
-    if (e == cudaSuccess) e = cudaMemset(base + o_pz, 0, (size_t)probs_chunk * 4);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         cudaFree(mem);
@@ -379,7 +377,6 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     h->probs_chunk = probs_chunk;
     h->probs_dt = (float *)(base + o_pdt);
     h->probs_stats = (float4 *)(base + o_pst);
-    h->probs_zero = (int32_t *)(base + o_pz);
     *out = h;
     return PCG_OK;
 }

@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
     constexpr int U = kBatch;
     constexpr int kChainSteps = 6;
     __shared__ float red_z[4 * NW];
-    __shared__ float red_s[2 * NW];
+    __shared__ float red_s[1];
     const int tid = threadIdx.x;
     const int V = G.V, K = a.K;
     const float s = a.s;
@@ -216,7 +216,9 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
     const float *u = a.uniforms + ((int64_t)b * (K + 1) + i) * 2;
     const uint64_t pol = l2_evict_first_policy();
 
-    // ---- dependent-load chain towards the label group's logits (every thread, redundantly) ----
+    // ---- dependent-load chain towards the label group's logits: WARP 0 only (lane k takes the group's k-th token;
+    // the other warps' streaming loops stay free of it) ----
+    const bool chain_warp = tid < 32;
     int c_x = 0, c_r0 = 0, c_n = 1, c_g = 0, c_lo = 0, c_hi = 0, c_t = 0, c_flag = 0;
     float c_u0 = 0.f, c_u1 = 0.f, c_lp = kNegInf, c_lq = kNegInf, c_w = 0.f;
     auto chain = [&](int step) {
@@ -282,7 +284,10 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
 #pragma unroll
                 for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * NT, pol);
             }
-            if (chained < kChainSteps) chain(chained++);
+            if (chained < kChainSteps) {
+                if (chain_warp) chain(chained);
+                ++chained;
+            }
 #pragma unroll
             for (int j = 0; j < U; ++j) {
                 float v[NV];
@@ -326,46 +331,40 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
     reduce_row(st, red_z, rs_p, Zp);
     st = RefSum{kRefInit * s, 0.f};
     stream_row(qrow, st);
-    while (chained < kChainSteps) chain(chained++);
+    if (chain_warp)
+        while (chained < kChainSteps) chain(chained++);
     reduce_row(st, red_z + 2 * NW, rs_q, Zq);
 
-    // ---- masses of the label group under the two rows (first element prefetched by the chain) ----
-    float part_p = __fmul_rn(ex2(__fmaf_rn(c_lp, s, -rs_p)), c_w);
-    float part_q = __fmul_rn(ex2(__fmaf_rn(c_lq, s, -rs_q)), c_w);
-    for (int k = c_lo + tid + NT; k < c_hi; k += NT) {  // groups larger than a block
-        const int t = G.group_tok[k];
-        const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
-        part_p += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs_p)), w);
-        part_q += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), s, -rs_q)), w);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        part_p += __shfl_xor_sync(0xffffffffu, part_p, o);
-        part_q += __shfl_xor_sync(0xffffffffu, part_q, o);
-    }
-    if ((tid & 31) == 0) {
-        red_s[tid >> 5] = part_p;
-        red_s[NW + (tid >> 5)] = part_q;
-    }
-    __syncthreads();
-
-    if (tid == 0) {
-        float Sp = red_s[0], Sq = red_s[NW];
-        for (int w = 1; w < NW; ++w) {
-            Sp += red_s[w];
-            Sq += red_s[NW + w];
+    // ---- masses of the label group under the two rows, by warp 0 (the first 32 tokens were prefetched by the
+    // chain), then the accept test ----
+    if (chain_warp) {
+        float part_p = __fmul_rn(ex2(__fmaf_rn(c_lp, s, -rs_p)), c_w);
+        float part_q = __fmul_rn(ex2(__fmaf_rn(c_lq, s, -rs_q)), c_w);
+        for (int k = c_lo + tid + 32; k < c_hi; k += 32) {  // groups of more than 32 tokens
+            const int t = G.group_tok[k];
+            const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
+            part_p += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), s, -rs_p)), w);
+            part_q += __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), s, -rs_q)), w);
         }
-        // acceptance u < min(1, P/Q) without a division: P = Sp/Zp, Q = Sq/Zq
-        const float lhs = Sp * Zq, rhs = Sq * Zp;
-        const int acc = (lhs >= rhs) || (c_u1 * rhs < __fmaf_rn(a.bias, rhs, lhs));
-        int flag = c_flag;
-        if (!(Zp > 0.f) || !(Zq > 0.f) || isinf(Zp) || isinf(Zq) || isinf(rs_p) || isinf(rs_q))
-            flag |= PCG_FLAG_NONFINITE;
-        a.accept[pos] = acc;
-        a.labels[pos] = c_g;
-        a.posflags[pos] = flag;
-        a.stats[pos] = make_float4(rs_p, 1.0f / Zp, rs_q, 1.0f / Zq);
-        red_s[0] = acc ? 1.f : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            part_p += __shfl_xor_sync(0xffffffffu, part_p, o);
+            part_q += __shfl_xor_sync(0xffffffffu, part_q, o);
+        }
+        if (tid == 0) {
+            const float Sp = part_p, Sq = part_q;
+            // acceptance u < min(1, P/Q) without a division: P = Sp/Zp, Q = Sq/Zq
+            const float lhs = Sp * Zq, rhs = Sq * Zp;
+            const int acc = (lhs >= rhs) || (c_u1 * rhs < __fmaf_rn(a.bias, rhs, lhs));
+            int flag = c_flag;
+            if (!(Zp > 0.f) || !(Zq > 0.f) || isinf(Zp) || isinf(Zq) || isinf(rs_p) || isinf(rs_q))
+                flag |= PCG_FLAG_NONFINITE;
+            a.accept[pos] = acc;
+            a.labels[pos] = c_g;
+            a.posflags[pos] = flag;
+            a.stats[pos] = make_float4(rs_p, 1.0f / Zp, rs_q, 1.0f / Zq);
+            red_s[0] = acc ? 1.f : 0.f;
+        }
     }
     if (a.bonus_stats && i == K - 1) {  // block-uniform: the last drafted position of its sequence
         __syncthreads();
@@ -942,7 +941,8 @@ struct TransposeArgs {
     float s;
     // The terminal position of a sequence comes from the accept bits of the position kernel (from_accept = 1: this
     // kernel finds the first rejection itself and leaves term_n / term_flags / term_stats for the kernels behind
-    // it), or is read from term_n / term_stats as filled by an earlier kernel (from_accept = 0).
+    // it), or is read from term_n / term_stats as filled by an earlier kernel (from_accept = 0), or is row 0 of a
+    // plain batch of rows whose statistics are in term_stats (from_accept = 2, with K = 0: pcg_group_probs).
     int from_accept;
     const int32_t *accept, *posflags;  // [B*K]
     const float4 *stats;               // [B*K]
@@ -1034,8 +1034,8 @@ __global__ void __launch_bounds__(kTrThreads, 2) residual_transpose_kernel(Trans
         int n = -1, flags = 0;
         float4 st = make_float4(0.f, 0.f, 0.f, 0.f);
         if (b < a.B) {
-            if (!a.from_accept) {
-                n = a.term_n[b];
+            if (a.from_accept != 1) {
+                n = a.from_accept == 2 ? 0 : a.term_n[b];
                 st = a.term_stats[b];
             } else {
                 n = K;
@@ -1892,6 +1892,7 @@ struct VerifyWorkspace {
     float *Dt, *Rt, *Psum;  // default mode
     float *Pws, *Qws;       // dense mode
     float *own_rows;        // dense mode, M beyond the draw kernel's shared memory
+    void *probs_scratch;    // dense mode: scratch of the two group-probability passes
     size_t bytes;
 };
 
@@ -1916,6 +1917,7 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
         w.Pws = (float *)(p + take((size_t)(B * (K + 1) * M) * 4));
         w.Qws = (float *)(p + take((size_t)(B * K * M) * 4));
         if (draw_smem_bytes((int)M) > kMaxDynSmem) w.own_rows = (float *)(p + take((size_t)(B * M) * 4));
+        w.probs_scratch = p + take(pcg_group_probs_workspace_bytes((int32_t)V));
     } else if (mode != PCG_VERIFY_CLUSTER_TERMINAL) {
         const int64_t chunk = terminal_chunk((int)B, (int)V);
         const int64_t chunks = (B + chunk - 1) / chunk;
@@ -1960,32 +1962,50 @@ static cudaError_t launch_spmm(const SpmmArgs &sp, int nb, int lanes, const Grou
 
 using namespace pcg;
 
-extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64_t rows, float temperature,
-                                      const pcg_groups *groups, float *out, pcg_stream stream) {
-    pcg_status st = check_common(groups, dtype, temperature, "pcg_group_probs");
+namespace pcg {
+struct ProbsScratch {
+    float4 *stats;  // [chunk]
+    float *dt;      // [chunk / 32][V][32]
+    size_t bytes;
+};
+static ProbsScratch carve_probs_scratch(void *base, int V) {
+    const size_t chunk = (size_t)probs_chunk_rows(V);
+    ProbsScratch w;
+    char *p = (char *)base;
+    w.stats = (float4 *)p;
+    const size_t off = (chunk * 16 + 255) & ~(size_t)255;
+    w.dt = (float *)(p + off);
+    w.bytes = off + (((size_t)V * chunk * 4 + 255) & ~(size_t)255);
+    return w;
+}
+
+static pcg_status group_probs_impl(const void *logits, pcg_dtype dtype, int64_t rows, float temperature,
+                                   const pcg_groups *groups, float *out, const ProbsScratch *scratch, cudaStream_t cs,
+                                   const char *who) {
+    pcg_status st = check_common(groups, dtype, temperature, who);
     if (st != PCG_OK) return st;
     if (rows < 0 || (rows > 0 && (!logits || !out))) {
-        set_error("pcg_group_probs: null pointer or negative row count");
+        set_error("%s: null pointer or negative row count", who);
         return PCG_ERR_INVALID_ARG;
     }
     if (rows == 0) return PCG_OK;
     const GroupsDev &G = groups->dev;
     if (rows * (int64_t)G.slices > INT32_MAX) {
-        set_error("pcg_group_probs: too many rows for one launch");
+        set_error("%s: too many rows for one launch", who);
         return PCG_ERR_UNSUPPORTED;
     }
     const float s = (float)((double)kLog2e / (double)temperature);
-    cudaStream_t cs = (cudaStream_t)stream;
     cudaError_t e;
     if (rows >= kProbsBatchedRows || !groups->has_sweep) {
         // many rows: the same transposed-operand / sparse-product kernels as the per-sequence stage of pcg_verify,
-        // a chunk of rows at a time through the handle's scratch (row statistics, then p(t) w in place of p - q)
-        const int chunk = groups->probs_chunk;  // a multiple of 128
+        // a chunk of rows at a time through the scratch (row statistics, then p(t) w in place of p - q)
+        const int chunk = probs_chunk_rows(G.V);  // a multiple of 128
         for (int64_t r0 = 0; r0 < rows; r0 += chunk) {
             const int nr = (int)std::min<int64_t>(chunk, rows - r0);
             const char *base = (const char *)logits + (size_t)r0 * G.V * dtype_bytes(dtype);
-            PCG_DISPATCH_DTYPE(dtype, launch_after(row_stats_kernel<LogitT>, dim3((unsigned)nr), dim3(kPrepThreads), 0, cs,
-                                                   (const void *)base, s, groups->probs_stats, G));
+            PCG_DISPATCH_DTYPE(dtype, e = launch_after(row_stats_kernel<LogitT>, dim3((unsigned)nr), dim3(kPrepThreads), 0, cs,
+                                                       (const void *)base, s, scratch->stats, G));
+            if (e != cudaSuccess) return cuda_fail(e, "launching row_stats_kernel");
             const int lanes = (chunk % 256 == 0 && nr >= 256) ? 8 : kSpmmWide;      // rows per lane of the sparse product
             const int nb = (nr + 32 * lanes - 1) / (32 * lanes) * lanes;          // batches of 32 rows, whole warps of it
             // every row is "a sequence whose only row is accepted": K = 0 makes the kernel form p alone
@@ -1993,16 +2013,14 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
             tr.target = tr.draft = base;
             tr.B = nr;
             tr.s = s;
-            tr.term_n = groups->probs_zero;
-            tr.term_stats = groups->probs_stats;
-            tr.Dt = groups->probs_dt;
+            tr.from_accept = 2;
+            tr.term_stats = scratch->stats;
+            tr.Dt = scratch->dt;
             PCG_DISPATCH_DTYPE(dtype, e = launch_transpose<LogitT>(tr, nb, G, groups->sm_count, cs));
             if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
-            e = launch_spmm<true>(SpmmArgs{groups->probs_dt, nr, 0, chunk, out + (size_t)r0 * G.M, nullptr}, nb, lanes, G, cs);
+            e = launch_spmm<true>(SpmmArgs{scratch->dt, nr, 0, chunk, out + (size_t)r0 * G.M, nullptr}, nb, lanes, G, cs);
             if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
         }
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return cuda_fail(e, "launching the batched group-probability kernels");
         return PCG_OK;
     }
     ProbsArgs a{logits, out, s};
@@ -2010,6 +2028,37 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
                                                  groups->agg_smem_bytes, cs, a, G));
     if (e != cudaSuccess) return cuda_fail(e, "launching group_probs_kernel");
     return PCG_OK;
+}
+}  // namespace pcg
+
+extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64_t rows, float temperature,
+                                      const pcg_groups *groups, float *out, pcg_stream stream) {
+    ProbsScratch own = {};
+    if (groups) {  // the scratch that belongs to the handle
+        own.stats = groups->probs_stats;
+        own.dt = groups->probs_dt;
+    }
+    return group_probs_impl(logits, dtype, rows, temperature, groups, out, &own, (cudaStream_t)stream, "pcg_group_probs");
+}
+
+extern "C" size_t pcg_group_probs_workspace_bytes(int32_t V) {
+    return V < 1 ? 256 : carve_probs_scratch(nullptr, V).bytes;
+}
+
+extern "C" pcg_status pcg_group_probs_ws(const void *logits, pcg_dtype dtype, int64_t rows, float temperature,
+                                         const pcg_groups *groups, float *out, void *workspace, size_t workspace_bytes,
+                                         pcg_stream stream) {
+    if (!groups) {
+        set_error("pcg_group_probs_ws: null group handle");
+        return PCG_ERR_INVALID_ARG;
+    }
+    const size_t need = pcg_group_probs_workspace_bytes(groups->dev.V);
+    if (!workspace || ((uintptr_t)workspace & 255u) || workspace_bytes < need) {
+        set_error("pcg_group_probs_ws: workspace must be 256-byte aligned and hold %zu bytes (got %zu)", need, workspace_bytes);
+        return PCG_ERR_WORKSPACE;
+    }
+    const ProbsScratch ws = carve_probs_scratch(workspace, groups->dev.V);
+    return group_probs_impl(logits, dtype, rows, temperature, groups, out, &ws, (cudaStream_t)stream, "pcg_group_probs_ws");
 }
 
 extern "C" size_t pcg_verify_workspace_bytes(int32_t B, int32_t K, int32_t V, int32_t M, pcg_dtype dtype,
@@ -2084,8 +2133,9 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
     // ---- per-position stage: statistics, label, accept bit ----
     if (dense) {
         // P and Q of ALL groups at EVERY position, then the accept test on the stored masses
-        pcg_status st2 = pcg_group_probs(target_logits, dtype, (int64_t)B * (K + 1), temperature, groups, w.Pws, stream);
-        if (st2 == PCG_OK) st2 = pcg_group_probs(draft_logits, dtype, (int64_t)B * K, temperature, groups, w.Qws, stream);
+        const ProbsScratch ps = carve_probs_scratch(w.probs_scratch, G.V);
+        pcg_status st2 = group_probs_impl(target_logits, dtype, (int64_t)B * (K + 1), temperature, groups, w.Pws, &ps, cs, "pcg_verify");
+        if (st2 == PCG_OK) st2 = group_probs_impl(draft_logits, dtype, (int64_t)B * K, temperature, groups, w.Qws, &ps, cs, "pcg_verify");
         if (st2 != PCG_OK) return st2;
         DenseAcceptArgs da{draft_tokens, uniforms, B, K, w.Pws, w.Qws, groups->accept_bias, w.accept, w.labels, w.posflags};
         dense_accept_kernel<<<(B * K + 127) / 128, 128, 0, cs>>>(da, G);

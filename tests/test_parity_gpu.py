@@ -66,6 +66,21 @@ def test_group_probs_batched_route(oracle, name, rows):
     np.testing.assert_allclose(got.sum(axis=1), 1.0, rtol=4e-6)
     again = binding.pcg_group_probs(logits_to_device(x), h, cfg.temperature).cpu().numpy()
     assert np.array_equal(again.astype(np.float64), got)  # bit-reproducible
+    # the caller-workspace form: same numbers; two calls with separate workspaces on two streams do not disturb each other
+    xd = logits_to_device(x)
+    ws = [torch.empty(binding.pcg_group_probs_workspace_bytes(cfg.V), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    outs = [torch.empty((rows, groups.M), dtype=torch.float32, device="cuda") for _ in range(2)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for _ in range(3):
+        for k in range(2):
+            with torch.cuda.stream(streams[k]):
+                binding.pcg_group_probs(xd, h, cfg.temperature, out=outs[k], workspace=ws[k], stream=streams[k])
+    torch.cuda.synchronize()
+    assert np.array_equal(outs[0].cpu().numpy(), again) and np.array_equal(outs[1].cpu().numpy(), again)
+    with pytest.raises(binding.PcgError) as ei:
+        binding.pcg_group_probs(xd, h, cfg.temperature, workspace=ws[0][:1024])
+    assert ei.value.status == 4
     # with general weights
     rng = np.random.default_rng(3)
     raw = rng.random(groups.nnz) + 0.05
