@@ -213,10 +213,7 @@ __global__ void __launch_bounds__(kAsgThreads) asg_similarity_kernel(const __nv_
 constexpr int kTcBK = 64;        // bf16 per row and stage
 constexpr int kTcTile = 256;     // columns of a tile (rows of the B operand); Vp is a multiple of it
 constexpr int kTcRows = 128;     // rows of a tile (rows of the A operand) = lanes of tensor memory
-#ifndef PCG_TC_STAGES
-#define PCG_TC_STAGES 4
-#endif
-constexpr int kTcStages = PCG_TC_STAGES;
+constexpr int kTcStages = 4;     // stages of the operand ring
 constexpr int kTcEpilogueWarps = 8, kTcProducerWarps = 1;
 constexpr int kTcRasterRows = 16, kTcRasterCols = 8;  // tiles are visited in blocks of 16 x 8 (see tile_origin)
 constexpr int kTcThreads = 32 * (kTcEpilogueWarps + kTcProducerWarps + 1);

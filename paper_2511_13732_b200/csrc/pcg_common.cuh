@@ -155,10 +155,8 @@ struct Elem<f16_t> {
 // do the same with respect to this one, then waits until the previous grid has completed and its writes are
 // visible.  Nothing a previous kernel wrote may be read before it.  Without the launch attribute both are no-ops.
 __device__ __forceinline__ void pdl_enter() {
-#ifndef PCG_NO_PDL
     asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
 }
 
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {

@@ -1,6 +1,6 @@
 // Kernels and entry points of libpcg: PCG group-level verification on sm_100a.
 //
-//   position_kernel  one thread block per drafted position (b,i).  Streams the target and the draft row once
+//   position_kernel  one thread block per drafted position (b,i).  Streams the target row, then the draft row
 //                    (softmax statistics with a lazy reference, 128-bit loads), draws the group label of the draft
 //                    token, forms the label group's target and draft mass from a handful of gathered logits and
 //                    takes the accept decision.  This kernel moves ~all of the bytes.
@@ -8,11 +8,13 @@
 // draw, token draw, outputs) exists in two forms:
 //   terminal_kernel  one thread-block cluster per sequence: a token-sliced segmented reduction in shared memory,
 //                    slices combined over distributed shared memory (a handful of sequences: lowest latency).
-//   batched          terminal_prepare_kernel, residual_transpose_kernel, group_spmm_kernel, terminal_draw_kernel:
-//                    the residual of all sequences as one sparse product over a transposed, L2-resident operand.
-// pcg_group_probs writes P of every row with the same two aggregations; pcg_verify_thinning replaces the
-// per-sequence stage by thinning_kernel (pcg_thinning.cuh), which enumerates nothing.  Every kernel after the
-// first of a call is launched with programmatic stream serialisation (pdl_enter, launch_after).
+//   batched          residual_transpose_kernel (which also finds the first rejections), group_spmm_kernel,
+//                    terminal_pick_kernel: the residual of all sequences as one sparse product over a transposed,
+//                    L2-resident operand.
+// pcg_group_probs writes P of every row with the same two aggregations; dense mode of pcg_verify stores P and Q of
+// every position that way and draws with terminal_prepare_kernel / terminal_draw_kernel; pcg_verify_thinning
+// replaces the per-sequence stage by thinning_kernel (pcg_thinning.cuh), which enumerates nothing.  Every kernel
+// after the first of a call is launched with programmatic stream serialisation (pdl_enter, launch_after).
 #include <cooperative_groups.h>
 
 #include <algorithm>
@@ -24,9 +26,6 @@
 
 namespace cg = cooperative_groups;
 
-#ifndef PCG_STATIC_SCRATCH_BYTES
-#define PCG_STATIC_SCRATCH_BYTES (1u << 20)  // built-in scratch of pcg_verify_static, per GPU
-#endif
 
 namespace pcg {
 
@@ -206,9 +205,17 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
     // Block order: the LAST drafted position of every sequence first (blocks 0 .. B-1), then the others.  Those
     // blocks may have a third row to stream (the bonus row, see PositionArgs::bonus_stats); up front that extra
     // work is spread over the first wave instead of lengthening the tail of the kernel.
+    // (Without bonus rows -- the cluster terminal and the thinning entry point fetch them themselves -- the blocks
+    // simply follow the positions: measured 3 us faster at B = 256, K = 16, V = 65536.)
     const int nseq = (int)gridDim.x / K;
-    const int b = (int)blockIdx.x < nseq ? (int)blockIdx.x : ((int)blockIdx.x - nseq) / (K - 1);
-    const int i = (int)blockIdx.x < nseq ? K - 1 : ((int)blockIdx.x - nseq) - b * (K - 1);
+    int b, i;
+    if (a.bonus_stats) {
+        b = (int)blockIdx.x < nseq ? (int)blockIdx.x : ((int)blockIdx.x - nseq) / (K - 1);
+        i = (int)blockIdx.x < nseq ? K - 1 : ((int)blockIdx.x - nseq) - b * (K - 1);
+    } else {
+        b = (int)blockIdx.x / K;
+        i = (int)blockIdx.x - b * K;
+    }
     const int pos = b * K + i;
     pdl_enter();  // (the first kernel of a call: lets the kernel behind it be scheduled while this one drains)
     const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + i) * V;
@@ -1809,14 +1816,10 @@ static cudaError_t launch_after(void (*kern)(KArgs...), dim3 grid, dim3 block, s
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
-    int nattr = 0;
-#ifndef PCG_NO_PDL
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    nattr = 1;
-#endif
     cfg.attrs = attr;
-    cfg.numAttrs = nattr;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
@@ -2323,7 +2326,7 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
 // exits.  In host code `g_static_scratch` is only a stand-in for the symbol, never a device address; the
 // address a kernel may use comes from cudaGetSymbolAddress, asked once per device and remembered here.
 namespace pcg {
-constexpr size_t kStaticScratchBytes = PCG_STATIC_SCRATCH_BYTES;
+constexpr size_t kStaticScratchBytes = (size_t)1 << 20;  // built-in scratch of pcg_verify_static, per GPU
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 constexpr int kMaxStaticDevices = 64;
 static void *g_static_scratch_addr[kMaxStaticDevices];  // zero-initialised; written once per device

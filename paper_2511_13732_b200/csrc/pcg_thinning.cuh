@@ -216,12 +216,9 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
     const bool usable = Ztot > 0.0 && Ztot < (double)__builtin_huge_valf();
     if (!usable) flags |= PCG_FLAG_NONFINITE;
     const int max_trials = usable ? (residual ? a.n_trials : 1) : 0;
-#ifndef PCG_THIN_FIRST_ROUND
-#define PCG_THIN_FIRST_ROUND 8
-#endif
     // trials of the first round (every trial reads its slot's words, scattered over the whole row: fewer side by
     // side means less traffic, more means fewer sequences need a second round)
-    constexpr int kFirstRound = PCG_THIN_FIRST_ROUND;
+    constexpr int kFirstRound = 8;
     for (int r0 = 0, width = kFirstRound; r0 < max_trials && gsel < 0; r0 += width, width = NW) {
         const int r = r0 + warp;
         int kept = -1;
