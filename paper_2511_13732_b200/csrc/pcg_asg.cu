@@ -475,8 +475,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) asg_similarity_tc_kernel(const 
 
 // The lower triangle of the bit matrix from the upper one (cos is symmetric, so t' in G(t) iff t in G(t')): the
 // block of 256 rows x 256 columns at (TR, TC), TC < TR, is the transpose of the block at (TC, TR).  One thread block
-// per such pair: 256 rows x 32 bytes in (whole sectors), the 256 x 256 bits turned with warp ballots (lane = input
-// row; one ballot per bit position gives a word of the output row of that position), 256 rows x 32 bytes out.
+// per such pair: 256 rows x 32 bytes in (whole sectors), the 256 x 256 bits turned 32 x 32 at a time by exchanges
+// between lanes (lane = input row before, output row after), 256 rows x 32 bytes out.
 constexpr int kMirrorBits = 256;
 static_assert(kMirrorBits == kTcTile, "the tensor-core kernel computes whole diagonal blocks of this size");
 __global__ void __launch_bounds__(kMirrorBits) asg_mirror_kernel(uint32_t *bits, int V, int W) {
@@ -499,14 +499,16 @@ __global__ void __launch_bounds__(kMirrorBits) asg_mirror_kernel(uint32_t *bits,
     __syncthreads();
 #pragma unroll
     for (int k = 0; k < WB; ++k) {
-        const uint32_t word = win[32 * warp + lane][k];  // input row 32 warp + lane, columns 32 k .. 32 k + 31
-        uint32_t mine = 0;
+        // lane = input row 32 warp + lane, bits = columns 32 k .. 32 k + 31: the 32 x 32 bit block is transposed across
+        // the lanes in five exchange steps (blocks of 16, 8, 4, 2, 1 swapped across the diagonal)
+        uint32_t x = win[32 * warp + lane][k];
 #pragma unroll
-        for (int bpos = 0; bpos < 32; ++bpos) {
-            const uint32_t col = __ballot_sync(0xffffffffu, (word >> bpos) & 1u);  // column 32 k + bpos of the 32 rows
-            if (lane == bpos) mine = col;
+        for (int j = 16; j > 0; j >>= 1) {
+            const uint32_t m = j == 16 ? 0x0000ffffu : j == 8 ? 0x00ff00ffu : j == 4 ? 0x0f0f0f0fu : j == 2 ? 0x33333333u : 0x55555555u;
+            const uint32_t partner = __shfl_xor_sync(0xffffffffu, x, j);
+            x = (lane & j) ? ((x & ~m) | ((partner & ~m) >> j)) : ((x & m) | ((partner & m) << j));
         }
-        wout[32 * k + lane][warp] = mine;  // output row 32 k + lane, columns 32 warp .. 32 warp + 31
+        wout[32 * k + lane][warp] = x;  // output row 32 k + lane, columns 32 warp .. 32 warp + 31
     }
     __syncthreads();
     {
