@@ -267,6 +267,25 @@ def quick_workload(binding, torch, wcfg, peak, steps=300):
         gbs = B * (2 * K + 1) * V * esz / (ms * 1e-3) / 1e9
         res[key] = {"ms_per_step": ms, "steps": steps, "value": B * K / (ms * 1e-3), "unit": UNIT,
                     "whole_step_gbs": gbs, "whole_step_frac_of_measured_peak": gbs / peak}
+        # the same call captured in a CUDA graph and replayed: the device-side time without the host's launch work
+        # (at these sizes the Python caller, not the GPU, paces the plain calls)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            one(0)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            one(0)
+        for _ in range(3):
+            graph.replay()
+        e0.record()
+        for _ in range(steps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        res[key]["cuda_graph_replay_ms_per_step"] = e0.elapsed_time(e1) / steps
     handle.close()
     return res
 
