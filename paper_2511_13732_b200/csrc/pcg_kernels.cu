@@ -49,7 +49,9 @@ constexpr size_t kMaxDynSmem = 227 * 1024;  // dynamic shared memory a block may
 // logits (token -> its groups -> label -> group's token list -> logits) is spread over the streaming loop, one hop
 // per batch, so its latency is hidden.
 
-constexpr int kPosThreads = 256;
+constexpr int kPosThreads = 256;       // threads of a position block for long rows ...
+constexpr int kPosThreadsSmall = 128;  // ... and for rows of at most kPosSmallRowBytes (more batches per row, more blocks per SM)
+constexpr size_t kPosSmallRowBytes = 64 * 1024;
 constexpr int kBatch = 4;
 constexpr float kRefInit = -1.0e30f;     // "no logit seen yet": finite, so that -inf logits give 2^-inf = 0, not NaN
 constexpr float kVecSumLimit = 4294967296.f;  // 2^32
@@ -109,8 +111,8 @@ struct PositionArgs {
     int32_t *labels;         // [B*K] group label of the draft token
     int32_t *posflags;       // [B*K]
     float4 *stats;           // [B*K] (RS_p, 1/Z_p, RS_q, 1/Z_q): scaled reference and reciprocal normaliser
-    float2 *strata;          // [B*K, kPosThreads] or null: every thread's own (reference, sum) of the target row; thread h
-                             // has summed its 16-byte words h, h + 256, h + 512, ... (see pcg_thinning.cuh)
+    float2 *strata;          // [B*K, NT] or null: every thread's own (reference, sum) of the target row; thread h of the
+                             // block's NT has summed its 16-byte words h, h + NT, h + 2 NT, ... (see pcg_thinning.cuh)
     float4 *bonus_stats;     // [B] or null: (RS, 1/Z, 0, 0) of the bonus row (target row K), written by the block of a
                              // sequence's LAST drafted position if that position was accepted (no sequence that
                              // needs its bonus row can have its last position rejected)
@@ -146,9 +148,9 @@ __device__ __forceinline__ int draw_label(const GroupsDev &G, int r0, int n, flo
 
 // Softmax statistics of one row by the whole block (the bonus row of a sequence whose last drafted position was
 // accepted).  Kept out of line so that the streaming loop of the position kernel keeps its registers.
-template <typename T>
+template <typename T, int NT>
 __device__ __noinline__ void bonus_row_stats(const T *row, int V, float s, float *red, float4 *stats_out, int32_t *flags_out) {
-    constexpr int NT = kPosThreads, NW = NT / 32, NV = Elem<T>::kPerVec;
+    constexpr int NW = NT / 32, NV = Elem<T>::kPerVec;
     const int tid = threadIdx.x;
     RefSum st{kRefInit * s, 0.f};
     int head = (int)(((16u - (unsigned)((uintptr_t)row & 15u)) & 15u) / sizeof(T));
@@ -191,9 +193,9 @@ __device__ __noinline__ void bonus_row_stats(const T *row, int V, float s, float
     }
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a, GroupsDev G) {
-    constexpr int NT = kPosThreads, NW = NT / 32;
+template <typename T, int NT>
+__global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a, GroupsDev G) {
+    constexpr int NW = NT / 32;
     constexpr int NV = Elem<T>::kPerVec;
     constexpr int U = kBatch;
     constexpr int kChainSteps = 6;
@@ -376,7 +378,7 @@ __global__ void __launch_bounds__(kPosThreads, 4) position_kernel(PositionArgs a
     if (a.bonus_stats && i == K - 1) {  // block-uniform: the last drafted position of its sequence
         __syncthreads();
         if (red_s[0] != 0.f)  // accepted: the sequence may need its bonus row
-            bonus_row_stats<T>(reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + K) * V, V, s, red_z,
+            bonus_row_stats<T, NT>(reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + K) * V, V, s, red_z,
                                a.bonus_stats + b, a.bonus_flags + b);
     }
 }
@@ -1934,6 +1936,18 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
     return w;
 }
 
+// Threads of a position block: rows of at most 64 KB are streamed by 128 threads (four or more batches per row even
+// at V = 16384, so that the dependent-load chain towards the label group stays hidden, and eight blocks per SM).
+static int position_threads(int V, pcg_dtype dtype) {
+    return (size_t)V * dtype_bytes(dtype) <= kPosSmallRowBytes ? kPosThreadsSmall : kPosThreads;
+}
+static void launch_position(pcg_dtype dtype, const PositionArgs &pa, const GroupsDev &G, int positions, cudaStream_t cs) {
+    if (position_threads(G.V, dtype) == kPosThreadsSmall)
+        PCG_DISPATCH_DTYPE(dtype, (position_kernel<LogitT, kPosThreadsSmall><<<positions, kPosThreadsSmall, 0, cs>>>(pa, G)));
+    else
+        PCG_DISPATCH_DTYPE(dtype, (position_kernel<LogitT, kPosThreads><<<positions, kPosThreads, 0, cs>>>(pa, G)));
+}
+
 // The transposed-operand kernel over nb batches of 32 sequences: two resident blocks per SM, shared out
 // over the batches, each walking a run of its batch's rows.
 template <typename T>
@@ -2149,7 +2163,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
                         w.accept,      w.labels,     w.posflags,   w.stats,  nullptr,
                         cluster_terminal ? nullptr : w.bonus_stats, cluster_terminal ? nullptr : w.bonus_flags};
-        PCG_DISPATCH_DTYPE(dtype, position_kernel<LogitT><<<B * K, kPosThreads, 0, cs>>>(pa, G));
+        launch_position(dtype, pa, G, B * K, cs);
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
     }
@@ -2233,7 +2247,7 @@ static ThinWorkspace carve_thin_workspace(void *base, int64_t B, int64_t K, int6
     w.labels = (int32_t *)(p + take((size_t)(B * K) * 4));
     w.posflags = (int32_t *)(p + take((size_t)(B * K) * 4));
     w.fallback_rows = (float *)(p + take((size_t)(B * M) * 4));
-    w.strata = (float2 *)(p + take((size_t)(B * K) * kPosThreads * 8));
+    w.strata = (float2 *)(p + take((size_t)(B * K) * kPosThreads * 8));  // (128 pairs per position are used for short rows)
     w.bytes = off ? off : 256;
     return w;
 }
@@ -2295,7 +2309,7 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
     const bool strata = ((uintptr_t)target_logits & 15u) == 0 && ((size_t)G.V * esz) % 16 == 0;
     PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
                     w.accept,      w.labels,     w.posflags,   w.stats,  strata ? w.strata : nullptr, nullptr, nullptr};
-    PCG_DISPATCH_DTYPE(dtype, position_kernel<LogitT><<<B * K, kPosThreads, 0, cs>>>(pa, G));
+    launch_position(dtype, pa, G, B * K, cs);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
     if (stage_events) {
@@ -2305,7 +2319,7 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
     ThinArgs ta{target_logits, draft_logits, draft_tokens, uniforms,        thin_uniforms, n_trials,
                 K,             s,            w.accept,     w.labels,        w.posflags,    w.stats,
                 w.fallback_rows, out_accept_len, out_tokens, out_groups,    out_flags,     out_trials,
-                strata ? w.strata : nullptr};
+                strata ? w.strata : nullptr, position_threads(G.V, dtype)};
     auto launch = [&](auto kern) -> cudaError_t {
         cudaError_t le = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (le != cudaSuccess) return le;

@@ -35,11 +35,13 @@ struct ThinArgs {
     const float4 *stats;                        // [B*K]
     float *fallback_rows;                       // [B, M] staging for sequences whose trials ran out
     int32_t *out_accept_len, *out_tokens, *out_groups, *out_flags, *out_trials;
-    const float2 *strata;  // [B*K, 2 * kThinSlots] (reference, sum) of every target-row thread of the position kernel, or null
+    const float2 *strata;  // [B*K, strata_threads] (reference, sum) of every thread of the position kernel's target-row pass, or null
+    int strata_threads;    // threads of a position block: kThinSlots or 2 * kThinSlots
 };
 
 constexpr int kThinSlots = 128;  // slots of the candidate order (the interface's rule: slot of token t = (t div W) mod 128)
-static_assert(kPosThreads == 2 * kThinSlots, "a slot is the union of the words of two threads of the position kernel");
+static_assert(kPosThreads == 2 * kThinSlots && kPosThreadsSmall == kThinSlots,
+              "a slot is the words of one thread of the position kernel (short rows) or of two (long rows)");
 static_assert(kThinThreads % kThinSlots == 0, "the block sums the slots with a whole number of threads per slot");
 
 static size_t thin_smem_bytes() {
@@ -172,12 +174,17 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
     // ---- 2. the slot masses of the target row (slot of token t = (t div NV) mod S), then their prefix ----
     float mass = 0.f;  // of slot tid, in threads tid < S
     if (a.strata && residual) {
-        // the position kernel's threads h and h + S summed exactly slot h between them (words h, h + 2S, ... and
-        // h + S, h + 3S, ...), each relative to a reference of its own that is at most the row's final one
+        // the position kernel's thread h (short rows: S threads per block) or its threads h and h + S between them
+        // (long rows: words h, h + 2S, ... and h + S, h + 3S, ...) summed exactly slot h, each relative to a reference
+        // of its own that is at most the row's final one
         if (tid < S) {
-            const float2 v0 = a.strata[(size_t)(b * K + n) * (2 * S) + tid];
-            const float2 v1 = a.strata[(size_t)(b * K + n) * (2 * S) + S + tid];
-            mass = __fmul_rn(v0.y, ex2(v0.x - rs_p)) + __fmul_rn(v1.y, ex2(v1.x - rs_p));
+            const float2 *pairs = a.strata + (size_t)(b * K + n) * a.strata_threads;
+            const float2 v0 = pairs[tid];
+            mass = __fmul_rn(v0.y, ex2(v0.x - rs_p));
+            if (a.strata_threads == 2 * S) {
+                const float2 v1 = pairs[S + tid];
+                mass += __fmul_rn(v1.y, ex2(v1.x - rs_p));
+            }
         }
     } else {
         // SUB threads per slot walk the slot's words, four loads in flight each; partial sums added in fixed order
