@@ -1941,11 +1941,16 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
 static int position_threads(int V, pcg_dtype dtype) {
     return (size_t)V * dtype_bytes(dtype) <= kPosSmallRowBytes ? kPosThreadsSmall : kPosThreads;
 }
+// (Launched with programmatic stream serialisation like the kernels behind it: after whatever precedes the call on
+// the stream -- in a decoding loop the previous call's last kernel -- its blocks are scheduled during that kernel's
+// drain and wait at the top, pdl_enter, until it has completed.)
 static void launch_position(pcg_dtype dtype, const PositionArgs &pa, const GroupsDev &G, int positions, cudaStream_t cs) {
     if (position_threads(G.V, dtype) == kPosThreadsSmall)
-        PCG_DISPATCH_DTYPE(dtype, (position_kernel<LogitT, kPosThreadsSmall><<<positions, kPosThreadsSmall, 0, cs>>>(pa, G)));
+        PCG_DISPATCH_DTYPE(dtype, launch_after(position_kernel<LogitT, kPosThreadsSmall>, dim3((unsigned)positions),
+                                               dim3(kPosThreadsSmall), 0, cs, pa, G));
     else
-        PCG_DISPATCH_DTYPE(dtype, (position_kernel<LogitT, kPosThreads><<<positions, kPosThreads, 0, cs>>>(pa, G)));
+        PCG_DISPATCH_DTYPE(dtype, launch_after(position_kernel<LogitT, kPosThreads>, dim3((unsigned)positions),
+                                               dim3(kPosThreads), 0, cs, pa, G));
 }
 
 // The transposed-operand kernel over nb batches of 32 sequences: two resident blocks per SM, shared out
