@@ -121,7 +121,7 @@ const char *pcg_last_error(void);
  * group id -- the "optional reverse indices" of the same paragraph), the 1/N(t)
  * table and a token-sliced copy of the CSR with 16-bit in-slice token offsets,
  * uploads them and synchronises the device.  The handle also holds the scratch of pcg_group_probs
- * (4 * V * min(256, ...) bytes: 64 MB at V = 65536; pcg_group_probs_ws does not use it).
+ * (4 * (V + M) * min(256, ...) bytes: 80 MB at V = 65536, M = 16384; pcg_group_probs_ws does not use it).
  *
  *   slices_hint: 0 = choose automatically; 1, 2, 4 or 8 = force that many token
  *                slices (= cluster size).  Rounded up if a slice would not fit
@@ -161,14 +161,14 @@ pcg_status pcg_groups_set_accept_bias(pcg_groups *groups, float bias);
  * From 64 rows on the rows go, up to 256 at a time, through scratch memory (a transposed copy of the rows'
  * probabilities).  pcg_group_probs uses scratch that belongs to the handle: two such calls with the SAME handle
  * must not overlap on the device (different streams).  pcg_group_probs_ws is the same call with the scratch
- * supplied by the caller (pcg_group_probs_workspace_bytes(V) bytes, 256-byte aligned, contents irrelevant): calls
+ * supplied by the caller (pcg_group_probs_workspace_bytes(V, M) bytes, 256-byte aligned, contents irrelevant): calls
  * with separate workspaces may overlap freely, the handle is only read.
  * rows == 0 is a no-op.  Errors: INVALID_ARG (null, rows < 0, temperature <= 0 or not finite, bad dtype,
  * wrong device), WORKSPACE (pcg_group_probs_ws: workspace missing, misaligned or too small), CUDA (launch failure).
  */
 pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64_t rows, float temperature,
                            const pcg_groups *groups, float *out, pcg_stream stream);
-size_t pcg_group_probs_workspace_bytes(int32_t V);
+size_t pcg_group_probs_workspace_bytes(int32_t V, int32_t M);
 pcg_status pcg_group_probs_ws(const void *logits, pcg_dtype dtype, int64_t rows, float temperature,
                               const pcg_groups *groups, float *out, void *workspace, size_t workspace_bytes,
                               pcg_stream stream);

@@ -85,7 +85,7 @@ def load(build_if_missing: bool = True):
     lib.pcg_groups_set_accept_bias.argtypes, lib.pcg_groups_set_accept_bias.restype = [vp, f32], ctypes.c_int
     lib.pcg_group_probs.argtypes = [vp, ctypes.c_int, i64, f32, vp, vp, vp]
     lib.pcg_group_probs.restype = ctypes.c_int
-    lib.pcg_group_probs_workspace_bytes.argtypes, lib.pcg_group_probs_workspace_bytes.restype = [i32], sz
+    lib.pcg_group_probs_workspace_bytes.argtypes, lib.pcg_group_probs_workspace_bytes.restype = [i32, i32], sz
     lib.pcg_group_probs_ws.argtypes = [vp, ctypes.c_int, i64, f32, vp, vp, vp, sz, vp]
     lib.pcg_group_probs_ws.restype = ctypes.c_int
     lib.pcg_verify_workspace_bytes.argtypes = [i32, i32, i32, i32, ctypes.c_int, u32]
@@ -178,14 +178,14 @@ class Groups:
             pass
 
 
-def pcg_group_probs_workspace_bytes(V: int) -> int:
-    return int(load().pcg_group_probs_workspace_bytes(int(V)))
+def pcg_group_probs_workspace_bytes(V: int, M: int) -> int:
+    return int(load().pcg_group_probs_workspace_bytes(int(V), int(M)))
 
 
 def pcg_group_probs(logits, groups: Groups, temperature: float = 1.0, out=None, stream=None, workspace=None):
     """``pcg_group_probs``: logits [rows, V] (CUDA, float32, bfloat16 or float16) -> float32 [rows, M].
 
-    With ``workspace`` (a uint8 CUDA tensor of at least ``pcg_group_probs_workspace_bytes(V)`` bytes) the call goes
+    With ``workspace`` (a uint8 CUDA tensor of at least ``pcg_group_probs_workspace_bytes(V, M)`` bytes) the call goes
     through ``pcg_group_probs_ws`` and touches no scratch of the handle, so calls with separate workspaces may run
     side by side on different streams."""
     import torch

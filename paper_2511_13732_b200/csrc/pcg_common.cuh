@@ -67,6 +67,7 @@ struct pcg_groups {
     int probs_chunk;
     float *probs_dt;
     float4 *probs_stats;
+    float *probs_rt;  // [M, probs_chunk] group-major sums of one chunk
 };
 
 namespace pcg {

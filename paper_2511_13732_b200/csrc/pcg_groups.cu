@@ -314,6 +314,7 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     // scratch of the batched route of pcg_group_probs: 128 rows per chunk, more while Dt stays within 64 MB
     const int probs_chunk = probs_chunk_rows(V);
     const size_t o_pdt = cv.take((size_t)V * probs_chunk * 4), o_pst = cv.take((size_t)probs_chunk * 16);
+    const size_t o_prt = cv.take((size_t)M * probs_chunk * 4);
     const size_t total = cv.off ? cv.off : 256;
     void *mem = nullptr;
     if (!have_device) {
@@ -377,6 +378,7 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     h->probs_chunk = probs_chunk;
     h->probs_dt = (float *)(base + o_pdt);
     h->probs_stats = (float4 *)(base + o_pst);
+    h->probs_rt = (float *)(base + o_prt);
     *out = h;
     return PCG_OK;
 }

@@ -1173,8 +1173,8 @@ struct SpmmArgs {
     int B;
     int b0;           // first sequence of this chunk
     int bpad;         // sequences per row of Rt and Psum (the chunk size, a multiple of 32 * SPL)
-    float *R;         // ROWMAJOR: [B, M] raw sums by sequence (pcg_group_probs); else Rt [M, bpad] by group
-    float *Psum;      // [nparts, bpad]: per part, the sum of the positive parts of its groups' sums (not ROWMAJOR)
+    float *R;         // Rt [M, bpad]: raw sums by group
+    float *Psum;      // [nparts, bpad]: per part, the sum of the positive parts of its groups' sums (PSUM only)
 };
 
 template <int SPL>
@@ -1216,17 +1216,14 @@ struct SeqVec<8> {  // one 256-bit load per lane
 // keeps up to 2 * DEPTH lines of Dt in flight at all times.  Token ids are fetched 32 at a time, one block of 32
 // ahead.  Sums run in CSR order; a group ends where the running entry index reaches the next group pointer.
 // Output by group (verification): a closed group's SPL sums go straight to Rt[g, sequences], their positive
-// parts are added up per part and written to Psum[part, sequences].  ROWMAJOR output (pcg_group_probs): the
-// part's sums are turned in shared memory and written along the group index, R[sequence, g].
-template <int SPL, int DEPTH, bool HAS_W, bool ROWMAJOR>
-__global__ void __launch_bounds__(kSpmmThreads, ROWMAJOR ? 4 : 5) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
+// parts are added up per part and written to Psum[part, sequences] (PSUM; pcg_group_probs needs no part sums and
+// turns Rt into its row-major output with rows_from_groups_kernel).
+template <int SPL, int DEPTH, bool HAS_W, bool PSUM>
+__global__ void __launch_bounds__(kSpmmThreads, 5) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
     pdl_enter();
     constexpr int NS = 32 * SPL;  // sequences per warp
-    constexpr int TS = NS + 4;    // row stride of the result tile (keeps 16-byte alignment, spreads banks)
     static_assert(32 % DEPTH == 0 && DEPTH <= 16, "a batch never straddles two blocks of 32 token ids");
-    __shared__ __align__(16) float tiles[ROWMAJOR ? (kSpmmThreads / 32) * kPartMaxGroups * TS : 4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float *tile = tiles + (ROWMAJOR ? warp * kPartMaxGroups * TS : 0);
     const int part = blockIdx.x * (kSpmmThreads / 32) + warp;
     if (part >= G.nparts) return;  // warp-uniform; the kernel has no block-wide barrier
     // the part's groups and stored pairs (both pairs of bounds in one round trip, so that the group pointers and
@@ -1269,11 +1266,8 @@ __global__ void __launch_bounds__(kSpmmThreads, ROWMAJOR ? 4 : 5) group_spmm_ker
     int gend = __shfl_sync(0xffffffffu, ptr_l, 1);
     auto close_groups = [&](int k) {  // the entry index reached k: close every group that ends at or before k
         while (gi < ng && gend <= k) {
-            if (ROWMAJOR) {
-#pragma unroll
-                for (int q = 0; q < SPL; ++q) tile[gi * TS + lane * SPL + q] = acc.v[q];
-            } else {
-                acc.store(a.R + (size_t)(g0 + gi) * a.bpad + sq0);
+            acc.store(a.R + (size_t)(g0 + gi) * a.bpad + sq0);
+            if (PSUM) {
 #pragma unroll
                 for (int q = 0; q < SPL; ++q) pos.v[q] += fmaxf(acc.v[q], 0.f);  // (P - Q)_+ ; NaN counts as 0
             }
@@ -1333,15 +1327,23 @@ __global__ void __launch_bounds__(kSpmmThreads, ROWMAJOR ? 4 : 5) group_spmm_ker
         if (i + 1 < nbatch) consume(i + 1, xb);
     }
     close_groups(e1);  // trailing empty groups (gi reaches ng)
-    if (ROWMAJOR) {
-        __syncwarp();
-        const int bbase = a.b0 + blockIdx.y * NS;
-        for (int i = lane; i < NS * ng; i += 32) {  // ng consecutive lanes: the part's groups of one sequence
-            const int sq = i / ng, t = i - sq * ng;
-            if (bbase + sq < a.B) a.R[(size_t)(bbase + sq) * G.M + g0 + t] = tile[t * TS + sq];
-        }
-    } else {
-        pos.store(a.Psum + (size_t)part * a.bpad + sq0);
+    if (PSUM) pos.store(a.Psum + (size_t)part * a.bpad + sq0);
+}
+
+// out[row, g] = Rt[g, row]: the group-major sums of the sparse product as the row-major result of pcg_group_probs.
+// Grid (ceil(M / 32), ceil(rows / 32)) x (32, 8): a 32 x 32 tile through padded shared memory, both sides coalesced.
+__global__ void __launch_bounds__(256) rows_from_groups_kernel(const float *Rt, int bpad, int rows, int M, float *out) {
+    pdl_enter();
+    __shared__ float tile[32][33];
+    const int g0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int g = g0 + j, r = r0 + (int)threadIdx.x;
+        tile[j][threadIdx.x] = (g < M && r < rows) ? Rt[(size_t)g * bpad + r] : 0.f;
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int r = r0 + j, g = g0 + (int)threadIdx.x;
+        if (r < rows && g < M) out[(size_t)r * M + g] = tile[threadIdx.x][j];
     }
 }
 
@@ -1922,7 +1924,7 @@ static VerifyWorkspace carve_workspace(void *base, int64_t B, int64_t K, int64_t
         w.Pws = (float *)(p + take((size_t)(B * (K + 1) * M) * 4));
         w.Qws = (float *)(p + take((size_t)(B * K * M) * 4));
         if (draw_smem_bytes((int)M) > kMaxDynSmem) w.own_rows = (float *)(p + take((size_t)(B * M) * 4));
-        w.probs_scratch = p + take(pcg_group_probs_workspace_bytes((int32_t)V));
+        w.probs_scratch = p + take(pcg_group_probs_workspace_bytes((int32_t)V, (int32_t)M));
     } else if (mode != PCG_VERIFY_CLUSTER_TERMINAL) {
         const int64_t chunk = terminal_chunk((int)B, (int)V);
         const int64_t chunks = (B + chunk - 1) / chunk;
@@ -1966,16 +1968,16 @@ static cudaError_t launch_transpose(const TransposeArgs &tr, int nb, const Group
 }
 
 // The sparse product over nb batches of 32 sequences (nb a multiple of `lanes`, the sequences per lane: 8, 4 or 1).
-template <bool ROWMAJOR>
+template <bool PSUM>
 static cudaError_t launch_spmm(const SpmmArgs &sp, int nb, int lanes, const GroupsDev &G, cudaStream_t cs) {
     const bool has_w = G.pair_w != nullptr;
     const dim3 grid((unsigned)((G.nparts + kSpmmThreads / 32 - 1) / (kSpmmThreads / 32)), (unsigned)(nb / lanes));
     auto go = [&](auto kern) { return launch_after(kern, grid, dim3(kSpmmThreads), 0, cs, sp, G); };
-    if (lanes == 8) return has_w ? go(group_spmm_kernel<8, 4, true, ROWMAJOR>) : go(group_spmm_kernel<8, 4, false, ROWMAJOR>);
+    if (lanes == 8) return has_w ? go(group_spmm_kernel<8, 4, true, PSUM>) : go(group_spmm_kernel<8, 4, false, PSUM>);
     if (lanes == kSpmmWide)
-        return has_w ? go(group_spmm_kernel<kSpmmWide, kSpmmDepth, true, ROWMAJOR>)
-                     : go(group_spmm_kernel<kSpmmWide, kSpmmDepth, false, ROWMAJOR>);
-    return has_w ? go(group_spmm_kernel<1, 16, true, ROWMAJOR>) : go(group_spmm_kernel<1, 16, false, ROWMAJOR>);
+        return has_w ? go(group_spmm_kernel<kSpmmWide, kSpmmDepth, true, PSUM>)
+                     : go(group_spmm_kernel<kSpmmWide, kSpmmDepth, false, PSUM>);
+    return has_w ? go(group_spmm_kernel<1, 16, true, PSUM>) : go(group_spmm_kernel<1, 16, false, PSUM>);
 }
 
 #include "pcg_thinning.cuh"
@@ -1988,16 +1990,20 @@ namespace pcg {
 struct ProbsScratch {
     float4 *stats;  // [chunk]
     float *dt;      // [chunk / 32][V][32]
+    float *rt;      // [M][chunk] group-major sums of one chunk of rows
     size_t bytes;
 };
-static ProbsScratch carve_probs_scratch(void *base, int V) {
+static ProbsScratch carve_probs_scratch(void *base, int V, int M) {
     const size_t chunk = (size_t)probs_chunk_rows(V);
     ProbsScratch w;
     char *p = (char *)base;
     w.stats = (float4 *)p;
-    const size_t off = (chunk * 16 + 255) & ~(size_t)255;
+    size_t off = (chunk * 16 + 255) & ~(size_t)255;
     w.dt = (float *)(p + off);
-    w.bytes = off + (((size_t)V * chunk * 4 + 255) & ~(size_t)255);
+    off += ((size_t)V * chunk * 4 + 255) & ~(size_t)255;
+    w.rt = (float *)(p + off);
+    off += ((size_t)M * chunk * 4 + 255) & ~(size_t)255;
+    w.bytes = off;
     return w;
 }
 
@@ -2040,8 +2046,11 @@ static pcg_status group_probs_impl(const void *logits, pcg_dtype dtype, int64_t 
             tr.Dt = scratch->dt;
             PCG_DISPATCH_DTYPE(dtype, e = launch_transpose<LogitT>(tr, nb, G, groups->sm_count, cs));
             if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
-            e = launch_spmm<true>(SpmmArgs{scratch->dt, nr, 0, chunk, out + (size_t)r0 * G.M, nullptr}, nb, lanes, G, cs);
+            e = launch_spmm<false>(SpmmArgs{scratch->dt, nr, 0, chunk, scratch->rt, nullptr}, nb, lanes, G, cs);
             if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");
+            e = launch_after(rows_from_groups_kernel, dim3((unsigned)((G.M + 31) / 32), (unsigned)((nr + 31) / 32)), dim3(32, 8), 0,
+                             cs, (const float *)scratch->rt, chunk, nr, G.M, out + (size_t)r0 * G.M);
+            if (e != cudaSuccess) return cuda_fail(e, "launching rows_from_groups_kernel");
         }
         return PCG_OK;
     }
@@ -2059,12 +2068,13 @@ extern "C" pcg_status pcg_group_probs(const void *logits, pcg_dtype dtype, int64
     if (groups) {  // the scratch that belongs to the handle
         own.stats = groups->probs_stats;
         own.dt = groups->probs_dt;
+        own.rt = groups->probs_rt;
     }
     return group_probs_impl(logits, dtype, rows, temperature, groups, out, &own, (cudaStream_t)stream, "pcg_group_probs");
 }
 
-extern "C" size_t pcg_group_probs_workspace_bytes(int32_t V) {
-    return V < 1 ? 256 : carve_probs_scratch(nullptr, V).bytes;
+extern "C" size_t pcg_group_probs_workspace_bytes(int32_t V, int32_t M) {
+    return (V < 1 || M < 1) ? 256 : carve_probs_scratch(nullptr, V, M).bytes;
 }
 
 extern "C" pcg_status pcg_group_probs_ws(const void *logits, pcg_dtype dtype, int64_t rows, float temperature,
@@ -2074,12 +2084,12 @@ extern "C" pcg_status pcg_group_probs_ws(const void *logits, pcg_dtype dtype, in
         set_error("pcg_group_probs_ws: null group handle");
         return PCG_ERR_INVALID_ARG;
     }
-    const size_t need = pcg_group_probs_workspace_bytes(groups->dev.V);
+    const size_t need = pcg_group_probs_workspace_bytes(groups->dev.V, groups->dev.M);
     if (!workspace || ((uintptr_t)workspace & 255u) || workspace_bytes < need) {
         set_error("pcg_group_probs_ws: workspace must be 256-byte aligned and hold %zu bytes (got %zu)", need, workspace_bytes);
         return PCG_ERR_WORKSPACE;
     }
-    const ProbsScratch ws = carve_probs_scratch(workspace, groups->dev.V);
+    const ProbsScratch ws = carve_probs_scratch(workspace, groups->dev.V, groups->dev.M);
     return group_probs_impl(logits, dtype, rows, temperature, groups, out, &ws, (cudaStream_t)stream, "pcg_group_probs_ws");
 }
 
@@ -2155,7 +2165,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
     // ---- per-position stage: statistics, label, accept bit ----
     if (dense) {
         // P and Q of ALL groups at EVERY position, then the accept test on the stored masses
-        const ProbsScratch ps = carve_probs_scratch(w.probs_scratch, G.V);
+        const ProbsScratch ps = carve_probs_scratch(w.probs_scratch, G.V, G.M);
         pcg_status st2 = group_probs_impl(target_logits, dtype, (int64_t)B * (K + 1), temperature, groups, w.Pws, &ps, cs, "pcg_verify");
         if (st2 == PCG_OK) st2 = group_probs_impl(draft_logits, dtype, (int64_t)B * K, temperature, groups, w.Qws, &ps, cs, "pcg_verify");
         if (st2 != PCG_OK) return st2;
@@ -2210,7 +2220,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
                              w.term_stats,  w.Dt};
             PCG_DISPATCH_DTYPE(dtype, e = launch_transpose<LogitT>(tr, nb, G, groups->sm_count, cs));
             if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
-            e = launch_spmm<false>(SpmmArgs{w.Dt, B, b0, chunk, w.Rt + (size_t)ci * G.M * chunk,
+            e = launch_spmm<true>(SpmmArgs{w.Dt, B, b0, chunk, w.Rt + (size_t)ci * G.M * chunk,
                                             w.Psum + (size_t)ci * G.nparts * chunk},
                                    nb, lanes, G, cs);
             if (e != cudaSuccess) return cuda_fail(e, "launching group_spmm_kernel");

@@ -95,8 +95,8 @@ def test_workspace_queries():
     assert a >= 256 * 16 * 28 and b >= 256 and a % 256 == 0 and b % 256 == 0
     arena = lib.pcg_verify_host_arena_bytes(256, 16, 65536, 16384, 1, 0)
     assert arena >= 256 * 33 * 65536 * 2 + a
-    g = lib.pcg_group_probs_workspace_bytes(65536)
-    assert g >= 256 * 65536 * 4 and g % 256 == 0 and lib.pcg_group_probs_workspace_bytes(0) == 256
+    g = lib.pcg_group_probs_workspace_bytes(65536, 16384)
+    assert g >= 256 * (65536 + 16384) * 4 and g % 256 == 0 and lib.pcg_group_probs_workspace_bytes(0, 5) == 256
     assert lib.pcg_group_probs_ws(None, 0, 4, 1.0, None, None, None, 0, None) == 1  # null handle
     t = lib.pcg_verify_thinning_workspace_bytes(256, 16, 65536, 16384, 1)
     assert t >= 256 * 16 * 28 + 256 * 16384 * 4 and t % 256 == 0

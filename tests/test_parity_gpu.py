@@ -68,7 +68,7 @@ def test_group_probs_batched_route(oracle, name, rows):
     assert np.array_equal(again.astype(np.float64), got)  # bit-reproducible
     # the caller-workspace form: same numbers; two calls with separate workspaces on two streams do not disturb each other
     xd = logits_to_device(x)
-    ws = [torch.empty(binding.pcg_group_probs_workspace_bytes(cfg.V), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    ws = [torch.empty(binding.pcg_group_probs_workspace_bytes(cfg.V, groups.M), dtype=torch.uint8, device="cuda") for _ in range(2)]
     outs = [torch.empty((rows, groups.M), dtype=torch.float32, device="cuda") for _ in range(2)]
     streams = [torch.cuda.Stream(), torch.cuda.Stream()]
     torch.cuda.synchronize()
