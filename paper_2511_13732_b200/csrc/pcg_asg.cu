@@ -598,26 +598,34 @@ __global__ void asg_representative_kernel(const uint32_t *bits, int V, int W, co
     if (lane == 0) rep[t] = found;
 }
 
-// Exclusive prefix sum of n ints by one block (set-up sizes: n <= 2^20), total to out[n].
-__global__ void asg_scan_kernel(const int32_t *in, int n, int32_t *out) {
-    __shared__ int32_t part[1024];
-    const int tid = threadIdx.x, per = (n + 1023) / 1024;
+// Exclusive prefix sum of n ints by one block (set-up sizes: n <= 2^20), total to out[n]: a contiguous run per
+// thread, the 1024 run totals scanned by warp shuffles (32 warp scans, then one over the warps' totals).
+__global__ void __launch_bounds__(1024) asg_scan_kernel(const int32_t *in, int n, int32_t *out) {
+    __shared__ int32_t warp_tot[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, per = (n + 1023) / 1024;
     const int lo = min(n, tid * per), hi = min(n, lo + per);
     int32_t s = 0;
     for (int i = lo; i < hi; ++i) s += in[i];
-    part[tid] = s;
+    int32_t inc = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t up = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += up;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
     __syncthreads();
-    if (tid == 0) {
-        int32_t run = 0;
-        for (int i = 0; i < 1024; ++i) {
-            const int32_t v = part[i];
-            part[i] = run;
-            run += v;
+    if (warp == 0) {
+        int32_t w = warp_tot[lane], winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t up = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += up;
         }
-        out[n] = run;
+        warp_tot[lane] = winc - w;  // exclusive prefix of the warps' totals
+        if (lane == 31) out[n] = winc;
     }
     __syncthreads();
-    int32_t run = part[tid];
+    int32_t run = warp_tot[warp] + inc - s;
     for (int i = lo; i < hi; ++i) {
         const int32_t v = in[i];
         out[i] = run;
