@@ -313,17 +313,21 @@ pcg_status pcg_verify_static(const void *target_logits, const void *draft_logits
  * inside the kept group is drawn from the target-conditional p(t) w / P(k) with uniforms[b, K, 1], as in
  * pcg_verify.  The paper's loop is unbounded; this call runs at most n_trials trials per sequence and, if all
  * are turned down, draws the group from the enumerated residual with uniforms[b, K, 0] (what pcg_verify does;
- * same law) and sets PCG_FLAG_THINNING_EXHAUSTED for that sequence.  That fallback is slow -- one thread block
- * walks all nnz memberships of the sequence, 0.47 ms at V = 65536, M = 16384, nnz = 393216 on a B200, more than
- * the rest of a 256-sequence call -- whereas trials are cheap: they run side by side (8 in the first round, 16 in
- * each later one), and a further round (about 4 microseconds) is entered only by sequences whose earlier candidates were all turned down.  So supply trials
+ * same law) and sets PCG_FLAG_THINNING_EXHAUSTED for that sequence.  That fallback costs more than a trial, and how
+ * much depends on n_trials.  From 24 supplied trials on (running out is then rare) it is done by the sequence's own
+ * thread block, which walks all nnz memberships alone: 0.47 ms for one such sequence at V = 65536, M = 16384,
+ * nnz = 393216 on a B200, more than the rest of a 256-sequence call.  With fewer trials the call launches one more
+ * kernel (about 3 microseconds when it finds nothing to do) in which ALL thread blocks share the enumeration of the
+ * sequences that ran out: about 15 microseconds for one, about 10 for each further one.  Trials themselves are cheap:
+ * they run side by side (8 in the first round, 16 in each later one), and a further round (about 4 microseconds) is
+ * entered only by sequences whose earlier candidates were all turned down.  So supply trials
  * generously: a rejected sequence runs out of n_trials with probability (1 - TV(P,Q))^n_trials.  Results are a deterministic function of
  * the inputs; they equal pcg_verify's in distribution, not draw by draw (the two consume different uniforms).
  *
  *   thin_uniforms [B, n_trials, 3] float in [0,1), device, read-only; 1 <= n_trials <= 65536
  *   out_trials    [B] int32 or NULL: candidates drawn (1 after an all-accepted sequence; n_trials when exhausted)
  *   workspace     device, 256-byte aligned, at least pcg_verify_thinning_workspace_bytes(...) bytes (2076 bytes per
- *                 drafted position plus B*M*4 for sequences whose trials run out); contents need no initialisation
+ *                 drafted position plus 2*B*M*4 for sequences whose trials run out); contents need no initialisation
  *   the remaining arguments, ownership, asynchrony (no allocation, no synchronisation, the caller's stream only)
  *   and errors are pcg_verify's.  Rows that do not start on 16-byte boundaries or are not whole 16-byte words
  *   long (V * bytes per logit not a multiple of 16) give the same results, a little slower (their slot masses

@@ -117,6 +117,8 @@ struct PositionArgs {
                              // sequence's LAST drafted position if that position was accepted (no sequence that
                              // needs its bonus row can have its last position rejected)
     int32_t *bonus_flags;    // [B] flags of that row (with bonus_stats)
+    int32_t *zero_words;     // counters of a later kernel of the call that must start at zero (block 0 clears them), or null
+    int zero_count;          // how many
 };
 
 // Group-label coupling: the label of draft token x is drawn from the groups containing x (reverse membership
@@ -220,6 +222,8 @@ __global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a,
     }
     const int pos = b * K + i;
     pdl_enter();  // (the first kernel of a call: lets the kernel behind it be scheduled while this one drains)
+    if (a.zero_words && blockIdx.x == 0)  // (this grid completes before their user starts)
+        for (int k = tid; k < a.zero_count; k += NT) a.zero_words[k] = 0;
     const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + i) * V;
     const T *qrow = reinterpret_cast<const T *>(a.draft) + (int64_t)pos * V;
     const float *u = a.uniforms + ((int64_t)b * (K + 1) + i) * 2;
@@ -1524,30 +1528,21 @@ __device__ __noinline__ int slow_target_group_draw(const GroupsDev &G, const T *
     return ibox[4] >= 0 ? ibox[4] : ibox[3];
 }
 
-// One block per sequence.  The cumulative distribution over the groups is walked in two levels: the parts' sums
-// (a contiguous run of parts per thread, held in registers; prefix sums in double, block scan), then the groups
-// of the one part in which the cumulative mass passes u * Z, by the warp of the thread that owns that part, which
-// goes on to draw the token inside the group.
-template <typename T>
-__global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a, GroupsDev G) {
-    constexpr int NT = kPickThreads, PER = 16;  // PER: part sums a thread keeps in registers
-    __shared__ double dscratch[32];
-    __shared__ int ibox[8];
-    const int M = G.M, V = G.V, K = a.K, NP = G.nparts;
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // inputs of the call (not results of the kernels before): fetched before those are waited for
-    const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
-    const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
-    pdl_enter();
-    const int n = a.term_n[b];
-    int flags = a.term_flags[b];
-    const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
-    const bool residual = n < K;  // false: draw from the target's coarse distribution itself (bonus token)
-    const int c = b / a.chunk, colb = b - c * a.chunk;
-    const size_t cs = (size_t)a.chunk;
-    const float *Rt = a.Rt + (size_t)c * M * cs + colb;    // group g of this sequence: Rt[g * chunk]
-    const float *Ps = a.Psum + (size_t)c * NP * cs + colb;  // part p of this sequence: Ps[p * chunk]
-
+// Group and token of one sequence's terminal draw, by the whole block, from the sums of the parts (Ps[p * pstride])
+// and of the groups (Rt[g * rstride]).  The cumulative distribution over the groups is walked in two levels: the
+// parts' sums (a contiguous run of parts per thread, held in registers; prefix sums in double, block scan), then
+// the groups of the one part in which the cumulative mass passes u * Z, by the warp of the thread that owns that
+// part, which goes on to draw the token inside the group.  If the sums are all zero after a rejection the group is
+// drawn from the target's own masses (rs_target: the scaled reference of the target row) and the sequence flagged.
+template <typename T, int NT>
+__device__ __forceinline__ void pick_group_and_token(const GroupsDev &G, const T *trow, float s, float rs_target, bool residual,
+                                                     float u_group, float u_token, const float *Rt, size_t rstride,
+                                                     const float *Ps, size_t pstride, double *dscratch, int *ibox,
+                                                     int &flags, int &gsel, int &z) {
+    constexpr int PER = 16;  // part sums a thread keeps in registers
+    const int NP = G.nparts;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __syncthreads();  // the boxes may still be read from an earlier use
     const int per = (NP + NT - 1) / NT;
     const int p0 = min(NP, tid * per), p1 = min(NP, p0 + per);
     if (tid == 0) {
@@ -1558,7 +1553,7 @@ __global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a,
     }
     float v[PER];  // the first PER part sums of this thread's run (all of it unless there are very many parts)
 #pragma unroll
-    for (int j = 0; j < PER; ++j) v[j] = p0 + j < p1 ? Ps[(size_t)(p0 + j) * cs] : 0.f;
+    for (int j = 0; j < PER; ++j) v[j] = p0 + j < p1 ? Ps[(size_t)(p0 + j) * pstride] : 0.f;
     double my_sum = 0.0;
     int my_last = -1;  // last part with mass in this thread's run
 #pragma unroll
@@ -1567,14 +1562,15 @@ __global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a,
         if (v[j] > 0.f) my_last = p0 + j;
     }
     for (int p = p0 + PER; p < p1; ++p) {
-        const float x = Ps[(size_t)p * cs];
+        const float x = Ps[(size_t)p * pstride];
         my_sum += (double)x;
         if (x > 0.f) my_last = p;
     }
     double my_excl, my_incl, Ztot;
     block_scan<NT>(my_sum, dscratch, &my_excl, &my_incl, &Ztot);  // (its barriers publish the boxes)
 
-    int gsel = -1, z = -1;
+    gsel = -1;
+    z = -1;
     if (Ztot > 0.0) {
         // ---- group draw: first group whose inclusive prefix exceeds u * Z ----
         const double target = (double)u_group * Ztot;
@@ -1603,7 +1599,7 @@ __global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a,
                     }
                 }
                 for (int p = p0 + PER; p < p1 && !found; ++p) {
-                    const float x = Ps[(size_t)p * cs];
+                    const float x = Ps[(size_t)p * pstride];
                     if (x > 0.f && run + (double)x > target) {
                         part = p;
                         found = 1;
@@ -1619,7 +1615,7 @@ __global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a,
                 // the group inside it (lane j holds group j of the part): the running sum continues from the parts
                 // before; if no prefix passes the target (rounding), the last group with mass
                 const int g0 = G.part_ptr[part], ng = G.part_ptr[part + 1] - g0;  // at most kPartMaxGroups
-                const float r = lane < ng ? fmaxf(Rt[(size_t)(g0 + lane) * cs], 0.f) : 0.f;
+                const float r = lane < ng ? fmaxf(Rt[(size_t)(g0 + lane) * rstride], 0.f) : 0.f;
                 const int gp = lane <= ng ? G.group_ptr[g0 + lane] : 0;
                 int pick = -1, last = -1;
                 for (int j = 0; j < ng; ++j) {
@@ -1633,7 +1629,7 @@ __global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a,
                 const int j = pick >= 0 ? pick : last;
                 if (j >= 0) {
                     const int lo = __shfl_sync(0xffffffffu, gp, j), hi = __shfl_sync(0xffffffffu, gp, j + 1);
-                    const int zt = warp_token_in_range<T>(G, trow, lo, hi - lo, a.s, u_token, lane);
+                    const int zt = warp_token_in_range<T>(G, trow, lo, hi - lo, s, u_token, lane);
                     if (lane == 0) {
                         ibox[4] = g0 + j;
                         ibox[5] = zt;
@@ -1652,14 +1648,38 @@ __global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a,
     } else if (residual) {
         // a rejection whose residual vanished (P == Q to rounding): draw from P instead
         flags |= PCG_FLAG_ZERO_RESIDUAL;
-        gsel = slow_target_group_draw<T, NT>(G, trow, a.s, a.term_stats[b].x, u_group, dscratch, ibox);
-        if (gsel >= 0) z = block_token_in_group<T>(G, trow, gsel, a.s, u_token, ibox, flags);
+        gsel = slow_target_group_draw<T, NT>(G, trow, s, rs_target, u_group, dscratch, ibox);
+        if (gsel >= 0) z = block_token_in_group<T>(G, trow, gsel, s, u_token, ibox, flags);
     }
     if (gsel < 0) {  // no mass anywhere (non-finite inputs): emit group 0 / token 0 and flag it
         gsel = 0;
         z = 0;
         flags |= PCG_FLAG_NONFINITE;
     }
+}
+
+// One block per sequence: pick_group_and_token on the sums the sparse product left, then the outputs.
+template <typename T>
+__global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a, GroupsDev G) {
+    constexpr int NT = kPickThreads;
+    __shared__ double dscratch[32];
+    __shared__ int ibox[8];
+    const int M = G.M, V = G.V, K = a.K, NP = G.nparts;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    // inputs of the call (not results of the kernels before): fetched before those are waited for
+    const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
+    const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
+    pdl_enter();
+    const int n = a.term_n[b];
+    int flags = a.term_flags[b];
+    const float rs_target = a.term_stats[b].x;
+    const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
+    const int c = b / a.chunk, colb = b - c * a.chunk;
+    const size_t cs = (size_t)a.chunk;
+    const float *Rt = a.Rt + (size_t)c * M * cs + colb;    // group g of this sequence: Rt[g * chunk]
+    const float *Ps = a.Psum + (size_t)c * NP * cs + colb;  // part p of this sequence: Ps[p * chunk]
+    int gsel, z;
+    pick_group_and_token<T, NT>(G, trow, a.s, rs_target, n < K, u_group, u_token, Rt, cs, Ps, cs, dscratch, ibox, flags, gsel, z);
     emit_sequence<NT>(G, b, K, n, z, gsel, flags, a.draft_tokens, a.labels, a.out_accept_len, a.out_tokens, a.out_groups,
                       a.out_flags);
     // The transposed operand has been consumed (workspace contents are of no interest after the call):
@@ -2177,7 +2197,7 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
         // (the batched per-sequence stage takes the bonus row's statistics from this kernel)
         PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
                         w.accept,      w.labels,     w.posflags,   w.stats,  nullptr,
-                        cluster_terminal ? nullptr : w.bonus_stats, cluster_terminal ? nullptr : w.bonus_flags};
+                        cluster_terminal ? nullptr : w.bonus_stats, cluster_terminal ? nullptr : w.bonus_flags, nullptr, 0};
         launch_position(dtype, pa, G, B * K, cs);
         e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
@@ -2242,9 +2262,9 @@ extern "C" pcg_status pcg_verify(const void *target_logits, const void *draft_lo
 
 namespace pcg {
 struct ThinWorkspace {
-    int32_t *accept, *labels, *posflags;
-    float4 *stats;
-    float *fallback_rows;
+    int32_t *accept, *labels, *posflags, *exh, *exh_meta;
+    float4 *stats, *exh_stats;
+    float *fallback_rows, *exh_psum;
     float2 *strata;
     size_t bytes;
 };
@@ -2262,6 +2282,10 @@ static ThinWorkspace carve_thin_workspace(void *base, int64_t B, int64_t K, int6
     w.labels = (int32_t *)(p + take((size_t)(B * K) * 4));
     w.posflags = (int32_t *)(p + take((size_t)(B * K) * 4));
     w.fallback_rows = (float *)(p + take((size_t)(B * M) * 4));
+    w.exh_psum = (float *)(p + take((size_t)(B * M) * 4));  // (a part holds at least one group)
+    w.exh = (int32_t *)(p + take((size_t)(B + 2) * 4));
+    w.exh_meta = (int32_t *)(p + take((size_t)B * 8));
+    w.exh_stats = (float4 *)(p + take((size_t)B * 16));
     w.strata = (float2 *)(p + take((size_t)(B * K) * kPosThreads * 8));  // (128 pairs per position are used for short rows)
     w.bytes = off ? off : 256;
     return w;
@@ -2323,7 +2347,7 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
     // (t div W) mod 128), so the thinning kernel needs no pass of its own over the row.
     const bool strata = ((uintptr_t)target_logits & 15u) == 0 && ((size_t)G.V * esz) % 16 == 0;
     PositionArgs pa{target_logits, draft_logits, draft_tokens, uniforms, K, s, groups->accept_bias,
-                    w.accept,      w.labels,     w.posflags,   w.stats,  strata ? w.strata : nullptr, nullptr, nullptr};
+                    w.accept,      w.labels,     w.posflags,   w.stats,  strata ? w.strata : nullptr, nullptr, nullptr, w.exh, 2};
     launch_position(dtype, pa, G, B * K, cs);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launching position_kernel");
@@ -2334,7 +2358,8 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
     ThinArgs ta{target_logits, draft_logits, draft_tokens, uniforms,        thin_uniforms, n_trials,
                 K,             s,            w.accept,     w.labels,        w.posflags,    w.stats,
                 w.fallback_rows, out_accept_len, out_tokens, out_groups,    out_flags,     out_trials,
-                strata ? w.strata : nullptr, position_threads(G.V, dtype)};
+                strata ? w.strata : nullptr, position_threads(G.V, dtype), w.exh, w.exh_stats, w.exh_meta, w.exh_psum,
+                n_trials < kEnumBelowTrials ? 1 : 0};
     auto launch = [&](auto kern) -> cudaError_t {
         cudaError_t le = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (le != cudaSuccess) return le;
@@ -2342,6 +2367,13 @@ extern "C" pcg_status pcg_verify_thinning(const void *target_logits, const void 
     };
     PCG_DISPATCH_DTYPE(dtype, e = launch(thinning_kernel<LogitT>));
     if (e != cudaSuccess) return cuda_fail(e, "launching thinning_kernel");
+    // the shared enumeration for sequences whose trials ran out (returns at once when there is none): only where
+    // running out is likely enough to pay for the launch
+    if (ta.coop) {
+        const dim3 egrid((unsigned)((G.nparts + kEnumThreads / 32 - 1) / (kEnumThreads / 32)));
+        PCG_DISPATCH_DTYPE(dtype, e = launch_after(thinning_enumerate_kernel<LogitT>, egrid, dim3(kEnumThreads), 0, cs, ta, G));
+        if (e != cudaSuccess) return cuda_fail(e, "launching thinning_enumerate_kernel");
+    }
     if (stage_events) {
         e = cudaEventRecord((cudaEvent_t)stage_events[2], cs);
         if (e != cudaSuccess) return cuda_fail(e, "cudaEventRecord");

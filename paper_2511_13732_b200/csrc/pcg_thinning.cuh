@@ -16,11 +16,15 @@
 //      inside a kept group.  The first kept candidate in trial order wins, so the result is the sequential
 //      sampler's although several trials run side by side;
 //   4. outputs.
-// If all supplied trials are turned down, the block enumerates the residual itself (one thread per group,
-// staged in a row of the workspace) and draws from it with the sequence's terminal-group uniform: same law,
-// flagged PCG_FLAG_THINNING_EXHAUSTED.
+// If all supplied trials of a sequence are turned down, the residual is enumerated after all and the group drawn
+// from it with the sequence's terminal-group uniform: same law, flagged PCG_FLAG_THINNING_EXHAUSTED.  Calls with
+// many supplied trials (where that is rare) do it in the sequence's own block (one thread per group, staged in a
+// row of the workspace: 0.47 ms at C5).  Calls with fewer than kEnumBelowTrials trials run thinning_enumerate_kernel
+// behind this kernel (an empty launch costs them about 3 us): the exhausted sequences are put on a list and
+// enumerated by ALL its blocks (a warp per part of the groups, as in the sparse product): 15 us for one.
 
 constexpr int kThinThreads = 512;
+constexpr int kEnumBelowTrials = 24;  // that kernel is launched for calls with fewer supplied trials than this
 
 struct ThinArgs {
     const void *target;           // [B, K+1, V]
@@ -37,6 +41,13 @@ struct ThinArgs {
     int32_t *out_accept_len, *out_tokens, *out_groups, *out_flags, *out_trials;
     const float2 *strata;  // [B*K, strata_threads] (reference, sum) of every thread of the position kernel's target-row pass, or null
     int strata_threads;    // threads of a position block: kThinSlots or 2 * kThinSlots
+    // Sequences whose trials all failed are handed to thinning_enumerate_kernel (below) through these:
+    int32_t *exh;          // [2 + B], [0] and [1] zero on entry: [0] how many, [1] blocks of that kernel that are done,
+                           // [2 + j] the j-th such sequence
+    float4 *exh_stats;     // [B] (RS_p, 1/Z_p, RS_q, 1/Z_q) of its rejected position
+    int32_t *exh_meta;     // [2B] (n, flags) of the sequence
+    float *exh_psum;       // [B, nparts] part sums written by that kernel (group sums go to fallback_rows[j, M])
+    int coop;              // 1: thinning_enumerate_kernel runs behind this kernel
 };
 
 constexpr int kThinSlots = 128;  // slots of the candidate order (the interface's rule: slot of token t = (t div W) mod 128)
@@ -338,7 +349,22 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
         __syncthreads();
     }
 
-    // ---- every supplied trial was turned down: enumerate the residual and invert its CDF (same law) ----
+    // ---- every supplied trial was turned down ----
+    // With the enumeration kernel behind this one (a.coop) the sequence is handed to it: all blocks of the GPU then
+    // share its enumeration.  Without, it is enumerated right here by its own block.  (One route per call, so that
+    // a sequence's result never depends on which other sequences ran out.)
+    if (usable && gsel < 0 && a.coop) {
+        if (tid == 0) {
+            const int slot = atomicAdd(&a.exh[0], 1);
+            a.exh[2 + slot] = b;
+            a.exh_stats[b] = make_float4(rs_p, iz_p, rs_q, iz_q);
+            a.exh_meta[2 * b] = n;
+            a.exh_meta[2 * b + 1] = flags | PCG_FLAG_THINNING_EXHAUSTED;
+            if (a.out_trials) a.out_trials[b] = used;
+        }
+        return;  // (block-uniform) that kernel draws group and token and writes the sequence's outputs
+    }
+    // ---- enumerate the residual in this block and invert its CDF (same law) ----
     if (usable && gsel < 0) {
         flags |= PCG_FLAG_THINNING_EXHAUSTED;
         float *own = a.fallback_rows + (size_t)b * M;
@@ -443,5 +469,95 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
         a.out_accept_len[b] = n;
         if (a.out_flags) a.out_flags[b] = flags;
         if (a.out_trials) a.out_trials[b] = used;
+    }
+}
+
+// Enumerated residual for the sequences whose thinning trials ran out (a.exh), by the whole grid.
+// Grid: ceil(nparts / 4) blocks of 4 warps, as the sparse product.  Nothing to do (the usual case): every block
+// returns right after the wait.  Otherwise warp = one part of the groups: for every listed sequence it gathers the
+// two logits of each of its stored pairs straight from the rows (lane = pair, 32 at a time), forms
+// (p - q) w, adds the terms group by group (per-lane partial sums, then a butterfly: a fixed order), writes the
+// group sums to fallback_rows[j, g] and the sum of their positive parts to exh_psum[j, part].  The block that
+// finishes last (a counter; nobody waits for anybody) then draws group and token of every listed sequence with
+// pick_group_and_token and writes its outputs.  (A counter per sequence, so that the draws spread over the blocks,
+// was slower: 740 additions to one word per sequence.)
+constexpr int kEnumThreads = 128;
+
+template <typename T>
+__global__ void __launch_bounds__(kEnumThreads) thinning_enumerate_kernel(ThinArgs a, GroupsDev G) {
+    constexpr int NT = kEnumThreads;
+    __shared__ double dscratch[32];
+    __shared__ int ibox[8];
+    pdl_enter();
+    const int ne = a.exh[0];
+    if (ne == 0) return;
+    const int V = G.V, M = G.M, K = a.K, NP = G.nparts;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int part = blockIdx.x * (NT / 32) + warp;
+    const bool working = part < NP;  // (warp-uniform; the last block may have warps without a part)
+    const int g0 = working ? G.part_ptr[part] : 0, ng = working ? G.part_ptr[part + 1] - g0 : 0;  // at most kPartMaxGroups
+    const int ptr_l = (working && lane <= ng) ? G.group_ptr[g0 + lane] : 0;                          // lane i: group_ptr[g0 + i]
+    const int e0 = __shfl_sync(0xffffffffu, ptr_l, 0), e1 = __shfl_sync(0xffffffffu, ptr_l, ng);
+    for (int j = 0; j < ne; ++j) {
+        if (working) {
+            const int b = a.exh[2 + j];
+            const float4 st = a.exh_stats[b];
+            const int n = a.exh_meta[2 * b];
+            const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
+            const T *qrow = reinterpret_cast<const T *>(a.draft) + ((int64_t)b * K + min(n, K - 1)) * V;
+            float gsum[kPartMaxGroups];
+#pragma unroll
+            for (int gi = 0; gi < kPartMaxGroups; ++gi) gsum[gi] = 0.f;
+            for (int k0 = e0; k0 < e1; k0 += 32) {
+                const int k = k0 + lane;
+                float d = 0.f;
+                if (k < e1) {
+                    const int t = G.group_tok[k];
+                    const float w = G.pair_w ? G.pair_w[k] : G.inv_deg[t];
+                    float v = __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(trow[t]), a.s, -st.x)), st.y);
+                    v -= __fmul_rn(ex2(__fmaf_rn(Elem<T>::widen(qrow[t]), a.s, -st.z)), st.w);
+                    d = __fmul_rn(v, w);
+                }
+#pragma unroll
+                for (int gi = 0; gi < kPartMaxGroups; ++gi) {
+                    const int lo = __shfl_sync(0xffffffffu, ptr_l, gi), hi = __shfl_sync(0xffffffffu, ptr_l, gi + 1);
+                    if (gi < ng && k >= lo && k < hi) gsum[gi] += d;
+                }
+            }
+            float pos = 0.f;
+#pragma unroll
+            for (int gi = 0; gi < kPartMaxGroups; ++gi) {
+                float r = gsum[gi];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
+                if (gi < ng) {
+                    if (lane == 0) a.fallback_rows[(size_t)j * M + g0 + gi] = r;
+                    pos += fmaxf(r, 0.f);  // (P - Q)_+ ; NaN counts as 0
+                }
+            }
+            if (lane == 0) a.exh_psum[(size_t)j * NP + part] = pos;
+        }
+    }
+    // ---- the block that finishes last draws for the listed sequences (a counter; nobody waits for anybody) ----
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) ibox[7] = atomicAdd(&a.exh[1], 1);
+    __syncthreads();
+    if (ibox[7] != (int)gridDim.x - 1) return;
+    __threadfence();
+    for (int j = 0; j < ne; ++j) {
+        const int b = a.exh[2 + j];
+        const int n = a.exh_meta[2 * b];
+        int flags = a.exh_meta[2 * b + 1];
+        const float rs_p = a.exh_stats[b].x;
+        const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
+        const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
+        const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
+        int gsel, z;
+        pick_group_and_token<T, NT>(G, trow, a.s, rs_p, true, u_group, u_token, a.fallback_rows + (size_t)j * M, 1,
+                                    a.exh_psum + (size_t)j * NP, 1, dscratch, ibox, flags, gsel, z);
+        emit_sequence<NT>(G, b, K, n, z, gsel, flags, a.draft_tokens, a.labels, a.out_accept_len, a.out_tokens, a.out_groups,
+                          a.out_flags);
+        __syncthreads();
     }
 }

@@ -120,28 +120,42 @@ def test_thinning_long_accepts_small_tv_and_bonus(oracle, K):
         assert (ref.accept_len == K).any() and ref.trials.max() > 16
 
 
-def test_thinning_exhaustion_falls_back_to_the_enumerated_draw(oracle):
+@pytest.mark.parametrize("n_trials,weighted", [(3, False), (30, False), (5, True)])
+def test_thinning_exhaustion_falls_back_to_the_enumerated_draw(oracle, n_trials, weighted):
     """Keep uniforms just below one: no candidate is kept, every rejected sequence is drawn from the enumerated
-    residual with its terminal-group uniform -- which is what pcg_verify's oracle does."""
+    residual with its terminal-group uniform -- which is what pcg_verify's oracle does.  With few supplied trials
+    the first eight such sequences of the call are enumerated by a kernel of their own and the others by their own
+    blocks; with many, all by their own blocks: both routes must give the oracle's draw."""
     cfg = W.scaled(W.CONFIGS["C3"], B=40, K=5, V=6000, M=1500)
     groups = W.make_groups(cfg)
     bt = W.make_batch(cfg)
-    tu = W.make_thin_uniforms(cfg, 3)
+    w = None
+    if weighted:
+        rng = np.random.default_rng(8)
+        raw = rng.random(groups.nnz) + 0.05
+        tot = np.zeros(cfg.V)
+        np.add.at(tot, groups.group_tok, raw)
+        w = (raw / tot[groups.group_tok]).astype(np.float32)
+    w64 = None if w is None else w.astype(np.float64)
+    tu = W.make_thin_uniforms(cfg, n_trials)
     tu[:, :, 2] = np.float32(1.0 - 2.0 ** -24)
-    ref = oracle_thin(oracle, bt, groups, tu)
+    ref = oracle_thin(oracle, bt, groups, tu, weights=w64)
     plain = oracle.verify(bt.target_logits, bt.draft_logits, bt.draft_tokens, groups.group_ptr, groups.group_tok,
-                          groups.tok_degree, bt.uniforms, bt.temperature, threads=0)
+                          groups.tok_degree, bt.uniforms, bt.temperature, weights=w64, threads=0)
     rej = plain.accept_len < cfg.K
     assert rej.sum() > 10 and np.array_equal(ref.tokens[rej], plain.tokens[rej])
-    got = run_thin(bt, make_handle(groups), tu)
-    assert_thin_parity(got, ref)
-    assert np.all((got[3][rej] & EXHAUSTED) != 0) and np.all(got[4][rej] == 3)
+    handle = make_handle(groups, weights=w)
+    got = run_thin(bt, handle, tu)
+    assert_thin_parity(got, ref, max_excused=1 if weighted else 0)
+    assert np.all((got[3][rej] & EXHAUSTED) != 0) and np.all(got[4][rej] == n_trials)
     assert np.all((got[3][~rej] & EXHAUSTED) == 0)
+    again = run_thin(bt, handle, tu)  # the list order of the shared enumeration may differ from run to run; results may not
+    assert all(np.array_equal(x, y) for x, y in zip(got, again))
     # a few trials only: some sequences run out, some do not
     tu2 = W.make_thin_uniforms(cfg, 2)
-    ref2 = oracle_thin(oracle, bt, groups, tu2)
-    got2 = run_thin(bt, make_handle(groups), tu2)
-    assert_thin_parity(got2, ref2)
+    ref2 = oracle_thin(oracle, bt, groups, tu2, weights=w64)
+    got2 = run_thin(bt, handle, tu2)
+    assert_thin_parity(got2, ref2, max_excused=1 if weighted else 0)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
