@@ -66,7 +66,7 @@ struct pcg_groups {
     // probs_chunk; the transposed operand Dt[V, probs_chunk] and per-row statistics
     int probs_chunk;
     float *probs_dt;
-    float4 *probs_stats;
+    float4 *probs_stats;  // [probs_stats_rows]
     float *probs_rt;  // [M, probs_chunk] group-major sums of one chunk
 };
 
@@ -84,6 +84,10 @@ inline int probs_chunk_rows(int V) {
     const int64_t fit = ((int64_t)64 << 20) / ((int64_t)V * 4) / 128 * 128;
     return (int)(fit < 128 ? 128 : (fit > 256 ? 256 : fit));
 }
+
+// Rows whose softmax statistics the batched route forms in ONE launch ahead of their chunks (a launch per chunk
+// of 128 or 256 rows leaves most of the GPU idle): sixteen chunks.
+inline int probs_stats_rows(int V) { return 16 * probs_chunk_rows(V); }
 
 // Runs `...` with LogitT bound to the element type of `dtype` (float, uint16_t for bfloat16 bit patterns, f16_t).
 #define PCG_DISPATCH_DTYPE(dtype, ...)        \

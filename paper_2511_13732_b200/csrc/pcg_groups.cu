@@ -313,7 +313,7 @@ extern "C" pcg_status pcg_groups_create(const pcg_csr *csr, int slices_hint, pcg
     const size_t o_part = cv.take(part_ptr.size() * 4), o_pent = cv.take(part_ent.size() * 4);
     // scratch of the batched route of pcg_group_probs: 128 rows per chunk, more while Dt stays within 64 MB
     const int probs_chunk = probs_chunk_rows(V);
-    const size_t o_pdt = cv.take((size_t)V * probs_chunk * 4), o_pst = cv.take((size_t)probs_chunk * 16);
+    const size_t o_pdt = cv.take((size_t)V * probs_chunk * 4), o_pst = cv.take((size_t)probs_stats_rows(V) * 16);
     const size_t o_prt = cv.take((size_t)M * probs_chunk * 4);
     const size_t total = cv.off ? cv.off : 256;
     void *mem = nullptr;

@@ -2008,7 +2008,7 @@ using namespace pcg;
 
 namespace pcg {
 struct ProbsScratch {
-    float4 *stats;  // [chunk]
+    float4 *stats;  // [probs_stats_rows]
     float *dt;      // [chunk / 32][V][32]
     float *rt;      // [M][chunk] group-major sums of one chunk of rows
     size_t bytes;
@@ -2018,7 +2018,7 @@ static ProbsScratch carve_probs_scratch(void *base, int V, int M) {
     ProbsScratch w;
     char *p = (char *)base;
     w.stats = (float4 *)p;
-    size_t off = (chunk * 16 + 255) & ~(size_t)255;
+    size_t off = ((size_t)probs_stats_rows(V) * 16 + 255) & ~(size_t)255;
     w.dt = (float *)(p + off);
     off += ((size_t)V * chunk * 4 + 255) & ~(size_t)255;
     w.rt = (float *)(p + off);
@@ -2048,12 +2048,17 @@ static pcg_status group_probs_impl(const void *logits, pcg_dtype dtype, int64_t 
         // many rows: the same transposed-operand / sparse-product kernels as the per-sequence stage of pcg_verify,
         // a chunk of rows at a time through the scratch (row statistics, then p(t) w in place of p - q)
         const int chunk = probs_chunk_rows(G.V);  // a multiple of 128
+        const int stats_rows = probs_stats_rows(G.V);
         for (int64_t r0 = 0; r0 < rows; r0 += chunk) {
             const int nr = (int)std::min<int64_t>(chunk, rows - r0);
             const char *base = (const char *)logits + (size_t)r0 * G.V * dtype_bytes(dtype);
-            PCG_DISPATCH_DTYPE(dtype, e = launch_after(row_stats_kernel<LogitT>, dim3((unsigned)nr), dim3(kPrepThreads), 0, cs,
-                                                       (const void *)base, s, scratch->stats, G));
-            if (e != cudaSuccess) return cuda_fail(e, "launching row_stats_kernel");
+            const int64_t rs = r0 % stats_rows;  // this chunk's place in the statistics of its run of chunks
+            if (rs == 0) {  // the statistics of the next stats_rows rows, one block per row
+                const int ns = (int)std::min<int64_t>(stats_rows, rows - r0);
+                PCG_DISPATCH_DTYPE(dtype, e = launch_after(row_stats_kernel<LogitT>, dim3((unsigned)ns), dim3(kPrepThreads), 0, cs,
+                                                           (const void *)base, s, scratch->stats, G));
+                if (e != cudaSuccess) return cuda_fail(e, "launching row_stats_kernel");
+            }
             const int lanes = (chunk % 256 == 0 && nr >= 256) ? 8 : kSpmmWide;      // rows per lane of the sparse product
             const int nb = (nr + 32 * lanes - 1) / (32 * lanes) * lanes;          // batches of 32 rows, whole warps of it
             // every row is "a sequence whose only row is accepted": K = 0 makes the kernel form p alone
@@ -2062,7 +2067,7 @@ static pcg_status group_probs_impl(const void *logits, pcg_dtype dtype, int64_t 
             tr.B = nr;
             tr.s = s;
             tr.from_accept = 2;
-            tr.term_stats = scratch->stats;
+            tr.term_stats = scratch->stats + rs;
             tr.Dt = scratch->dt;
             PCG_DISPATCH_DTYPE(dtype, e = launch_transpose<LogitT>(tr, nb, G, groups->sm_count, cs));
             if (e != cudaSuccess) return cuda_fail(e, "launching residual_transpose_kernel");
