@@ -1224,7 +1224,6 @@ struct SeqVec<8> {  // one 256-bit load per lane
 // turns Rt into its row-major output with rows_from_groups_kernel).
 template <int SPL, int DEPTH, bool HAS_W, bool PSUM>
 __global__ void __launch_bounds__(kSpmmThreads, 5) group_spmm_kernel(SpmmArgs a, GroupsDev G) {
-    pdl_enter();
     constexpr int NS = 32 * SPL;  // sequences per warp
     static_assert(32 % DEPTH == 0 && DEPTH <= 16, "a batch never straddles two blocks of 32 token ids");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -1251,6 +1250,12 @@ __global__ void __launch_bounds__(kSpmmThreads, 5) group_spmm_kernel(SpmmArgs a,
     float w_cur, w_nxt;
     load_ids(0, ids_cur, w_cur);
     load_ids(1, ids_nxt, w_nxt);
+    // Everything above reads the handle's tables only, so it runs while the kernel before (which wrote Dt) drains.
+    // The kernel behind this one is released only AFTER the wait: once its blocks run, the kernel that wrote Dt --
+    // and with it the terminal positions and their statistics -- is known to have completed, and those may be read
+    // ahead of that kernel's own wait (terminal_pick_kernel does).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
     // issue the loads of batch i (its ids live in ids_cur if it belongs to block `blk_cur`, else in ids_nxt)
     int blk_cur = 0;
     auto issue = [&](int i, SeqVec<SPL>(&x)[DEPTH]) {
@@ -1552,8 +1557,11 @@ __device__ __forceinline__ void pick_group_and_token(const GroupsDev &G, const T
         ibox[5] = -1;  // drawn token
     }
     float v[PER];  // the first PER part sums of this thread's run (all of it unless there are very many parts)
+    int pp[PER + 1];  // ... and those parts' group bounds, fetched in the same round trip (one dependent load less later)
 #pragma unroll
     for (int j = 0; j < PER; ++j) v[j] = p0 + j < p1 ? Ps[(size_t)(p0 + j) * pstride] : 0.f;
+#pragma unroll
+    for (int j = 0; j <= PER; ++j) pp[j] = p0 + j <= p1 ? G.part_ptr[p0 + j] : 0;
     double my_sum = 0.0;
     int my_last = -1;  // last part with mass in this thread's run
 #pragma unroll
@@ -1583,7 +1591,7 @@ __device__ __forceinline__ void pick_group_and_token(const GroupsDev &G, const T
             // the part: the first of the owner's run whose prefix passes the target; if rounding left none, the
             // last part with mass (of the run, or of all parts)
             int part = ibox[3];
-            int found = 0;
+            int found = 0, pg0 = -1, pg1 = -1;  // (group bounds of the part, if they are among the prefetched ones)
             double run = my_excl;
             if (tid == owner && !none) {
                 part = my_last;
@@ -1592,6 +1600,8 @@ __device__ __forceinline__ void pick_group_and_token(const GroupsDev &G, const T
                     if (!found) {
                         if (v[j] > 0.f && run + (double)v[j] > target) {
                             part = p0 + j;
+                            pg0 = pp[j];
+                            pg1 = pp[j + 1];
                             found = 1;
                         } else {
                             run += (double)v[j];
@@ -1611,10 +1621,13 @@ __device__ __forceinline__ void pick_group_and_token(const GroupsDev &G, const T
             part = __shfl_sync(0xffffffffu, part, owner & 31);
             found = __shfl_sync(0xffffffffu, found, owner & 31);
             run = __shfl_sync(0xffffffffu, run, owner & 31);
+            pg0 = __shfl_sync(0xffffffffu, pg0, owner & 31);
+            pg1 = __shfl_sync(0xffffffffu, pg1, owner & 31);
             if (part >= 0) {
                 // the group inside it (lane j holds group j of the part): the running sum continues from the parts
                 // before; if no prefix passes the target (rounding), the last group with mass
-                const int g0 = G.part_ptr[part], ng = G.part_ptr[part + 1] - g0;  // at most kPartMaxGroups
+                const int g0 = pg0 >= 0 ? pg0 : G.part_ptr[part];
+                const int ng = (pg0 >= 0 ? pg1 : G.part_ptr[part + 1]) - g0;  // at most kPartMaxGroups
                 const float r = lane < ng ? fmaxf(Rt[(size_t)(g0 + lane) * rstride], 0.f) : 0.f;
                 const int gp = lane <= ng ? G.group_ptr[g0 + lane] : 0;
                 int pick = -1, last = -1;
@@ -1669,10 +1682,13 @@ __global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a,
     // inputs of the call (not results of the kernels before): fetched before those are waited for
     const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
     const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
-    pdl_enter();
+    // the terminal position and its statistics were left by the transposed-operand kernel, which has completed
+    // by the time a block of this kernel runs (the sparse product between the two releases its dependents only
+    // after its own wait): read ahead of the wait as well
     const int n = a.term_n[b];
     int flags = a.term_flags[b];
     const float rs_target = a.term_stats[b].x;
+    pdl_enter();
     const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
     const int c = b / a.chunk, colb = b - c * a.chunk;
     const size_t cs = (size_t)a.chunk;
