@@ -1017,6 +1017,17 @@ __device__ __forceinline__ void ld_stream_32(const void *p, uint32_t (&w)[8]) {
                  : "l"(p));
 }
 
+// A store whose line should be the last to leave the L2: Dt is read back about six times per line by the sparse
+// product, and lines of it that were pushed out in between went to DRAM and came back (about 20 MB per call before).
+__device__ __forceinline__ uint64_t l2_evict_last_policy() {
+    uint64_t pol;
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void st_keep(float *p, float v, uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(p), "f"(v), "l"(pol) : "memory");
+}
+
 // Grid (blocks per batch, batches of 32 sequences); block = 8 warps.  LANE = SEQUENCE throughout: a lane reads
 // 64 bytes of its own sequence's two rows per step (two whole sectors, one DRAM access: with 32 bytes per step a
 // third more bytes than needed came from DRAM; the eight warps of a block take neighbouring steps, so a row is
@@ -1102,6 +1113,7 @@ __global__ void __launch_bounds__(kTrThreads, 2) residual_transpose_kernel(Trans
     const int step_lo = (int)(((int64_t)nsteps * blockIdx.x) / gridDim.x);
     const int step_hi = (int)(((int64_t)nsteps * (blockIdx.x + 1)) / gridDim.x);
     float *dst = a.Dt + ((size_t)blockIdx.y * V) * 32 + lane;
+    const uint64_t keep = l2_evict_last_policy();
 
     auto fetch = [&](int step, uint32_t(&wp)[WPS], uint32_t(&wq)[WPS]) {
         const int t = step * CH;
@@ -1155,7 +1167,7 @@ __global__ void __launch_bounds__(kTrThreads, 2) residual_transpose_kernel(Trans
                 float v = __fmul_rn(ex2(__fmaf_rn(lp[e], a.s, -st.x)), st.y);
                 v -= __fmul_rn(ex2(__fmaf_rn(lq[e], a.s, -st.z)), st.w);
                 const int r = t + j * PW + e;
-                if (r < V) dst[(size_t)r * 32] = __fmul_rn(v, inv[j * PW + e]);
+                if (r < V) st_keep(dst + (size_t)r * 32, __fmul_rn(v, inv[j * PW + e]), keep);
             }
         }
     };
