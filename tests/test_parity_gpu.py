@@ -93,6 +93,24 @@ def test_group_probs_batched_route(oracle, name, rows):
     np.testing.assert_allclose(got_w, want_w, rtol=1e-5, atol=1e-37)
 
 
+def test_group_probs_past_one_run_of_row_statistics(oracle):
+    """The batched route forms the softmax statistics of sixteen chunks of rows (4096 rows at this size) in one launch;
+    4396 rows reach into a second run, whose chunks must pick up their own statistics."""
+    from paper_2511_13732_b200 import binding
+
+    cfg = W.scaled(W.CONFIGS["C3"], V=1500, M=200, emb_dim=16)
+    groups = W.make_groups(cfg)
+    rows = 4096 + 300
+    bt = W.make_batch(cfg, B=rows // cfg.K + 1)
+    x = np.ascontiguousarray(bt.draft_logits.reshape(-1, cfg.V)[:rows])
+    want = oracle.group_probs(x, groups.group_ptr, groups.group_tok, groups.tok_degree, cfg.temperature)
+    h = make_handle(groups)
+    got = binding.pcg_group_probs(logits_to_device(x), h, cfg.temperature).cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(got, want, rtol=1e-3, atol=1e-37)
+    assert np.max(np.abs(got - want) / np.maximum(want, 1e-37)) < 1e-5
+    np.testing.assert_allclose(got.sum(axis=1), 1.0, rtol=4e-6)
+
+
 @pytest.mark.parametrize("hint", [1, 2, 4, 8])
 def test_group_probs_any_slicing(oracle, hint):
     from paper_2511_13732_b200 import binding
