@@ -1692,14 +1692,16 @@ __global__ void __launch_bounds__(kPickThreads) terminal_pick_kernel(PickArgs a,
     const int M = G.M, V = G.V, K = a.K, NP = G.nparts;
     const int b = blockIdx.x, tid = threadIdx.x;
     // inputs of the call (not results of the kernels before): fetched before those are waited for
-    const float u_group = a.uniforms[((int64_t)b * (K + 1) + K) * 2];
-    const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
+    // (everything read ahead of the wait is read from L2, not through the L1: a line an earlier kernel left in this
+    // SM's L1 must not stand in for what was written since)
+    const float u_group = __ldcg(a.uniforms + ((int64_t)b * (K + 1) + K) * 2);
+    const float u_token = __ldcg(a.uniforms + ((int64_t)b * (K + 1) + K) * 2 + 1);
     // the terminal position and its statistics were left by the transposed-operand kernel, which has completed
     // by the time a block of this kernel runs (the sparse product between the two releases its dependents only
     // after its own wait): read ahead of the wait as well
-    const int n = a.term_n[b];
-    int flags = a.term_flags[b];
-    const float rs_target = a.term_stats[b].x;
+    const int n = __ldcg(a.term_n + b);
+    int flags = __ldcg(a.term_flags + b);
+    const float rs_target = __ldcg(&a.term_stats[b].x);
     pdl_enter();
     const T *trow = reinterpret_cast<const T *>(a.target) + ((int64_t)b * (K + 1) + n) * V;
     const int c = b / a.chunk, colb = b - c * a.chunk;

@@ -107,10 +107,10 @@ __global__ void __launch_bounds__(kThinThreads, 2) thinning_kernel(ThinArgs a, G
     float u_first[3] = {0.f, 0.f, 0.f};
     if (warp < a.n_trials) {
 #pragma unroll
-        for (int j = 0; j < 3; ++j) u_first[j] = tu[3 * warp + j];
+        for (int j = 0; j < 3; ++j) u_first[j] = __ldcg(tu + 3 * warp + j);  // (from L2: ahead of the wait nothing vouches for this SM's L1)
     }
-    const float u_token = a.uniforms[((int64_t)b * (K + 1) + K) * 2 + 1];
-    const int pre_tok = tid < K ? a.draft_tokens[b * K + tid] : -1;  // for the emission at the end
+    const float u_token = __ldcg(a.uniforms + ((int64_t)b * (K + 1) + K) * 2 + 1);
+    const int pre_tok = tid < K ? __ldcg(a.draft_tokens + b * K + tid) : -1;  // for the emission at the end
     pdl_enter();  // everything above may overlap the tail of the position kernel; none of its results is read before here
 
     // ---- 1. first rejected position and the flags of the positions up to it ----
