@@ -74,6 +74,17 @@ def hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def hold_device(torch, ms: float) -> float:
+    """Enqueues a device-side delay of about `ms` milliseconds on the current stream (torch's spin kernel; nothing
+    of it lies inside a timed region).  Returns the delay asked for, 0.0 if the kernel is not available."""
+    try:
+        khz = torch.cuda.get_device_properties(torch.cuda.current_device()).clock_rate  # kHz
+        torch.cuda._sleep(int(ms * khz))
+        return ms
+    except Exception:
+        return 0.0
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs (read-only)."""
 
@@ -451,6 +462,11 @@ def main():
     barrier()
     sampler = ClockSampler(physical_gpu_index(local_rank), period_s=0.002).start()
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # After the barrier the device is idle: without more ado the start event would fire at once and the region
+    # would open with the host's latency of issuing the first step (0.1 ms, i.e. 5 us per step of a 20-step run).
+    # A short device-side delay ahead of the start event lets the first steps queue up behind it, so that the region
+    # holds the device time of K steps, as it does by itself in a long run.
+    hold_ms = hold_device(torch, 0.4)
     t_begin.record()
     for i in range(args.steps):
         step()
@@ -638,6 +654,10 @@ def main():
                          "whole_call": {"achieved": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9,
                                         "frac": B * (2 * K + 1) * V * esz / (ms_step * 1e-3) / 1e9 / peak,
                                         "counted_bytes_per_step": B * (2 * K + 1) * V * esz, "ms_per_step": ms_step}},
+            "timing": {"events": "CUDA events on the launching stream around the K steps",
+                       "device_hold_before_start_event_ms": hold_ms,
+                       "why": "the device is idle after the barrier; the hold lets the first steps queue up, so the "
+                              "region holds K steps of device work and not the host's latency of issuing the first one"},
             "stages_ms": {"per_position_stage": pos_ms, "per_sequence_stage": term_ms,
                           "samples": STAGE_STEPS, "sampled": "on a separate loop of steps after the timed region"},
             "mode": args.mode + (" (per-sequence stage: " + ("cluster" if default_is_cluster else "batched") + ")"
