@@ -55,6 +55,7 @@ constexpr size_t kPosSmallRowBytes = 64 * 1024;
 constexpr int kBatch = 4;
 constexpr float kRefInit = -1.0e30f;     // "no logit seen yet": finite, so that -inf logits give 2^-inf = 0, not NaN
 constexpr float kVecSumLimit = 4294967296.f;  // 2^32
+constexpr float kRunSumLimit = 1.8446744e19f;  // 2^64: a thread's unchecked running sum beyond it is formed again, checked
 
 struct RefSum {
     float rs;   // scaled reference: the exponent subtracted from l*s
@@ -86,6 +87,32 @@ __device__ __forceinline__ void absorb(RefSum &st, const float (&v)[NV], float s
         st.acc += vs;
     else  // reference too low for this vector (always so for a thread's first vector): raise it and redo
         absorb_slow<NV>(st, v, s);
+}
+
+// The same without the check: the sum is added as it is.  A vector far above the reference makes the running sum
+// huge, infinite or NaN, and it stays so: the caller tests the sum once per row (kRunSumLimit) and, if it left the
+// safe range, forms the thread's sum again with absorb.  A sum that is large but inside the range is as exact as any
+// other (floating point); the limit keeps the 256 threads' sums of a row from overflowing when they are merged.
+template <int NV>
+__device__ __forceinline__ void absorb_unchecked(RefSum &st, const float (&v)[NV], float s) {
+    float vs = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) vs += ex2(__fmaf_rn(v[i], s, -st.rs));
+    st.acc += vs;
+}
+
+// A thread's whole vectors of a row once more, every sum checked (out of line: rare, and the streaming loop keeps
+// its registers).
+template <typename T>
+__device__ __noinline__ float2 redo_vectors(const uint4 *vp, int count, int stride, float s) {
+    constexpr int NV = Elem<T>::kPerVec;
+    RefSum st{kRefInit * s, 0.f};
+    for (int k = 0; k < count; ++k) {
+        float v[NV];
+        Elem<T>::unpack(ld_stream(vp + (size_t)k * stride), v);
+        absorb<NV>(st, v, s);
+    }
+    return make_float2(st.rs, st.acc);
 }
 
 __device__ __forceinline__ void absorb1(RefSum &st, float l, float s) {
@@ -291,6 +318,18 @@ __global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a,
         const int nfull = nvec / (NT * U);  // batches in which every thread has all U vectors
         const uint4 *p = reinterpret_cast<const uint4 *>(row + head) + tid;
         uint4 nxt[U];
+        // The reference of a thread is set by its first vector (as the checked form does when that vector's sum
+        // overflows against the initial reference); the batches are then summed without a branch per vector: the
+        // branch kept the exponentials of one vector from overlapping the next one's (4 us of the kernel at
+        // B = 256, K = 16, V = 65536).
+        if (nfull > 0) {
+            float v[NV];
+            Elem<T>::unpack(cur[0], v);
+            float vm = v[0];
+#pragma unroll
+            for (int i = 1; i < NV; ++i) vm = fmaxf(vm, v[i]);
+            if (vm > kNegInf) st.rs = vm * s;
+        }
         for (int bi = 0; bi < nfull; ++bi) {
             p += NT * U;
             if (bi + 1 < nfull) {
@@ -305,10 +344,15 @@ __global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a,
             for (int j = 0; j < U; ++j) {
                 float v[NV];
                 Elem<T>::unpack(cur[j], v);
-                absorb<NV>(st, v, s);
+                absorb_unchecked<NV>(st, v, s);
             }
 #pragma unroll
             for (int j = 0; j < U; ++j) cur[j] = nxt[j];
+        }
+        if (!(st.acc <= kRunSumLimit)) {  // (rare: a later vector far above the thread's reference, or NaN) this thread's vectors again, checked
+            const float2 r = redo_vectors<T>(reinterpret_cast<const uint4 *>(row + head) + tid, nfull * U, NT, s);
+            st.rs = r.x;
+            st.acc = r.y;
         }
         // remaining whole vectors (fewer than NT*U), then the scalar head and tail
         for (int idx = nfull * NT * U + tid; idx < nvec; idx += NT) {

@@ -511,3 +511,38 @@ def test_full_size_bench_configuration_on_sampled_sequences(oracle, mode):
                   bt.temperature, bt.dtype)
     ref = run_oracle(oracle, sub, groups)
     _assert_parity((n[sample], tok[sample], grp[sample], flg[sample]), ref)
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_rows_that_rise_far_above_their_start(oracle, dtype, mode):
+    """The streaming kernel sums a thread's vectors against the reference its FIRST vector set and checks the
+    running sum once per row; a row whose logits climb by hundreds of nats makes that sum overflow (or exceed the
+    limit) in most threads, which then form their sums again with the reference raised as they go.  Rising,
+    falling and saw-tooth rows, against the oracle."""
+    cfg = W.scaled(W.CONFIGS["C3"], B=9, K=3, V=20000, M=3000, emb_dim=16, dtype=dtype)
+    groups = W.make_groups(cfg)
+    bt = W.make_batch(cfg)
+    rng = np.random.default_rng(77)
+    t = np.arange(cfg.V, dtype=np.float64) / cfg.V
+    shapes = [-300.0 + 600.0 * t, 300.0 - 600.0 * t, 250.0 * np.abs(((7.0 * t) % 2.0) - 1.0) - 125.0]
+
+    def reshape(a, scale):
+        rows = a.shape[0] * a.shape[1]
+        out = np.empty((rows, cfg.V), np.float64)
+        for r in range(rows):
+            out[r] = scale * shapes[r % 3] + 2.0 * rng.standard_normal(cfg.V)
+        out = out.reshape(a.shape).astype(np.float32)
+        return W.f32_to_bf16_bits(out) if dtype == "bf16" else out
+
+    tl, dl = reshape(bt.target_logits, 1.0), reshape(bt.draft_logits, 0.97)
+    # drafted tokens among the 200 likeliest of their draft row (a token of vanishing mass has no float32 ratio to test)
+    dl32 = W.bf16_bits_to_f32(dl) if dtype == "bf16" else dl
+    x = np.empty_like(bt.draft_tokens)
+    for b in range(cfg.B):
+        for i in range(cfg.K):
+            x[b, i] = rng.choice(np.argpartition(-dl32[b, i], 200)[:200])
+    hard = W.Batch(tl, dl, x, bt.uniforms, bt.temperature, dtype)
+    ref = run_oracle(oracle, hard, groups)
+    got = run_verify(hard, make_handle(groups), mode=mode)
+    _assert_parity(got, ref, max_excused=1)
+    assert np.all(got[3] == 0)
