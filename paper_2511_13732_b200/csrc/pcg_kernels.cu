@@ -101,20 +101,6 @@ __device__ __forceinline__ void absorb_unchecked(RefSum &st, const float (&v)[NV
     st.acc += vs;
 }
 
-// A thread's whole vectors of a row once more, every sum checked (out of line: rare, and the streaming loop keeps
-// its registers).
-template <typename T>
-__device__ __noinline__ float2 redo_vectors(const uint4 *vp, int count, int stride, float s) {
-    constexpr int NV = Elem<T>::kPerVec;
-    RefSum st{kRefInit * s, 0.f};
-    for (int k = 0; k < count; ++k) {
-        float v[NV];
-        Elem<T>::unpack(ld_stream(vp + (size_t)k * stride), v);
-        absorb<NV>(st, v, s);
-    }
-    return make_float2(st.rs, st.acc);
-}
-
 __device__ __forceinline__ void absorb1(RefSum &st, float l, float s) {
     const float v[1] = {l};
     absorb<1>(st, v, s);
@@ -350,9 +336,14 @@ __global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a,
             for (int j = 0; j < U; ++j) cur[j] = nxt[j];
         }
         if (!(st.acc <= kRunSumLimit)) {  // (rare: a later vector far above the thread's reference, or NaN) this thread's vectors again, checked
-            const float2 r = redo_vectors<T>(reinterpret_cast<const uint4 *>(row + head) + tid, nfull * U, NT, s);
-            st.rs = r.x;
-            st.acc = r.y;
+            st = RefSum{kRefInit * s, 0.f};
+            const uint4 *vp = reinterpret_cast<const uint4 *>(row + head) + tid;
+#pragma unroll 1
+            for (int k = 0; k < nfull * U; ++k) {  // (not unrolled, and not a call: either cost the loop above registers)
+                float v[NV];
+                Elem<T>::unpack(ld_stream(vp + (size_t)k * NT), v);
+                absorb<NV>(st, v, s);
+            }
         }
         // remaining whole vectors (fewer than NT*U), then the scalar head and tail
         for (int idx = nfull * NT * U + tid; idx < nvec; idx += NT) {
