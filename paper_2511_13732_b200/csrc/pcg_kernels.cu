@@ -316,15 +316,32 @@ __global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a,
             for (int i = 1; i < NV; ++i) vm = fmaxf(vm, v[i]);
             if (vm > kNegInf) st.rs = vm * s;
         }
-        for (int bi = 0; bi < nfull; ++bi) {
+        // the batches during which the chain advances, then the rest in a loop of their own, free of the chain's test
+        // and dispatch (1.6 us of the kernel at B = 256, K = 16, V = 65536)
+        const int nchain = min(nfull, kChainSteps - min(chained, kChainSteps));
+        int bi = 0;
+        for (; bi < nchain; ++bi) {
             p += NT * U;
             if (bi + 1 < nfull) {
 #pragma unroll
                 for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * NT, pol);
             }
-            if (chained < kChainSteps) {
-                if (chain_warp) chain(chained);
-                ++chained;
+            if (chain_warp) chain(chained);
+            ++chained;
+#pragma unroll
+            for (int j = 0; j < U; ++j) {
+                float v[NV];
+                Elem<T>::unpack(cur[j], v);
+                absorb_unchecked<NV>(st, v, s);
+            }
+#pragma unroll
+            for (int j = 0; j < U; ++j) cur[j] = nxt[j];
+        }
+        for (; bi < nfull; ++bi) {
+            p += NT * U;
+            if (bi + 1 < nfull) {
+#pragma unroll
+                for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * NT, pol);
             }
 #pragma unroll
             for (int j = 0; j < U; ++j) {
