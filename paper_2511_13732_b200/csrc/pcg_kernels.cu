@@ -322,7 +322,7 @@ __global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a,
         int bi = 0;
         for (; bi < nchain; ++bi) {
             p += NT * U;
-            if (bi + 1 < nfull) {
+            if (bi + 1 < nfull) {  // (making these loads unconditional as in the second loop costs registers: spills)
 #pragma unroll
                 for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * NT, pol);
             }
@@ -337,12 +337,10 @@ __global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a,
 #pragma unroll
             for (int j = 0; j < U; ++j) cur[j] = nxt[j];
         }
-        for (; bi < nfull; ++bi) {
+        for (; bi + 1 < nfull; ++bi) {  // every batch but the last: the next one's loads go out unconditionally
             p += NT * U;
-            if (bi + 1 < nfull) {
 #pragma unroll
-                for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * NT, pol);
-            }
+            for (int j = 0; j < U; ++j) nxt[j] = ld_stream(p + j * NT, pol);
 #pragma unroll
             for (int j = 0; j < U; ++j) {
                 float v[NV];
@@ -351,6 +349,14 @@ __global__ void __launch_bounds__(NT, 1024 / NT) position_kernel(PositionArgs a,
             }
 #pragma unroll
             for (int j = 0; j < U; ++j) cur[j] = nxt[j];
+        }
+        if (bi < nfull) {  // the last batch
+#pragma unroll
+            for (int j = 0; j < U; ++j) {
+                float v[NV];
+                Elem<T>::unpack(cur[j], v);
+                absorb_unchecked<NV>(st, v, s);
+            }
         }
         if (!(st.acc <= kRunSumLimit)) {  // (rare: a later vector far above the thread's reference, or NaN) this thread's vectors again, checked
             st = RefSum{kRefInit * s, 0.f};
